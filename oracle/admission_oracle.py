@@ -1,0 +1,93 @@
+"""CPU oracle of the single-admission decision (paper Algorithm 1) and the per-SM
+utilisation registers (paper Section 3.3).  TEST INFRASTRUCTURE ONLY: the GPU
+library never imports or calls this.
+
+The steps follow the algorithm in the paper's order and notation:
+
+  state per SM j : CTA_count(k, j), U_TC[j], U_ALU[j], U_MEM[j]   (8-bit, cap U_max = 255)
+  per kernel k   : tau(k) = (tau_TC, tau_ALU, tau_MEM), each 0..15; pending(k); Feasible(k, j)
+
+  Phase 1: the first pending kernel, in dispatcher order, that has no CTA on SM j
+           and is feasible, is admitted; return.
+  Phase 2: otherwise, among pending feasible kernels, the one with the largest
+           s = sum_x (U_max - U_x[j]) * tau_x(k), strict '>' so ties keep the
+           first seen; admit it (or nothing when none is feasible).
+  Admit  : CTA_count += 1, U_x += tau_x (capped at U_max).
+  Completion: CTA_count -= 1, U_x -= tau_x.
+
+Reading of an ambiguity: the listing scans "in dispatcher order" while the prose
+of Section 3.4.1 says Phase 1 "picks one by round-robin".  ``rr_start`` lets the
+caller rotate the start of the Phase-1 scan; rr_start = 0 is the listing as
+printed.
+
+Pins: tests/test_admission_oracle.py (hand-derived decision sequence, the
+paper's arithmetic identities 17 x 15 = 255 and 24 + 12 = 36 bits, invariants).
+"""
+from __future__ import annotations
+
+U_MAX = 255
+TAU_MAX = 15
+
+
+class SMState:
+    def __init__(self, n_kernels: int):
+        self.cta_count = [0] * n_kernels
+        self.u = [0, 0, 0]                  # U_TC, U_ALU, U_MEM
+
+    def copy(self):
+        s = SMState(len(self.cta_count))
+        s.cta_count = list(self.cta_count)
+        s.u = list(self.u)
+        return s
+
+
+def score(state: SMState, tau) -> int:
+    """s = sum over pipelines of headroom times intensity."""
+    return sum((U_MAX - state.u[x]) * tau[x] for x in range(3))
+
+
+def admit(state: SMState, k: int, tau) -> None:
+    state.cta_count[k] += 1
+    for x in range(3):
+        state.u[x] = min(U_MAX, state.u[x] + tau[x])
+
+
+def complete(state: SMState, k: int, tau) -> None:
+    state.cta_count[k] -= 1
+    for x in range(3):
+        state.u[x] = max(0, state.u[x] - tau[x])
+
+
+def admission_decision(state: SMState, taus, pending, feasible, rr_start: int = 0):
+    """One invocation: returns (kernel admitted or None, phase 1|2|0) and updates ``state``.
+
+    taus[k] = (tau_TC, tau_ALU, tau_MEM); pending[k], feasible[k] booleans.
+    """
+    n = len(taus)
+    # Phase 1
+    for i in range(n):
+        k = (rr_start + i) % n
+        if not pending[k]:
+            continue
+        if state.cta_count[k] == 0 and feasible[k]:
+            admit(state, k, taus[k])
+            return k, 1
+    # Phase 2
+    best_score, best_kernel = -1, None
+    for k in range(n):
+        if not pending[k]:
+            continue
+        if not feasible[k]:
+            continue
+        s = score(state, taus[k])
+        if s > best_score:
+            best_score, best_kernel = s, k
+    if best_kernel is None:
+        return None, 0
+    admit(state, best_kernel, taus[best_kernel])
+    return best_kernel, 2
+
+
+def quantise_tau(fraction: float) -> int:
+    """Utilisation fraction of peak -> 4-bit intensity field (Section 3.2.2)."""
+    return max(0, min(TAU_MAX, int(round(TAU_MAX * fraction))))
