@@ -1,0 +1,185 @@
+/*
+ * vla.h -- C ABI of the B200 two-phase Vision-Language-Action inference library.
+ *
+ * The library serves several independent robot request streams.  Every frame of a
+ * stream goes through two phases (paper Section 2.1, Figure 1): a VLM prefill
+ * (vision patch encoder + decoder layers over image and text tokens) whose
+ * output feeds only that frame's action head, which runs a denoising loop and
+ * emits one action chunk.  The VLM phase of frame N+1 may run while the action
+ * head of frame N is still denoising (Section 2.1, "overlap"); how the two
+ * phases share the GPU is the run mode:
+ *
+ *   VLA_MODE_COSCHED    one persistent kernel, one CTA per SM; worker groups on
+ *                       each SM pull tiles from device-resident per-class queues
+ *                       under a resource-aware pick (software analogue of the
+ *                       paper's Algorithm 1 and Section 3.3 utilisation registers)
+ *   VLA_MODE_TWO_STREAM the same tile bodies launched as ordinary kernels, VLM
+ *                       nodes on stream_a and action-head nodes on stream_b, as
+ *                       CUDA graphs (the paper's "Baseline", Section 4, Fig. 7b)
+ *   VLA_MODE_SERIAL     everything on stream_a in program order (Fig. 7a)
+ *
+ * All three modes run identical tile bodies with identical tile shapes and
+ * reduction orders, so their action chunks are bit-identical.
+ *
+ * Conventions: every function returns an int status (VLA_OK = 0) and never
+ * throws or aborts.  "host" / "device" is stated per pointer.  The library owns
+ * nothing the caller passes in; it sub-allocates the caller's device arena and
+ * owns only a few pinned host buffers, which vla_destroy releases.  Calls on one
+ * context must come from one thread at a time.
+ */
+#ifndef VLA_H_
+#define VLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct vla_ctx vla_ctx; /* opaque; made by vla_init, freed by vla_destroy */
+
+enum {
+  VLA_OK = 0,
+  VLA_ERR_INVALID = 1,   /* bad argument; no side effects */
+  VLA_ERR_STATE = 2,     /* call not legal now (e.g. submit before weights are loaded) */
+  VLA_ERR_BUSY = 3,      /* the stream's frame ring is full: poll first */
+  VLA_ERR_NOT_READY = 4, /* no finished chunk for this stream yet */
+  VLA_ERR_TIMEOUT = 5,   /* a bounded device-side wait ran out (sticky) */
+  VLA_ERR_CUDA = 6,      /* a CUDA call failed (sticky) */
+  VLA_ERR_NOMEM = 7      /* arena too small or host allocation failed */
+};
+
+enum { VLA_MODE_COSCHED = 0, VLA_MODE_TWO_STREAM = 1, VLA_MODE_SERIAL = 2, VLA_MODE_MULTI_STREAM = 3 };
+/* VLA_MODE_MULTI_STREAM: like TWO_STREAM but one (VLM, head) pair of CUDA streams per
+ * request stream, created by the library; reported as extra context next to TWO_STREAM. */
+
+enum { VLA_MLP_GELU = 0, VLA_MLP_SWIGLU = 1, VLA_MLP_GEGLU = 2 };
+enum { VLA_HANDOFF_KV_LAST = 0, VLA_HANDOFF_KV_ALL = 1, VLA_HANDOFF_FEATURES = 2, VLA_HANDOFF_COG = 3 };
+enum { VLA_HEAD_A = 0, VLA_HEAD_B = 1, VLA_HEAD_C = 2, VLA_HEAD_D = 3 };
+enum { VLA_SOLVER_EULER = 0, VLA_SOLVER_DDIM = 1 };
+
+/* Model description: one "VLM phase feeding an action head" model (Section 2.1).
+ * Plain data; every field is a size or a flag.  Head kinds:
+ *   A  self-attention + cross-attention straight onto the VLM's last-layer K,V
+ *   B  expert whose layer l attends jointly over [VLM layer-l K,V ; its own K,V]
+ *   C  DiT alternating self / cross attention (odd layers cross-attend to the
+ *      VLM's final features), adaLN time conditioning
+ *   D  DiT conditioned in-context on one cognition token (last VLM position) */
+typedef struct {
+  int32_t n_cam, img, patch;                                   /* cameras, square image side, square patch side */
+  int32_t vis_layers, vis_d, vis_heads, vis_hd, vis_mlp;        /* vision encoder (vis_layers = 0: none) */
+  int32_t shuffle, connector;                                   /* s x s token pixel-shuffle; linear connector flag */
+  int32_t n_text, vocab;
+  int32_t llm_layers, d, hq, hkv, hd, mlp, mlp_kind, rope, causal;
+  int32_t handoff;
+  int32_t head, act_layers, act_d, act_heads, act_mlp, act_mlp_kind;
+  int32_t state_dim, horizon, act_dim, n_steps, solver;
+} vla_model_desc;
+
+typedef struct {
+  void* arena;              /* device; caller-owned, >= vla_required_arena_bytes, 256-byte aligned */
+  size_t arena_bytes;
+  void* stream_a;           /* cudaStream_t, caller-owned: VLM nodes / the persistent kernel */
+  void* stream_b;           /* cudaStream_t, caller-owned: action-head nodes (TWO_STREAM) */
+  int32_t mode;             /* VLA_MODE_* */
+  int32_t n_streams;        /* request streams R */
+  int32_t ring_depth;       /* frames in flight per request stream, >= 2 */
+  int32_t policy;           /* COSCHED pick: 0 = two-phase resource-aware pick, 1 = first-in-first-out */
+  uint64_t wait_limit_ns;   /* bound of every device-side wait; 0 = default (2 s) */
+  uint32_t trace_capacity;  /* tile records kept by the device trace; 0 = tracing off */
+  int32_t workers_per_sm;   /* COSCHED worker groups per SM; 0 = default */
+} vla_runtime_opts;
+
+typedef struct {
+  const char* name;         /* e.g. "llm.L3.wq" */
+  const void* host_ptr;     /* host; read during the call only */
+  int32_t dtype;            /* 0 = fp32 (rounded to bf16 nearest-even where stored as bf16), 1 = bf16 bits */
+  int32_t rank;
+  int64_t shape[4];
+} vla_tensor;
+
+/* One executed tile, as recorded by the device trace (all modes). */
+typedef struct {
+  uint32_t inst;            /* request stream * ring_depth + ring slot */
+  uint32_t node;            /* node index in the tile program */
+  uint32_t tile;            /* tile index inside the node */
+  uint16_t sm;              /* %smid */
+  uint8_t worker;           /* worker group on that SM (0 in the ordinary-kernel modes) */
+  uint8_t cls;              /* tile class: phase * 3 + kind */
+  uint64_t frame;           /* frame id the tile belonged to */
+  uint64_t t_start, t_end;  /* %globaltimer, ns */
+} vla_trace_rec;
+
+/* Static description of one node of the tile program (for the trace checker). */
+typedef struct {
+  int32_t op, cls, n_tiles, n_pred;
+  int32_t phase;            /* 0 VLM, 1 action head */
+  int32_t step;             /* denoising step, -1 outside the loop */
+  int32_t succ_begin, succ_count; /* range in the successor array */
+  char name[48];
+} vla_node_info;
+
+/* Bytes of device arena a context needs (weights, tile program, queues, per-frame buffers). */
+int vla_required_arena_bytes(const vla_model_desc* desc, const vla_runtime_opts* opts, size_t* out_bytes);
+
+/* Builds the tile program for `desc` and lays the arena out.  Problem statement: Section 2.1. */
+int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx** out_ctx);
+
+/* Copies the named tensors to the device (bf16), then runs the one-off constant
+ * precomputation (time-embedding MLP, adaLN modulation vectors) on the GPU.
+ * May be called several times; the call that completes the table arms the context.
+ * A missing or mis-shaped tensor -> VLA_ERR_INVALID, named in vla_last_error. */
+int vla_load_weights(vla_ctx* ctx, const vla_tensor* tensors, size_t n, int32_t final_call);
+
+/* Enqueues one frame of request stream `stream` (Section 2.1: each frame = image(s) +
+ * instruction tokens; the head also gets robot state and the initial noise sample).
+ * All pointers are HOST memory and are copied before the call returns:
+ * image fp32 [n_cam,3,img,img]; text_ids int32 [n_text]; state fp32 [state_dim] or NULL
+ * when the model has none; noise fp32 [horizon,act_dim].  Non-blocking with respect to
+ * the GPU.  Ring full -> VLA_ERR_BUSY.  frame_id (optional) gets the per-stream frame number. */
+int vla_submit_frame(vla_ctx* ctx, int32_t stream, const float* image, const int32_t* text_ids,
+                     const float* state, const float* noise, uint64_t* frame_id);
+
+/* Same as vla_submit_frame but the four inputs are DEVICE pointers (already resident
+ * in HBM); they are copied device-to-device into the frame slot. */
+int vla_submit_frame_device(vla_ctx* ctx, int32_t stream, const float* image, const int32_t* text_ids,
+                            const float* state, const float* noise, uint64_t* frame_id);
+
+/* Fetches the next finished action chunk of `stream`, in frame order (Section 2.1: the
+ * head of frame N consumed frame N's VLM output).  chunk: HOST fp32 [horizon,act_dim].
+ * Non-blocking; nothing ready -> VLA_ERR_NOT_READY. */
+int vla_poll_actions(vla_ctx* ctx, int32_t stream, float* chunk, uint64_t* frame_id);
+
+/* Blocks (host) until every submitted frame has produced its chunk or timeout_ms passed. */
+int vla_wait_idle(vla_ctx* ctx, uint32_t timeout_ms);
+
+/* Copies up to `cap` trace records (host memory) and reports how many exist. Call when idle. */
+int vla_get_trace(vla_ctx* ctx, vla_trace_rec* recs, size_t cap, size_t* n);
+int vla_reset_trace(vla_ctx* ctx);
+
+/* Tile-program introspection for the trace checker: node table and successor array. */
+int vla_program_info(vla_ctx* ctx, vla_node_info* nodes, size_t node_cap, size_t* n_nodes,
+                     int32_t* succ, size_t succ_cap, size_t* n_succ);
+
+/* Debug fetch of a named per-frame buffer (e.g. "llm.x", "llm.hidden", "act.v") of the ring
+ * slot last used by `stream`, widened to fp32 into HOST memory `out` (cap floats). Call when idle. */
+int vla_debug_fetch(vla_ctx* ctx, int32_t stream, int32_t slot, const char* buffer, float* out, size_t cap,
+                    size_t* n);
+
+/* Counters since init: tiles executed, kernels launched by the library, persistent-kernel launches. */
+int vla_get_counters(vla_ctx* ctx, uint64_t* tiles, uint64_t* kernel_launches, uint64_t* persistent_launches);
+
+/* Runs the device pick function (the COSCHED policy) once on the GPU for a given per-SM
+ * state, so tests can compare it with Algorithm 1.  All arrays HOST, n_cls <= 8.
+ * cta_count/u are updated as the admission would; *picked = class or -1; *phase = 1, 2 or 0. */
+int vla_policy_probe(int32_t n_cls, const int32_t* taus /*[n_cls*3]*/, const int32_t* pending, const int32_t* feasible,
+                     int32_t* cta_count, int32_t* u /*[3]*/, int32_t rr_start, int32_t* picked, int32_t* phase);
+
+const char* vla_last_error(vla_ctx* ctx);
+int vla_destroy(vla_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VLA_H_ */

@@ -1,0 +1,338 @@
+"""ctypes binding of libvla_b200.so: the same entry points as include/vla.h.
+
+Argument marshalling only -- every step of the forward pass runs inside the
+CUDA library.  PyTorch supplies the device arena and the CUDA streams.  There
+is no CPU fallback: importing this module without the built library, or
+creating an engine without a CUDA device, raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libvla_b200.so")
+
+VLA_OK, VLA_ERR_INVALID, VLA_ERR_STATE, VLA_ERR_BUSY, VLA_ERR_NOT_READY, VLA_ERR_TIMEOUT, VLA_ERR_CUDA, VLA_ERR_NOMEM = range(8)
+MODE_COSCHED, MODE_TWO_STREAM, MODE_SERIAL, MODE_MULTI_STREAM = 0, 1, 2, 3
+MODES = {"cosched": MODE_COSCHED, "two_stream": MODE_TWO_STREAM, "serial": MODE_SERIAL, "multi_stream": MODE_MULTI_STREAM}
+_MLP = {"gelu": 0, "swiglu": 1, "geglu": 2}
+_HANDOFF = {"kv_last": 0, "kv_all": 1, "features": 2, "cog": 3}
+_HEAD = {"A": 0, "B": 1, "C": 2, "D": 3}
+_SOLVER = {"euler": 0, "ddim": 1}
+
+EXPORTS = ["vla_required_arena_bytes", "vla_init", "vla_load_weights", "vla_submit_frame", "vla_submit_frame_device",
+           "vla_poll_actions", "vla_wait_idle", "vla_get_trace", "vla_reset_trace", "vla_program_info", "vla_debug_fetch",
+           "vla_get_counters", "vla_policy_probe", "vla_last_error", "vla_destroy"]
+
+
+class vla_model_desc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "n_cam", "img", "patch", "vis_layers", "vis_d", "vis_heads", "vis_hd", "vis_mlp", "shuffle", "connector",
+        "n_text", "vocab", "llm_layers", "d", "hq", "hkv", "hd", "mlp", "mlp_kind", "rope", "causal", "handoff",
+        "head", "act_layers", "act_d", "act_heads", "act_mlp", "act_mlp_kind", "state_dim", "horizon", "act_dim",
+        "n_steps", "solver")]
+
+
+class vla_runtime_opts(C.Structure):
+    _fields_ = [("arena", C.c_void_p), ("arena_bytes", C.c_size_t), ("stream_a", C.c_void_p), ("stream_b", C.c_void_p),
+                ("mode", C.c_int32), ("n_streams", C.c_int32), ("ring_depth", C.c_int32), ("policy", C.c_int32),
+                ("wait_limit_ns", C.c_uint64), ("trace_capacity", C.c_uint32), ("workers_per_sm", C.c_int32)]
+
+
+class vla_tensor(C.Structure):
+    _fields_ = [("name", C.c_char_p), ("host_ptr", C.c_void_p), ("dtype", C.c_int32), ("rank", C.c_int32),
+                ("shape", C.c_int64 * 4)]
+
+
+class vla_trace_rec(C.Structure):
+    _fields_ = [("inst", C.c_uint32), ("node", C.c_uint32), ("tile", C.c_uint32), ("sm", C.c_uint16), ("worker", C.c_uint8),
+                ("cls", C.c_uint8), ("frame", C.c_uint64), ("t_start", C.c_uint64), ("t_end", C.c_uint64)]
+
+
+class vla_node_info(C.Structure):
+    _fields_ = [("op", C.c_int32), ("cls", C.c_int32), ("n_tiles", C.c_int32), ("n_pred", C.c_int32), ("phase", C.c_int32),
+                ("step", C.c_int32), ("succ_begin", C.c_int32), ("succ_count", C.c_int32), ("name", C.c_char * 48)]
+
+
+TRACE_DTYPE = np.dtype([("inst", "<u4"), ("node", "<u4"), ("tile", "<u4"), ("sm", "<u2"), ("worker", "u1"), ("cls", "u1"),
+                        ("frame", "<u8"), ("t_start", "<u8"), ("t_end", "<u8")])
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads the in-tree shared library; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2609_22335_b200.build` (there is no CPU fallback)")
+    lib = C.CDLL(LIB_PATH)
+    P = C.POINTER
+    lib.vla_required_arena_bytes.argtypes = [P(vla_model_desc), P(vla_runtime_opts), P(C.c_size_t)]
+    lib.vla_init.argtypes = [P(vla_model_desc), P(vla_runtime_opts), P(C.c_void_p)]
+    lib.vla_load_weights.argtypes = [C.c_void_p, P(vla_tensor), C.c_size_t, C.c_int32]
+    for fn in (lib.vla_submit_frame, lib.vla_submit_frame_device):
+        fn.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, P(C.c_uint64)]
+    lib.vla_poll_actions.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, P(C.c_uint64)]
+    lib.vla_wait_idle.argtypes = [C.c_void_p, C.c_uint32]
+    lib.vla_get_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, P(C.c_size_t)]
+    lib.vla_reset_trace.argtypes = [C.c_void_p]
+    lib.vla_program_info.argtypes = [C.c_void_p, P(vla_node_info), C.c_size_t, P(C.c_size_t), P(C.c_int32), C.c_size_t,
+                                     P(C.c_size_t)]
+    lib.vla_debug_fetch.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_char_p, C.c_void_p, C.c_size_t, P(C.c_size_t)]
+    lib.vla_get_counters.argtypes = [C.c_void_p, P(C.c_uint64), P(C.c_uint64), P(C.c_uint64)]
+    lib.vla_policy_probe.argtypes = [C.c_int32, P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32),
+                                     C.c_int32, P(C.c_int32), P(C.c_int32)]
+    lib.vla_last_error.argtypes = [C.c_void_p]
+    lib.vla_last_error.restype = C.c_char_p
+    lib.vla_destroy.argtypes = [C.c_void_p]
+    for name in EXPORTS:
+        if name != "vla_last_error":
+            getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def make_desc(m) -> vla_model_desc:
+    """vla_synth ModelDesc (or any object with the same fields) -> C struct."""
+    d = vla_model_desc()
+    for name, _ in vla_model_desc._fields_:
+        v = getattr(m, name)
+        if name in ("mlp_kind", "act_mlp_kind"):
+            v = _MLP[v]
+        elif name == "handoff":
+            v = _HANDOFF[v]
+        elif name == "head":
+            v = _HEAD[v]
+        elif name == "solver":
+            v = _SOLVER[v]
+        setattr(d, name, int(v))
+    return d
+
+
+class VlaError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"vla error {code}: {msg}")
+        self.code = code
+
+
+def vla_required_arena_bytes(desc: vla_model_desc, opts: vla_runtime_opts) -> int:
+    out = C.c_size_t(0)
+    rc = load_library().vla_required_arena_bytes(C.byref(desc), C.byref(opts), C.byref(out))
+    if rc != VLA_OK:
+        raise VlaError(rc, "invalid model description or options")
+    return out.value
+
+
+class Engine:
+    """One library context plus the torch-owned arena and streams it runs on."""
+
+    def __init__(self, model, mode="cosched", n_streams=None, ring_depth=2, policy=0, trace_capacity=0,
+                 wait_limit_ns=0, workers_per_sm=0, device="cuda:0"):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required (there is no CPU fallback)")
+        self.lib = load_library()
+        self.torch = torch
+        self.model = model
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.desc = make_desc(model)
+        self.n_streams = int(n_streams if n_streams is not None else model.n_streams)
+        self.ring_depth = ring_depth
+        self.mode = MODES[mode] if isinstance(mode, str) else int(mode)
+        self.opts = vla_runtime_opts()
+        self.opts.mode = self.mode
+        self.opts.n_streams = self.n_streams
+        self.opts.ring_depth = ring_depth
+        self.opts.policy = policy
+        self.opts.wait_limit_ns = wait_limit_ns
+        self.opts.trace_capacity = trace_capacity
+        self.opts.workers_per_sm = workers_per_sm
+        self.arena_bytes = vla_required_arena_bytes(self.desc, self.opts)
+        self.arena = torch.empty(self.arena_bytes + 256, dtype=torch.uint8, device=self.device)
+        base = self.arena.data_ptr()
+        self.opts.arena = (base + 255) // 256 * 256
+        self.opts.arena_bytes = self.arena_bytes
+        self.stream_a = torch.cuda.Stream(device=self.device)
+        self.stream_b = torch.cuda.Stream(device=self.device)
+        self.opts.stream_a = self.stream_a.cuda_stream
+        self.opts.stream_b = self.stream_b.cuda_stream
+        self.ctx = C.c_void_p(None)
+        rc = self.lib.vla_init(C.byref(self.desc), C.byref(self.opts), C.byref(self.ctx))
+        if rc != VLA_OK:
+            msg = self.last_error() if self.ctx else "vla_init failed"
+            if self.ctx:
+                self.lib.vla_destroy(self.ctx)
+                self.ctx = C.c_void_p(None)
+            raise VlaError(rc, msg)
+        self.chunk_shape = (model.horizon, model.act_dim)
+
+    # ---- thin wrappers -------------------------------------------------------------
+    def last_error(self) -> str:
+        return (self.lib.vla_last_error(self.ctx) or b"").decode()
+
+    def _check(self, rc):
+        if rc != VLA_OK:
+            raise VlaError(rc, self.last_error())
+
+    def load_weights(self, weights, batch_bytes=1 << 30):
+        """weights: mapping name -> fp32 ndarray of bf16-representable values (vla_synth.gen.Weights)."""
+        from vla_synth.gen import bf16_bits
+        from vla_synth.configs import is_gain
+        names = list(weights.names())
+        batch, keep, size = [], [], 0
+
+        def flush(final):
+            arr = (vla_tensor * len(batch))(*batch)
+            self._check(self.lib.vla_load_weights(self.ctx, arr, len(batch), 1 if final else 0))
+            batch.clear(); keep.clear()
+
+        for i, name in enumerate(names):
+            w = weights[name]
+            fp32 = is_gain(name) or name in ("vis.pos", "llm.pos", "act.pos")
+            a = np.ascontiguousarray(w, dtype=np.float32) if fp32 else bf16_bits(w)
+            keep.append(a)
+            t = vla_tensor()
+            t.name = name.encode()
+            t.host_ptr = a.ctypes.data
+            t.dtype = 0 if fp32 else 1
+            t.rank = a.ndim
+            for k, s in enumerate(a.shape):
+                t.shape[k] = s
+            batch.append(t)
+            size += a.nbytes
+            if size >= batch_bytes and i + 1 < len(names):
+                flush(False)
+                size = 0
+        flush(True)
+
+    def submit(self, stream, frame) -> int:
+        """frame: dict image/text/state/noise of host numpy arrays. Returns VLA_OK or VLA_ERR_BUSY; raises otherwise."""
+        img = np.ascontiguousarray(frame["image"], dtype=np.float32)
+        txt = np.ascontiguousarray(frame["text"], dtype=np.int32)
+        st = None if frame.get("state") is None else np.ascontiguousarray(frame["state"], dtype=np.float32)
+        nz = np.ascontiguousarray(frame["noise"], dtype=np.float32)
+        rc = self.lib.vla_submit_frame(self.ctx, stream, img.ctypes.data, txt.ctypes.data,
+                                       None if st is None else st.ctypes.data, nz.ctypes.data, None)
+        if rc not in (VLA_OK, VLA_ERR_BUSY):
+            self._check(rc)
+        return rc
+
+    def submit_ptrs(self, stream, image_ptr, text_ptr, state_ptr, noise_ptr, device=False) -> int:
+        fn = self.lib.vla_submit_frame_device if device else self.lib.vla_submit_frame
+        rc = fn(self.ctx, stream, image_ptr, text_ptr, state_ptr, noise_ptr, None)
+        if rc not in (VLA_OK, VLA_ERR_BUSY):
+            self._check(rc)
+        return rc
+
+    def poll(self, stream, out=None):
+        """Returns (chunk ndarray, frame id) or None when nothing is ready."""
+        if out is None:
+            out = np.empty(self.chunk_shape, dtype=np.float32)
+        fid = C.c_uint64(0)
+        rc = self.lib.vla_poll_actions(self.ctx, stream, out.ctypes.data, C.byref(fid))
+        if rc == VLA_ERR_NOT_READY:
+            return None
+        self._check(rc)
+        return out, fid.value
+
+    def wait_idle(self, timeout_ms=60000):
+        self._check(self.lib.vla_wait_idle(self.ctx, timeout_ms))
+
+    def run(self, frames, timeout_s=600.0):
+        """frames[r][n] -> chunks[r][n]; submits as fast as the rings accept and polls in frame order."""
+        import time
+        R = len(frames)
+        nxt = [0] * R
+        got = [[None] * len(frames[r]) for r in range(R)]
+        remaining = sum(len(f) for f in frames)
+        t0 = time.time()
+        while remaining:
+            progressed = False
+            for r in range(R):
+                while nxt[r] < len(frames[r]):
+                    if self.submit(r, frames[r][nxt[r]]) == VLA_ERR_BUSY:
+                        break
+                    nxt[r] += 1
+                    progressed = True
+            for r in range(R):
+                while True:
+                    res = self.poll(r)
+                    if res is None:
+                        break
+                    chunk, fid = res
+                    got[r][fid] = chunk
+                    remaining -= 1
+                    progressed = True
+            if not progressed:
+                if time.time() - t0 > timeout_s:
+                    raise TimeoutError("no progress")
+                time.sleep(0.0002)
+        return got
+
+    def trace(self):
+        n = C.c_size_t(0)
+        self._check(self.lib.vla_get_trace(self.ctx, None, 0, C.byref(n)))
+        cap = min(n.value, self.opts.trace_capacity)
+        arr = np.zeros(cap, dtype=TRACE_DTYPE)
+        if cap:
+            self._check(self.lib.vla_get_trace(self.ctx, arr.ctypes.data, cap, C.byref(n)))
+        return arr, n.value
+
+    def reset_trace(self):
+        self._check(self.lib.vla_reset_trace(self.ctx))
+
+    def program_info(self):
+        nn, ns = C.c_size_t(0), C.c_size_t(0)
+        self._check(self.lib.vla_program_info(self.ctx, None, 0, C.byref(nn), None, 0, C.byref(ns)))
+        nodes = (vla_node_info * nn.value)()
+        succ = (C.c_int32 * max(ns.value, 1))()
+        self._check(self.lib.vla_program_info(self.ctx, nodes, nn.value, C.byref(nn), succ, ns.value, C.byref(ns)))
+        out = [dict(op=n.op, cls=n.cls, n_tiles=n.n_tiles, n_pred=n.n_pred, phase=n.phase, step=n.step,
+                    succ=[succ[n.succ_begin + i] for i in range(n.succ_count)], name=n.name.decode()) for n in nodes]
+        return out
+
+    def debug_fetch(self, stream, slot, name):
+        n = C.c_size_t(0)
+        self._check(self.lib.vla_debug_fetch(self.ctx, stream, slot, name.encode(), None, 0, C.byref(n)))
+        out = np.empty(n.value, dtype=np.float32)
+        self._check(self.lib.vla_debug_fetch(self.ctx, stream, slot, name.encode(), out.ctypes.data, n.value, C.byref(n)))
+        return out
+
+    def counters(self):
+        a, b, c = C.c_uint64(0), C.c_uint64(0), C.c_uint64(0)
+        self._check(self.lib.vla_get_counters(self.ctx, C.byref(a), C.byref(b), C.byref(c)))
+        return dict(tiles=a.value, kernel_launches=b.value, persistent_launches=c.value)
+
+    def close(self):
+        if self.ctx:
+            self.lib.vla_destroy(self.ctx)
+            self.ctx = C.c_void_p(None)
+        self.arena = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def policy_probe(taus, pending, feasible, cta_count, u, rr_start=0):
+    """Runs the device pick once on the GPU; returns (picked, phase, cta_count, u)."""
+    lib = load_library()
+    n = len(taus)
+    flat = (C.c_int32 * (3 * n))(*[int(x) for t in taus for x in t])
+    pend = (C.c_int32 * n)(*[int(bool(x)) for x in pending])
+    feas = (C.c_int32 * n)(*[int(bool(x)) for x in feasible])
+    cc = (C.c_int32 * n)(*[int(x) for x in cta_count])
+    uu = (C.c_int32 * 3)(*[int(x) for x in u])
+    picked, phase = C.c_int32(-1), C.c_int32(0)
+    rc = lib.vla_policy_probe(n, flat, pend, feas, cc, uu, rr_start, C.byref(picked), C.byref(phase))
+    if rc != VLA_OK:
+        raise VlaError(rc, "policy probe failed")
+    return picked.value, phase.value, list(cc), list(uu)

@@ -1,0 +1,878 @@
+// Tile-program compiler (host).  Turns a model description into:
+//   * the device weight table (fused / padded layouts),
+//   * per-frame-slot activation buffers,
+//   * a static DAG of nodes in program order, with dependencies derived from the
+//     buffers each node reads and writes (RAW, WAW and WAR edges),
+//   * the one-off constant precomputation program,
+//   * the arena layout.
+// The forward pass it encodes is the two-phase VLA model of paper Section 2.1 /
+// Figure 1 at the shapes of the five workload descriptions.
+#include "program.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+namespace vla {
+namespace {
+
+inline int64_t pad_to(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+struct View {          // rows [row0, row0+rows) of a buffer, starting at column col0
+  int buf = -1;
+  int64_t row0 = 0, rows = 0, col0 = 0;
+};
+
+struct Access {
+  uint64_t lo, hi;
+  int node;
+  bool write;
+};
+
+class Builder {
+ public:
+  Program& p;
+  const vla_model_desc& m;
+  std::vector<std::vector<Access>> acc;   // per buffer
+  std::vector<std::vector<int>> preds;    // per node
+  uint64_t slot_cursor = 0, const_cursor = 0, weight_cursor = 0;
+  int phase = PHASE_VLM, step = -1;
+  bool init_mode = false;                 // nodes go to the constant-precomputation program
+
+  Builder(Program& prog) : p(prog), m(prog.desc) {}
+
+  // ---------------------------------------------------------------- buffers
+  int buf(const std::string& name, int64_t rows, int64_t ld, int elem, bool slot = true) {
+    BufInfo b;
+    b.name = name; b.rows = rows; b.ld = ld; b.elem = elem; b.slot = slot;
+    b.bytes = (uint64_t)rows * ld * elem;
+    uint64_t& cur = slot ? slot_cursor : const_cursor;
+    cur = align_up(cur, 256);
+    b.offset = cur;
+    cur += b.bytes;
+    p.bufs.push_back(b);
+    p.buf_index[name] = (int)p.bufs.size() - 1;
+    acc.emplace_back();
+    return (int)p.bufs.size() - 1;
+  }
+  View all(int b) const { return View{b, 0, p.bufs[b].rows, 0}; }
+  View rows(int b, int64_t r0, int64_t n, int64_t c0 = 0) const { return View{b, r0, n, c0}; }
+  int64_t ld(const View& v) const { return p.bufs[v.buf].ld; }
+
+  Ref ref(const View& v) const {
+    if (v.buf < 0) return 0;
+    const BufInfo& b = p.bufs[v.buf];
+    uint64_t off = b.offset + (uint64_t)(v.row0 * b.ld + v.col0) * b.elem;
+    return b.slot ? (off | REF_SLOT) : (const_base + off);
+  }
+  static constexpr uint64_t WEIGHT_BASE = 4096;  // arena offset of the weight region (offset 0 stays "null")
+  uint64_t const_base = 0;                       // arena offset of the constant region, fixed once all weights are declared
+
+  // ---------------------------------------------------------------- weights
+  int dev_tensor(const std::string& name, int64_t rows, int64_t cols, bool is_bf16) {
+    DevTensor t;
+    t.name = name; t.rows = rows; t.cols = cols; t.is_bf16 = is_bf16;
+    t.ld = is_bf16 ? pad_to(cols, GEMM_BK) : cols;
+    weight_cursor = align_up(weight_cursor, 256);
+    t.offset = weight_cursor;
+    weight_cursor += (uint64_t)rows * t.ld * (is_bf16 ? 2 : 4);
+    p.dev_tensors.push_back(t);
+    p.dev_index[name] = (int)p.dev_tensors.size() - 1;
+    return (int)p.dev_tensors.size() - 1;
+  }
+  void source(const std::string& name, int64_t rows, int64_t cols, int dev, int64_t row_off) {
+    SourceTensor s;
+    s.name = name; s.rows = rows; s.cols = cols; s.dev = dev; s.row_offset = row_off;
+    p.source_index[name] = (int)p.sources.size();
+    p.sources.push_back(s);
+  }
+  // a matrix made of one or more caller tensors stacked by rows
+  int matrix(const std::string& dev_name, const std::vector<std::string>& parts, const std::vector<int64_t>& part_rows,
+             int64_t cols) {
+    int64_t rows = 0;
+    for (auto r : part_rows) rows += r;
+    int d = dev_tensor(dev_name, rows, cols, true);
+    int64_t off = 0;
+    for (size_t i = 0; i < parts.size(); ++i) {
+      source(parts[i], part_rows[i], cols, d, off);
+      off += part_rows[i];
+    }
+    return d;
+  }
+  int matrix1(const std::string& name, int64_t rows, int64_t cols) { return matrix(name, {name}, {rows}, cols); }
+  int table(const std::string& name, int64_t rows, int64_t cols) {   // fp32 position table
+    int d = dev_tensor(name, rows, cols, false);
+    source(name, rows, cols, d, 0);
+    return d;
+  }
+  int gain(const std::string& name, int64_t n) {
+    int d = dev_tensor(name, 1, n, false);
+    SourceTensor s;
+    s.name = name; s.rows = n; s.cols = 0; s.dev = d; s.row_offset = 0;
+    p.source_index[name] = (int)p.sources.size();
+    p.sources.push_back(s);
+    return d;
+  }
+  Ref wref(int dev, int64_t row0 = 0) const {
+    const DevTensor& t = p.dev_tensors[dev];
+    return WEIGHT_BASE + t.offset + (uint64_t)row0 * t.ld * (t.is_bf16 ? 2 : 4);
+  }
+
+  // ---------------------------------------------------------------- nodes and dependencies
+  void region(const View& v, uint64_t& lo, uint64_t& hi) const {
+    const BufInfo& b = p.bufs[v.buf];
+    lo = (uint64_t)v.row0 * b.ld * b.elem;
+    hi = (uint64_t)(v.row0 + v.rows) * b.ld * b.elem;
+  }
+  void read(int node, const View& v) {
+    if (v.buf < 0 || init_mode) return;
+    uint64_t lo, hi;
+    region(v, lo, hi);
+    for (const Access& a : acc[v.buf])
+      if (a.write && a.lo < hi && lo < a.hi && a.node != node) preds[node].push_back(a.node);
+    acc[v.buf].push_back(Access{lo, hi, node, false});
+  }
+  void write(int node, const View& v) {
+    if (v.buf < 0 || init_mode) return;
+    uint64_t lo, hi;
+    region(v, lo, hi);
+    auto& list = acc[v.buf];
+    for (const Access& a : list)
+      if (a.lo < hi && lo < a.hi && a.node != node) preds[node].push_back(a.node);
+    // accesses fully covered by this write are superseded: later nodes reach them through this one
+    list.erase(std::remove_if(list.begin(), list.end(),
+                              [&](const Access& a) { return a.lo >= lo && a.hi <= hi && a.node != node; }),
+               list.end());
+    list.push_back(Access{lo, hi, node, true});
+  }
+
+  int add(NodeDesc n, const std::string& name, int kind) {
+    n.phase = phase;
+    n.step = step;
+    n.cls = phase * 3 + kind;
+    n.n_pred = 0;
+    n.succ_begin = n.succ_count = 0;
+    if (init_mode) {
+      p.init_program.push_back(n);
+      return (int)p.init_program.size() - 1;
+    }
+    p.nodes.push_back(n);
+    p.node_names.push_back(name);
+    preds.emplace_back();
+    return (int)p.nodes.size() - 1;
+  }
+  NodeDesc& node(int i) { return init_mode ? p.init_program[i] : p.nodes[i]; }
+
+  // ---------------------------------------------------------------- op builders
+  struct GemmOpt {
+    View X; float c_x = 1.f, c_acc = 1.f;
+    Ref vec = 0;
+    Ref tab = 0; int ldtab = 0;
+    Ref tab2 = 0; int ldtab2 = 0;
+    View out32, out16;
+    int act = ACT_NONE;
+    int W2 = -1;
+    int64_t w_row0 = 0;
+  };
+  int gemm(const std::string& name, const View& A, int W, int64_t N, const GemmOpt& o) {
+    const DevTensor& wt = p.dev_tensors[W];
+    NodeDesc n;
+    std::memset(&n, 0, sizeof(n));
+    n.op = OP_GEMM;
+    GemmArgs& g = n.u.gemm;
+    g.A = ref(A); g.lda = (int)ld(A);
+    g.W = wref(W, o.w_row0);
+    g.W2 = o.W2 >= 0 ? wref(o.W2, o.w_row0) : 0;
+    g.dual = o.W2 >= 0;
+    g.M = (int)A.rows; g.N = (int)N; g.Kp = (int)wt.ld;
+    g.X = ref(o.X); g.ldx = o.X.buf >= 0 ? (int)ld(o.X) : 0;
+    g.c_x = o.c_x; g.c_acc = o.c_acc;
+    g.vec = o.vec; g.tab = o.tab; g.ldtab = o.ldtab; g.tab2 = o.tab2; g.ldtab2 = o.ldtab2;
+    g.out32 = ref(o.out32); g.ldo32 = o.out32.buf >= 0 ? (int)ld(o.out32) : 0;
+    g.out16 = ref(o.out16); g.ldo16 = o.out16.buf >= 0 ? (int)ld(o.out16) : 0;
+    g.act = o.act;
+    int tiles_t = (int)((g.M + 255) / 256);
+    int bt = (int)pad_to((g.M + tiles_t - 1) / tiles_t, 16);
+    if (g.dual && bt > 128) {              // two accumulators: keep both within the tensor-memory budget of one worker
+      tiles_t = (int)((g.M + 127) / 128);
+      bt = (int)pad_to((g.M + tiles_t - 1) / tiles_t, 16);
+    }
+    g.bt = bt; g.tiles_t = tiles_t;
+    g.amap_inst = -1; g.wmap = -1;
+    n.n_tiles = (int)((g.N + GEMM_BM - 1) / GEMM_BM) * tiles_t;
+    n.smem_bytes = GEMM_SMEM_BYTES;
+    int id = add(n, name, KIND_GEMM);
+    read(id, A);
+    if (o.X.buf >= 0) read(id, o.X);
+    if (o.out32.buf >= 0) write(id, o.out32);
+    if (o.out16.buf >= 0) write(id, o.out16);
+    if (A.rows * 1 > 0 && p.bufs[A.buf].ld < wt.ld && !init_mode) {
+      p.error = "internal: activation row pitch shorter than padded K in " + name;
+    }
+    return id;
+  }
+
+  int rmsnorm(const std::string& name, const View& x, int g_dev, const View& out, Ref mod = 0, int shuffle = 1,
+              int grid = 0) {
+    NodeDesc n;
+    std::memset(&n, 0, sizeof(n));
+    n.op = OP_RMSNORM;
+    NormArgs& a = n.u.norm;
+    a.x = ref(x); a.g = wref(g_dev); a.mod = mod; a.out = ref(out);
+    a.M = (int)x.rows; a.d = (int)p.dev_tensors[g_dev].cols; a.ldx = (int)ld(x); a.ldo = (int)ld(out);
+    a.rows_per_tile = 4; a.shuffle = shuffle; a.grid = grid;
+    n.n_tiles = (a.M + a.rows_per_tile - 1) / a.rows_per_tile;
+    int id = add(n, name, KIND_ELEM);
+    read(id, x);
+    write(id, out);
+    return id;
+  }
+
+  int attention(const std::string& name, const View& q, const View& k0, const View& v0, int t0, const View& k1,
+                const View& v1, int t1, const View& out, int hq, int hkv, int hd, bool causal) {
+    NodeDesc n;
+    std::memset(&n, 0, sizeof(n));
+    n.op = OP_ATTN;
+    AttnArgs& a = n.u.attn;
+    a.q = ref(q); a.k0 = ref(k0); a.v0 = ref(v0); a.k1 = ref(k1); a.v1 = ref(v1); a.out = ref(out);
+    a.ldq = (int)ld(q); a.ldk0 = k0.buf >= 0 ? (int)ld(k0) : 0; a.ldk1 = k1.buf >= 0 ? (int)ld(k1) : 0;
+    a.ldo = (int)ld(out);
+    a.tq = (int)q.rows; a.t0 = t0; a.t1 = t1; a.hq = hq; a.hkv = hkv; a.hd = hd; a.causal = causal;
+    a.bq = 16; a.q_blocks = (a.tq + a.bq - 1) / a.bq;
+    a.scale = 1.0f / std::sqrt((float)hd);
+    n.n_tiles = hq * a.q_blocks;
+    n.smem_bytes = 4 * (hd + t0 + t1) * 4 + 256;
+    int id = add(n, name, KIND_ATTN);
+    read(id, q);
+    if (k0.buf >= 0) { read(id, k0); if (v0.buf != k0.buf) read(id, v0); }
+    if (k1.buf >= 0 && k1.buf != q.buf) { read(id, k1); if (v1.buf != k1.buf) read(id, v1); }
+    write(id, out);
+    return id;
+  }
+
+  int elem_node(NodeDesc& n, const std::string& name) { return add(n, name, KIND_ELEM); }
+
+  int addrows(const std::string& name, const View& in, Ref in_raw, int ldi, int M, int N, Ref vec, Ref tab, int ldt,
+              const View& out, const View& out16) {
+    NodeDesc n;
+    std::memset(&n, 0, sizeof(n));
+    n.op = OP_ADDROWS;
+    AddRowsArgs& a = n.u.addrows;
+    a.in = in.buf >= 0 ? ref(in) : in_raw;
+    a.ldi = in.buf >= 0 ? (int)ld(in) : ldi;
+    a.vec = vec; a.tab = tab; a.ldt = ldt;
+    a.out = ref(out); a.ldo = out.buf >= 0 ? (int)ld(out) : 0;
+    a.out16 = ref(out16); a.ldo16 = out16.buf >= 0 ? (int)ld(out16) : 0;
+    a.M = M; a.N = N;
+    n.n_tiles = 1;
+    int id = add(n, name, KIND_ELEM);
+    if (in.buf >= 0) read(id, in);
+    if (out.buf >= 0) write(id, out);
+    if (out16.buf >= 0) write(id, out16);
+    return id;
+  }
+};
+
+constexpr uint64_t Builder::WEIGHT_BASE;
+
+void set_err(Program& p, const char* msg) { p.error = msg; }
+
+bool validate(const vla_model_desc& d, Program& p) {
+  auto bad = [&](const char* s) { set_err(p, s); return false; };
+  if (d.n_cam < 1 || d.img < 1 || d.patch < 1 || d.img % d.patch) return bad("image side must be a positive multiple of the patch side");
+  int grid = d.img / d.patch;
+  if (d.shuffle < 1 || grid % d.shuffle) return bad("token grid must be a multiple of the shuffle factor");
+  if (d.vis_layers < 0 || d.llm_layers < 1 || d.act_layers < 1) return bad("layer counts out of range");
+  if (d.vis_layers > 0 && (d.vis_heads < 1 || d.vis_hd < 1 || d.vis_mlp < 1)) return bad("vision encoder sizes missing");
+  if (d.vis_layers > 0 && !d.connector) return bad("a vision encoder needs the linear connector");
+  if (!d.connector && (d.shuffle != 1 || d.vis_d != d.d)) return bad("without a connector the patch width must equal the LLM width and shuffle must be 1");
+  if (d.vis_layers == 0 && d.shuffle != 1) return bad("pixel-shuffle needs a vision encoder");
+  if (d.vis_d < 1 || d.d < 1 || d.hq < 1 || d.hkv < 1 || d.hd < 2 || d.hq % d.hkv) return bad("LLM head geometry invalid");
+  if (d.hd % 2) return bad("head dimension must be even");
+  if (d.mlp < 1 || d.mlp_kind < 0 || d.mlp_kind > 2 || d.act_mlp < 1 || d.act_mlp_kind < 0 || d.act_mlp_kind > 2) return bad("MLP description invalid");
+  if (d.n_text < 1 || d.vocab < 1) return bad("text description invalid");
+  if (d.head < 0 || d.head > 3) return bad("unknown head kind");
+  if (d.act_d < 2 || d.act_d % 2) return bad("head width must be even");
+  if (d.head != VLA_HEAD_B && (d.act_heads < 1 || d.act_d % d.act_heads)) return bad("head width must be a multiple of its head count");
+  if (d.horizon < 1 || d.act_dim < 1 || d.n_steps < 1 || d.state_dim < 0) return bad("chunk description invalid");
+  if (d.solver < 0 || d.solver > 1) return bad("unknown solver");
+  if (d.solver == VLA_SOLVER_DDIM && (100 % d.n_steps)) return bad("DDIM step count must divide 100");
+  if (d.head == VLA_HEAD_A && d.handoff != VLA_HANDOFF_KV_LAST) return bad("head A needs the kv_last handoff");
+  if (d.head == VLA_HEAD_B && (d.handoff != VLA_HANDOFF_KV_ALL || d.act_layers != d.llm_layers)) return bad("head B needs kv_all and as many layers as the LLM");
+  if (d.head == VLA_HEAD_C && d.handoff != VLA_HANDOFF_FEATURES) return bad("head C needs the features handoff");
+  if (d.head == VLA_HEAD_D && (d.handoff != VLA_HANDOFF_COG || d.state_dim != 0)) return bad("head D needs the cog handoff and no state");
+  if (d.head == VLA_HEAD_A && d.state_dim == 0) return bad("head A needs a state token");
+  return true;
+}
+
+std::vector<double> ddim_alpha_bar(int T) {
+  auto c = [](double u) { double x = std::cos((u + 0.008) / 1.008 * M_PI / 2); return x * x; };
+  std::vector<double> ab;
+  double prod = 1.0;
+  for (int s = 0; s < T; ++s) {
+    double beta = std::min(1.0 - c((s + 1.0) / T) / c((double)s / T), 0.999);
+    prod *= 1.0 - beta;
+    ab.push_back(prod);
+  }
+  return ab;
+}
+
+}  // namespace
+
+bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& p) {
+  p = Program();
+  p.desc = d;
+  if (!validate(d, p)) return false;
+  if (o.n_streams < 1 || o.n_streams > 1024 || o.ring_depth < 2 || o.ring_depth > 64) {
+    set_err(p, "n_streams must be 1..1024 and ring_depth 2..64");
+    return false;
+  }
+  p.n_streams = o.n_streams;
+  p.ring_depth = o.ring_depth;
+  p.n_inst = o.n_streams * o.ring_depth;
+  if (p.n_inst >= 4096) { set_err(p, "too many frame slots"); return false; }
+
+  Builder b(p);
+  const int grid = d.img / d.patch;
+  const int T = grid * grid;                                   // tokens per camera in the encoder
+  const int tpc = T / (d.shuffle * d.shuffle);                 // tokens per camera entering the LLM
+  const int n_img = d.n_cam * tpc;
+  const int S = n_img + d.n_text;
+  const int patch_k = 3 * d.patch * d.patch;
+  const int dv = d.vis_d, D = d.d, da = d.act_d;
+  const bool has_state = d.state_dim > 0;
+  const int first = (has_state || d.head == VLA_HEAD_D) ? 1 : 0;
+  const int Ta = d.horizon + first;
+  const bool head_pos = !(d.head == VLA_HEAD_B && d.rope);
+  const bool gated = d.mlp_kind != VLA_MLP_GELU, agated = d.act_mlp_kind != VLA_MLP_GELU;
+  const int hvd = d.vis_heads * d.vis_hd;
+  const int nq = d.hq * d.hd, nkv = d.hkv * d.hd, nqkv = nq + 2 * nkv;
+  auto P64 = [](int64_t x) { return pad_to(x, GEMM_BK); };
+  char nm[96];
+  auto N_ = [&](const char* fmt, int a = 0, int c = 0) { std::snprintf(nm, sizeof nm, fmt, a, c); return std::string(nm); };
+
+  // ================================================================== weights
+  int w_patch = b.matrix1("vis.patch.w", dv, patch_k);
+  int w_vpos = b.table("vis.pos", T, dv);
+  struct EncW { int n1, wqkv, wo, n2, w1, w2; };
+  std::vector<EncW> venc(d.vis_layers);
+  for (int i = 0; i < d.vis_layers; ++i) {
+    std::string pre = N_("vis.L%d.", i);
+    venc[i].n1 = b.gain(pre + "n1", dv);
+    venc[i].wqkv = b.matrix(pre + "wqkv", {pre + "wq", pre + "wk", pre + "wv"}, {hvd, hvd, hvd}, dv);
+    venc[i].wo = b.matrix1(pre + "wo", dv, hvd);
+    venc[i].n2 = b.gain(pre + "n2", dv);
+    venc[i].w1 = b.matrix1(pre + "w1", d.vis_mlp, dv);
+    venc[i].w2 = b.matrix1(pre + "w2", dv, d.vis_mlp);
+  }
+  int w_vnorm = d.vis_layers > 0 ? b.gain("vis.norm", dv) : -1;
+  int w_conn = d.connector ? b.matrix1("conn.w", D, (int64_t)d.shuffle * d.shuffle * dv) : -1;
+  int w_emb = b.matrix1("txt.emb", d.vocab, D);
+  int w_lpos = d.rope ? -1 : b.table("llm.pos", S, D);
+  struct LlmW { int n1, wqkv, wo, n2, w1, w2, wg, wu, wd; };
+  std::vector<LlmW> lw(d.llm_layers);
+  for (int i = 0; i < d.llm_layers; ++i) {
+    std::string pre = N_("llm.L%d.", i);
+    lw[i].n1 = b.gain(pre + "n1", D);
+    lw[i].wqkv = b.matrix(pre + "wqkv", {pre + "wq", pre + "wk", pre + "wv"}, {nq, nkv, nkv}, D);
+    lw[i].wo = b.matrix1(pre + "wo", D, nq);
+    lw[i].n2 = b.gain(pre + "n2", D);
+    if (gated) {
+      lw[i].wg = b.matrix1(pre + "wg", d.mlp, D);
+      lw[i].wu = b.matrix1(pre + "wu", d.mlp, D);
+      lw[i].wd = b.matrix1(pre + "wd", D, d.mlp);
+    } else {
+      lw[i].w1 = b.matrix1(pre + "w1", d.mlp, D);
+      lw[i].w2 = b.matrix1(pre + "w2", D, d.mlp);
+    }
+  }
+  int w_lnorm = b.gain("llm.norm", D);
+
+  int w_ain = b.matrix1("act.in", da, d.act_dim);
+  int w_astate = has_state ? b.matrix1("act.state", da, d.state_dim) : -1;
+  int w_acond = d.head == VLA_HEAD_D ? b.matrix1("act.cond", da, D) : -1;
+  int w_apos = head_pos ? b.table("act.pos", Ta, da) : -1;
+  int w_t1 = b.matrix1("act.t1", da, da);
+  int w_t2 = b.matrix1("act.t2", da, da);
+  struct ActW { int n1, n2, n3, wqkv, wo, cq, ckv, co, ada1, ada2, w1, w2, wg, wu, wd; };
+  std::vector<ActW> aw(d.act_layers);
+  for (int i = 0; i < d.act_layers; ++i) {
+    std::string pre = N_("act.L%d.", i);
+    ActW& a = aw[i];
+    a.n1 = b.gain(pre + "n1", da);
+    if (d.head == VLA_HEAD_B) {
+      a.wqkv = b.matrix(pre + "wqkv", {pre + "wq", pre + "wk", pre + "wv"}, {nq, nkv, nkv}, da);
+      a.wo = b.matrix1(pre + "wo", da, nq);
+    } else if (d.head == VLA_HEAD_C && (i % 2 == 1)) {
+      a.cq = b.matrix1(pre + "cq", da, da);
+      a.ckv = b.matrix(pre + "ckv", {pre + "ck", pre + "cv"}, {da, da}, D);
+      a.co = b.matrix1(pre + "co", da, da);
+    } else {
+      a.wqkv = b.matrix(pre + "wqkv", {pre + "wq", pre + "wk", pre + "wv"}, {da, da, da}, da);
+      a.wo = b.matrix1(pre + "wo", da, da);
+    }
+    a.n2 = b.gain(pre + "n2", da);
+    if (d.head == VLA_HEAD_A) {
+      a.cq = b.matrix1(pre + "cq", nq, da);
+      a.co = b.matrix1(pre + "co", da, nq);
+      a.n3 = b.gain(pre + "n3", da);
+    }
+    if (d.head == VLA_HEAD_C) {
+      a.ada1 = b.matrix1(pre + "ada1", 2 * da, da);
+      a.ada2 = b.matrix1(pre + "ada2", 2 * da, da);
+    }
+    if (agated) {
+      a.wg = b.matrix1(pre + "wg", d.act_mlp, da);
+      a.wu = b.matrix1(pre + "wu", d.act_mlp, da);
+      a.wd = b.matrix1(pre + "wd", da, d.act_mlp);
+    } else {
+      a.w1 = b.matrix1(pre + "w1", d.act_mlp, da);
+      a.w2 = b.matrix1(pre + "w2", da, d.act_mlp);
+    }
+  }
+  int w_anorm = b.gain("act.norm", da);
+  int w_aout = b.matrix1("act.out", d.act_dim, da);
+
+  // ================================================================== solver constants
+  const int ns = d.n_steps;
+  p.step_args.resize(ns); p.step_c_x.resize(ns); p.step_c_acc.resize(ns);
+  if (d.solver == VLA_SOLVER_EULER) {
+    for (int k = 0; k < ns; ++k) {
+      p.step_args[k] = 1000.0f * (float)k / (float)ns;
+      p.step_c_x[k] = 1.0f;
+      p.step_c_acc[k] = 1.0f / (float)ns;
+    }
+  } else {
+    // deterministic DDIM: x' = sqrt(a_prev) (x - sqrt(1-a_t) e)/sqrt(a_t) + sqrt(1-a_prev) e, folded to c_x x + c_acc e
+    std::vector<double> ab = ddim_alpha_bar(100);
+    int stride = 100 / ns;
+    for (int k = 0; k < ns; ++k) {
+      int tau = (ns - 1 - k) * stride;
+      double a_t = ab[tau], a_prev = tau - stride >= 0 ? ab[tau - stride] : 1.0;
+      p.step_args[k] = (float)tau;
+      p.step_c_x[k] = (float)(std::sqrt(a_prev) / std::sqrt(a_t));
+      p.step_c_acc[k] = (float)(std::sqrt(1.0 - a_prev) - std::sqrt(a_prev) * std::sqrt(1.0 - a_t) / std::sqrt(a_t));
+    }
+  }
+
+  // ================================================================== constant buffers + their precomputation
+  b.const_base = align_up(Builder::WEIGHT_BASE + b.weight_cursor, 4096);
+  int c_args = b.buf("const.args", 1, pad_to(ns, 4), 4, false);
+  int c_temb = b.buf("const.temb", ns, P64(da), 2, false);
+  int c_th = b.buf("const.th", ns, P64(da), 2, false);
+  int c_ct = b.buf("const.ct", ns, da, 4, false);
+  int c_sct = d.head == VLA_HEAD_C ? b.buf("const.sct", ns, P64(da), 2, false) : -1;
+  std::vector<int> c_mod1(d.act_layers, -1), c_mod2(d.act_layers, -1);
+  if (d.head == VLA_HEAD_C)
+    for (int i = 0; i < d.act_layers; ++i) {
+      c_mod1[i] = b.buf(N_("const.mod1.%d", i), ns, 2 * da, 4, false);
+      c_mod2[i] = b.buf(N_("const.mod2.%d", i), ns, 2 * da, 4, false);
+    }
+  b.init_mode = true;
+  b.phase = PHASE_ACT;
+  {
+    NodeDesc n;
+    std::memset(&n, 0, sizeof n);
+    n.op = OP_TIMEEMB;
+    n.u.timeemb.args = b.ref(b.all(c_args));
+    n.u.timeemb.out = b.ref(b.all(c_temb));
+    n.u.timeemb.M = ns; n.u.timeemb.width = da; n.u.timeemb.ldo = (int)P64(da);
+    n.n_tiles = 1;
+    b.add(n, "init.temb", KIND_ELEM);
+    Builder::GemmOpt g1; g1.act = ACT_SILU; g1.out16 = b.all(c_th);
+    b.gemm("init.t1", b.all(c_temb), w_t1, da, g1);
+    Builder::GemmOpt g2; g2.out32 = b.all(c_ct);
+    b.gemm("init.t2", b.all(c_th), w_t2, da, g2);
+    if (d.head == VLA_HEAD_C) {
+      Builder::GemmOpt g3; g3.act = ACT_SILU; g3.out16 = b.all(c_sct);
+      b.gemm("init.t2s", b.all(c_th), w_t2, da, g3);
+      for (int i = 0; i < d.act_layers; ++i) {
+        Builder::GemmOpt ga; ga.out32 = b.all(c_mod1[i]);
+        b.gemm("init.ada1", b.all(c_sct), aw[i].ada1, 2 * da, ga);
+        Builder::GemmOpt gb; gb.out32 = b.all(c_mod2[i]);
+        b.gemm("init.ada2", b.all(c_sct), aw[i].ada2, 2 * da, gb);
+      }
+    }
+  }
+  b.init_mode = false;
+
+  // ================================================================== frame-slot buffers
+  // inputs
+  int in_img = b.buf("in.image", d.n_cam, (int64_t)3 * d.img * d.img, 4);
+  int in_txt = b.buf("in.text", 1, pad_to(d.n_text, 4), 4);
+  int in_state = has_state ? b.buf("in.state", 1, d.state_dim, 4) : -1;
+  int in_noise = b.buf("in.noise", d.horizon, d.act_dim, 4);
+  p.in_image = p.bufs[in_img].offset; p.image_bytes = p.bufs[in_img].bytes;
+  p.in_text = p.bufs[in_txt].offset; p.text_bytes = (uint64_t)d.n_text * 4;
+  if (has_state) { p.in_state = p.bufs[in_state].offset; p.state_bytes = (uint64_t)d.state_dim * 4; }
+  p.in_noise = p.bufs[in_noise].offset; p.noise_bytes = p.bufs[in_noise].bytes;
+
+  // LLM
+  int x = b.buf("llm.x", S, D, 4);
+  int h = b.buf("llm.h", S, P64(D), 2);
+  int qkv32 = d.rope ? b.buf("llm.qkv32", S, nqkv, 4) : -1;
+  std::vector<int> qkv(d.llm_layers);
+  {
+    int shared = -1;
+    for (int i = 0; i < d.llm_layers; ++i) {
+      bool own = d.handoff == VLA_HANDOFF_KV_ALL || (d.handoff == VLA_HANDOFF_KV_LAST && i == d.llm_layers - 1);
+      if (own) qkv[i] = b.buf(N_("llm.qkv.%d", i), S, nqkv, 2);
+      else {
+        if (shared < 0) shared = b.buf("llm.qkv", S, nqkv, 2);
+        qkv[i] = shared;
+      }
+    }
+  }
+  int att = b.buf("llm.att", S, P64(nq), 2);
+  int mid = b.buf("llm.mid", S, P64(d.mlp), 2);
+  int hidden = b.buf("llm.hidden", S, P64(D), 2);
+
+  // ================================================================== VLM phase
+  b.phase = PHASE_VLM;
+  b.step = -1;
+  for (int c = 0; c < d.n_cam; ++c) {
+    int patches = b.buf(N_("vis%d.patches", c), T, P64(patch_k), 2);
+    {
+      NodeDesc n;
+      std::memset(&n, 0, sizeof n);
+      n.op = OP_PATCHIFY;
+      PatchArgs& a = n.u.patch;
+      a.img = b.ref(b.rows(in_img, c, 1));
+      a.out = b.ref(b.all(patches));
+      a.img_side = d.img; a.patch = d.patch; a.grid = grid; a.ldo = (int)P64(patch_k); a.rows_per_tile = 4;
+      n.n_tiles = (T + 3) / 4;
+      int id = b.add(n, N_("vis%d.patchify", c), KIND_ELEM);
+      b.read(id, b.rows(in_img, c, 1));
+      b.write(id, b.all(patches));
+    }
+    if (d.vis_layers == 0 && !d.connector) {
+      // patch embedding feeds the LLM residual stream directly
+      Builder::GemmOpt g;
+      g.tab = b.wref(w_vpos); g.ldtab = dv;
+      if (w_lpos >= 0) { g.tab2 = b.wref(w_lpos, (int64_t)c * tpc); g.ldtab2 = D; }
+      g.out32 = b.rows(x, (int64_t)c * tpc, tpc);
+      b.gemm(N_("vis%d.patch", c), b.all(patches), w_patch, dv, g);
+      continue;
+    }
+    int xv = b.buf(N_("vis%d.x", c), T, dv, 4);
+    int hv = b.buf(N_("vis%d.h", c), T, P64(dv), 2);
+    int vqkv = d.vis_layers > 0 ? b.buf(N_("vis%d.qkv", c), T, 3 * hvd, 2) : -1;
+    int vatt = d.vis_layers > 0 ? b.buf(N_("vis%d.att", c), T, P64(hvd), 2) : -1;
+    int vmid = d.vis_layers > 0 ? b.buf(N_("vis%d.mid", c), T, P64(d.vis_mlp), 2) : -1;
+    int shuf = b.buf(N_("vis%d.shuf", c), tpc, P64((int64_t)d.shuffle * d.shuffle * dv), 2);
+    {
+      Builder::GemmOpt g;
+      g.tab = b.wref(w_vpos); g.ldtab = dv;
+      if (d.vis_layers > 0) g.out32 = b.all(xv); else g.out16 = b.all(shuf);
+      b.gemm(N_("vis%d.patch", c), b.all(patches), w_patch, dv, g);
+    }
+    for (int i = 0; i < d.vis_layers; ++i) {
+      b.rmsnorm(N_("vis%d.L%d.n1", c, i), b.all(xv), venc[i].n1, b.all(hv));
+      Builder::GemmOpt gq; gq.out16 = b.all(vqkv);
+      b.gemm(N_("vis%d.L%d.qkv", c, i), b.all(hv), venc[i].wqkv, 3 * hvd, gq);
+      b.attention(N_("vis%d.L%d.attn", c, i), b.rows(vqkv, 0, T, 0), b.rows(vqkv, 0, T, hvd), b.rows(vqkv, 0, T, 2 * hvd),
+                  T, View(), View(), 0, b.all(vatt), d.vis_heads, d.vis_heads, d.vis_hd, false);
+      Builder::GemmOpt go; go.X = b.all(xv); go.out32 = b.all(xv);
+      b.gemm(N_("vis%d.L%d.wo", c, i), b.all(vatt), venc[i].wo, dv, go);
+      b.rmsnorm(N_("vis%d.L%d.n2", c, i), b.all(xv), venc[i].n2, b.all(hv));
+      Builder::GemmOpt g1; g1.act = ACT_GELU; g1.out16 = b.all(vmid);
+      b.gemm(N_("vis%d.L%d.w1", c, i), b.all(hv), venc[i].w1, d.vis_mlp, g1);
+      Builder::GemmOpt g2; g2.X = b.all(xv); g2.out32 = b.all(xv);
+      b.gemm(N_("vis%d.L%d.w2", c, i), b.all(vmid), venc[i].w2, dv, g2);
+    }
+    if (d.vis_layers > 0)
+      b.rmsnorm(N_("vis%d.norm", c), b.all(xv), w_vnorm, b.all(shuf), 0, d.shuffle, grid);
+    {
+      Builder::GemmOpt g;
+      if (w_lpos >= 0) { g.tab = b.wref(w_lpos, (int64_t)c * tpc); g.ldtab = D; }
+      g.out32 = b.rows(x, (int64_t)c * tpc, tpc);
+      b.gemm(N_("vis%d.conn", c), b.all(shuf), w_conn, D, g);
+    }
+  }
+  {
+    NodeDesc n;
+    std::memset(&n, 0, sizeof n);
+    n.op = OP_EMBED;
+    EmbedArgs& a = n.u.embed;
+    a.ids = b.ref(b.all(in_txt));
+    a.table = b.wref(w_emb);
+    a.pos = w_lpos >= 0 ? b.wref(w_lpos, n_img) : 0;
+    a.out = b.ref(b.rows(x, n_img, d.n_text));
+    a.n = d.n_text; a.d = D; a.ldo = D; a.vocab = d.vocab; a.rows_per_tile = 4; a.ldt = (int)P64(D);
+    n.n_tiles = (d.n_text + 3) / 4;
+    int id = b.add(n, "llm.embed", KIND_ELEM);
+    b.read(id, b.all(in_txt));
+    b.write(id, b.rows(x, n_img, d.n_text));
+  }
+  for (int i = 0; i < d.llm_layers; ++i) {
+    b.rmsnorm(N_("llm.L%d.n1", i), b.all(x), lw[i].n1, b.all(h));
+    if (d.rope) {
+      Builder::GemmOpt gq; gq.out32 = b.all(qkv32);
+      b.gemm(N_("llm.L%d.qkv", i), b.all(h), lw[i].wqkv, nqkv, gq);
+      NodeDesc n;
+      std::memset(&n, 0, sizeof n);
+      n.op = OP_ROPE;
+      RopeArgs& a = n.u.rope;
+      a.in = b.ref(b.all(qkv32)); a.out = b.ref(b.all(qkv[i]));
+      a.M = S; a.ld = nqkv; a.n_rot_heads = d.hq + d.hkv; a.n_heads = d.hq + 2 * d.hkv; a.hd = d.hd; a.pos0 = 0;
+      a.rows_per_tile = 4;
+      n.n_tiles = (S + 3) / 4;
+      int id = b.add(n, N_("llm.L%d.rope", i), KIND_ELEM);
+      b.read(id, b.all(qkv32));
+      b.write(id, b.all(qkv[i]));
+    } else {
+      Builder::GemmOpt gq; gq.out16 = b.all(qkv[i]);
+      b.gemm(N_("llm.L%d.qkv", i), b.all(h), lw[i].wqkv, nqkv, gq);
+    }
+    b.attention(N_("llm.L%d.attn", i), b.rows(qkv[i], 0, S, 0), b.rows(qkv[i], 0, S, nq), b.rows(qkv[i], 0, S, nq + nkv), S,
+                View(), View(), 0, b.all(att), d.hq, d.hkv, d.hd, d.causal != 0);
+    Builder::GemmOpt go; go.X = b.all(x); go.out32 = b.all(x);
+    b.gemm(N_("llm.L%d.wo", i), b.all(att), lw[i].wo, D, go);
+    b.rmsnorm(N_("llm.L%d.n2", i), b.all(x), lw[i].n2, b.all(h));
+    Builder::GemmOpt g1; g1.out16 = b.all(mid);
+    if (gated) {
+      g1.W2 = lw[i].wu;
+      g1.act = d.mlp_kind == VLA_MLP_SWIGLU ? ACT_SILU : ACT_GELU;
+      b.gemm(N_("llm.L%d.gu", i), b.all(h), lw[i].wg, d.mlp, g1);
+    } else {
+      g1.act = ACT_GELU;
+      b.gemm(N_("llm.L%d.w1", i), b.all(h), lw[i].w1, d.mlp, g1);
+    }
+    Builder::GemmOpt g2; g2.X = b.all(x); g2.out32 = b.all(x);
+    b.gemm(N_("llm.L%d.w2", i), b.all(mid), gated ? lw[i].wd : lw[i].w2, D, g2);
+  }
+  b.rmsnorm("llm.norm", b.all(x), w_lnorm, b.all(hidden));
+  std::vector<int> ckv(d.act_layers, -1);
+  if (d.head == VLA_HEAD_C)
+    for (int i = 1; i < d.act_layers; i += 2) {
+      ckv[i] = b.buf(N_("act.ckv.%d", i), S, 2 * da, 2);
+      Builder::GemmOpt g; g.out16 = b.all(ckv[i]);
+      b.gemm(N_("act.L%d.ckv", i), b.all(hidden), aw[i].ckv, 2 * da, g);
+    }
+
+  // ================================================================== action-head phase
+  b.phase = PHASE_ACT;
+  b.step = -1;
+  const int ahd = d.head == VLA_HEAD_B ? d.hd : da / d.act_heads;
+  const int a_nq = d.head == VLA_HEAD_B ? nq : da, a_nkv = d.head == VLA_HEAD_B ? nkv : da;
+  const int a_nqkv = a_nq + 2 * a_nkv;
+  int xs = b.buf("act.x", d.horizon, d.act_dim, 4);
+  int xbf = b.buf("act.xbf", d.horizon, P64(d.act_dim), 2);
+  int z = b.buf("act.z", Ta, da, 4);
+  int hz = b.buf("act.h", Ta, P64(da), 2);
+  int aqkv = b.buf("act.qkv", Ta, a_nqkv, 2);
+  int aqkv32 = (d.head == VLA_HEAD_B && d.rope) ? b.buf("act.qkv32", Ta, a_nqkv, 4) : -1;
+  int aatt = b.buf("act.att", Ta, P64(std::max(a_nq, nq)), 2);
+  int aqc = (d.head == VLA_HEAD_A || d.head == VLA_HEAD_C) ? b.buf("act.qc", Ta, d.head == VLA_HEAD_A ? nq : da, 2) : -1;
+  int amid = b.buf("act.mid", Ta, P64(d.act_mlp), 2);
+  int tok0 = first ? b.buf("act.tok0", 1, da, 4) : -1;
+  int state_bf = has_state ? b.buf("act.state_bf", 1, P64(d.state_dim), 2) : -1;
+
+  if (has_state) {
+    b.addrows("act.state_cvt", b.all(in_state), 0, 0, 1, d.state_dim, 0, 0, 0, View(), b.all(state_bf));
+    Builder::GemmOpt g;
+    if (head_pos) { g.tab = b.wref(w_apos, 0); g.ldtab = da; }
+    g.out32 = b.all(tok0);
+    b.gemm("act.state_tok", b.all(state_bf), w_astate, da, g);
+  } else if (d.head == VLA_HEAD_D) {
+    Builder::GemmOpt g;
+    if (head_pos) { g.tab = b.wref(w_apos, 0); g.ldtab = da; }
+    g.out32 = b.all(tok0);
+    b.gemm("act.cond_tok", b.rows(hidden, S - 1, 1), w_acond, da, g);
+  }
+  b.addrows("act.x_init", b.all(in_noise), 0, 0, d.horizon, d.act_dim, 0, 0, 0, b.all(xs), b.all(xbf));
+
+  for (int k = 0; k < ns; ++k) {
+    b.step = k;
+    Ref ct_k = b.ref(b.rows(c_ct, k, 1));
+    if (first) {
+      b.addrows(N_("act.s%d.tok0", k), b.all(tok0), 0, 0, 1, da, d.head == VLA_HEAD_D ? ct_k : 0, 0, 0, b.rows(z, 0, 1),
+                View());
+    }
+    {
+      Builder::GemmOpt g;
+      if (d.head == VLA_HEAD_A || d.head == VLA_HEAD_B) g.vec = ct_k;
+      if (head_pos) { g.tab = b.wref(w_apos, first); g.ldtab = da; }
+      g.out32 = b.rows(z, first, d.horizon);
+      b.gemm(N_("act.s%d.in", k), b.all(xbf), w_ain, da, g);
+    }
+    for (int i = 0; i < d.act_layers; ++i) {
+      const ActW& a = aw[i];
+      auto NN = [&](const char* leaf) { std::snprintf(nm, sizeof nm, "act.s%d.L%d.%s", k, i, leaf); return std::string(nm); };
+      Ref mod1 = d.head == VLA_HEAD_C ? b.ref(b.rows(c_mod1[i], k, 1)) : 0;
+      Ref mod2 = d.head == VLA_HEAD_C ? b.ref(b.rows(c_mod2[i], k, 1)) : 0;
+      b.rmsnorm(NN("n1"), b.all(z), a.n1, b.all(hz), mod1);
+      bool cross_only = d.head == VLA_HEAD_C && (i % 2 == 1);
+      if (!cross_only) {
+        if (aqkv32 >= 0) {
+          Builder::GemmOpt gq; gq.out32 = b.all(aqkv32);
+          b.gemm(NN("qkv"), b.all(hz), a.wqkv, a_nqkv, gq);
+          NodeDesc n;
+          std::memset(&n, 0, sizeof n);
+          n.op = OP_ROPE;
+          RopeArgs& r = n.u.rope;
+          r.in = b.ref(b.all(aqkv32)); r.out = b.ref(b.all(aqkv));
+          r.M = Ta; r.ld = a_nqkv; r.n_rot_heads = d.hq + d.hkv; r.n_heads = d.hq + 2 * d.hkv; r.hd = d.hd; r.pos0 = S;
+          r.rows_per_tile = 4;
+          n.n_tiles = (Ta + 3) / 4;
+          int id = b.add(n, NN("rope"), KIND_ELEM);
+          b.read(id, b.all(aqkv32));
+          b.write(id, b.all(aqkv));
+        } else {
+          Builder::GemmOpt gq; gq.out16 = b.all(aqkv);
+          b.gemm(NN("qkv"), b.all(hz), a.wqkv, a_nqkv, gq);
+        }
+        View att_out = b.rows(aatt, 0, Ta);
+        if (d.head == VLA_HEAD_B) {
+          b.attention(NN("attn"), b.rows(aqkv, 0, Ta, 0), b.rows(qkv[i], 0, S, nq), b.rows(qkv[i], 0, S, nq + nkv), S,
+                      b.rows(aqkv, 0, Ta, a_nq), b.rows(aqkv, 0, Ta, a_nq + a_nkv), Ta, att_out, d.hq, d.hkv, d.hd, false);
+        } else {
+          b.attention(NN("attn"), b.rows(aqkv, 0, Ta, 0), b.rows(aqkv, 0, Ta, a_nq), b.rows(aqkv, 0, Ta, a_nq + a_nkv), Ta,
+                      View(), View(), 0, att_out, d.act_heads, d.act_heads, ahd, false);
+        }
+        Builder::GemmOpt go; go.X = b.all(z); go.out32 = b.all(z);
+        b.gemm(NN("wo"), b.all(aatt), a.wo, da, go);
+      }
+      if (d.head == VLA_HEAD_A) {
+        b.rmsnorm(NN("n2"), b.all(z), a.n2, b.all(hz));
+        Builder::GemmOpt gq; gq.out16 = b.all(aqc);
+        b.gemm(NN("cq"), b.all(hz), a.cq, nq, gq);
+        int kvb = qkv[d.llm_layers - 1];
+        b.attention(NN("xattn"), b.all(aqc), b.rows(kvb, 0, S, nq), b.rows(kvb, 0, S, nq + nkv), S, View(), View(), 0,
+                    b.all(aatt), d.hq, d.hkv, d.hd, false);
+        Builder::GemmOpt go; go.X = b.all(z); go.out32 = b.all(z);
+        b.gemm(NN("co"), b.all(aatt), a.co, da, go);
+        b.rmsnorm(NN("n3"), b.all(z), a.n3, b.all(hz));
+      } else if (cross_only) {
+        Builder::GemmOpt gq; gq.out16 = b.all(aqc);
+        b.gemm(NN("cq"), b.all(hz), a.cq, da, gq);
+        b.attention(NN("xattn"), b.all(aqc), b.rows(ckv[i], 0, S, 0), b.rows(ckv[i], 0, S, da), S, View(), View(), 0,
+                    b.all(aatt), d.act_heads, d.act_heads, ahd, false);
+        Builder::GemmOpt go; go.X = b.all(z); go.out32 = b.all(z);
+        b.gemm(NN("co"), b.all(aatt), a.co, da, go);
+        b.rmsnorm(NN("n2"), b.all(z), a.n2, b.all(hz), mod2);
+      } else {
+        b.rmsnorm(NN("n2"), b.all(z), a.n2, b.all(hz), mod2);
+      }
+      Builder::GemmOpt g1; g1.out16 = b.all(amid);
+      if (agated) {
+        g1.W2 = a.wu;
+        g1.act = d.act_mlp_kind == VLA_MLP_SWIGLU ? ACT_SILU : ACT_GELU;
+        b.gemm(NN("gu"), b.all(hz), a.wg, d.act_mlp, g1);
+      } else {
+        g1.act = ACT_GELU;
+        b.gemm(NN("w1"), b.all(hz), a.w1, d.act_mlp, g1);
+      }
+      Builder::GemmOpt g2; g2.X = b.all(z); g2.out32 = b.all(z);
+      b.gemm(NN("w2"), b.all(amid), agated ? a.wd : a.w2, da, g2);
+    }
+    b.rmsnorm(N_("act.s%d.norm", k), b.all(z), w_anorm, b.all(hz));
+    {
+      Builder::GemmOpt g;
+      g.X = b.all(xs); g.c_x = p.step_c_x[k]; g.c_acc = p.step_c_acc[k];
+      g.out32 = b.all(xs); g.out16 = b.all(xbf);
+      b.gemm(N_("act.s%d.out", k), b.rows(hz, first, d.horizon), w_aout, d.act_dim, g);
+    }
+  }
+  b.step = -1;
+  {
+    NodeDesc n;
+    std::memset(&n, 0, sizeof n);
+    n.op = OP_EMIT;
+    n.u.emit.x = b.ref(b.all(xs));
+    n.u.emit.H = d.horizon; n.u.emit.A = d.act_dim; n.u.emit.ldx = d.act_dim;
+    n.n_tiles = 1;
+    int id = b.add(n, "act.emit", KIND_ELEM);
+    b.read(id, b.all(xs));
+  }
+  if (!p.error.empty()) return false;
+
+  // ================================================================== successors, roots
+  const int nn = (int)p.nodes.size();
+  if (nn >= (1 << 20)) { set_err(p, "tile program too large"); return false; }
+  {
+    // the emit node closes the frame: it also waits for every node nothing else consumes,
+    // so a frame slot is never handed back while one of its tiles is still pending
+    std::vector<char> has_succ(nn, 0);
+    for (int i = 0; i < nn; ++i)
+      for (int q : b.preds[i]) has_succ[q] = 1;
+    for (int i = 0; i < nn - 1; ++i)
+      if (!has_succ[i]) b.preds[nn - 1].push_back(i);
+  }
+  std::vector<std::vector<int>> succ(nn);
+  for (int i = 0; i < nn; ++i) {
+    auto& pr = b.preds[i];
+    std::sort(pr.begin(), pr.end());
+    pr.erase(std::unique(pr.begin(), pr.end()), pr.end());
+    p.nodes[i].n_pred = (int)pr.size();
+    for (int q : pr) succ[q].push_back(i);
+    if (pr.empty()) p.roots.push_back(i);
+  }
+  for (int i = 0; i < nn; ++i) {
+    p.nodes[i].succ_begin = (int)p.succ.size();
+    p.nodes[i].succ_count = (int)succ[i].size();
+    for (int s : succ[i]) p.succ.push_back(s);
+  }
+
+  // ================================================================== per-class tags and resources
+  // (tau_TC, tau_ALU, tau_MEM): hand-assigned intensities per tile class (Section 3.2 of the paper
+  // derives them by profiling; the values below follow the per-class roofline of the tile bodies).
+  const int taus[N_CLASSES][3] = {{15, 2, 3}, {8, 8, 2}, {0, 4, 10}, {2, 3, 12}, {1, 8, 4}, {0, 3, 6}};
+  for (int c = 0; c < N_CLASSES; ++c) {
+    for (int x_ = 0; x_ < 3; ++x_) p.classes[c].tau[x_] = taus[c][x_];
+    p.classes[c].smem_units = 0;
+    p.classes[c].tmem_units = 0;
+    p.classes[c].pad[0] = p.classes[c].pad[1] = p.classes[c].pad[2] = 0;
+  }
+  for (const NodeDesc& n : p.nodes) {
+    ClassInfo& ci = p.classes[n.cls];
+    ci.smem_units = std::max(ci.smem_units, (n.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT);
+    ci.tmem_units = std::max(ci.tmem_units, (n.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT);
+  }
+
+  // ================================================================== arena layout
+  uint64_t cur = b.const_base + b.const_cursor;
+  auto place = [&](uint64_t bytes, uint64_t align = 256) {
+    cur = align_up(cur, align);
+    uint64_t o_ = cur;
+    cur += bytes;
+    return o_;
+  };
+  p.off_weights = Builder::WEIGHT_BASE;
+  p.off_consts = b.const_base;
+  p.zero_bytes_begin = b.const_base;
+  p.off_nodes = place(sizeof(NodeDesc) * p.nodes.size());
+  p.off_init_nodes = place(sizeof(NodeDesc) * p.init_program.size());
+  p.off_succ = place(sizeof(int32_t) * std::max<size_t>(p.succ.size(), 1));
+  p.off_roots = place(sizeof(int32_t) * std::max<size_t>(p.roots.size(), 1));
+  p.off_classes = place(sizeof(ClassInfo) * N_CLASSES);
+  p.off_control = place(sizeof(Control));
+  p.off_queues = place(sizeof(TileQueue) * N_CLASSES);
+  // queue capacity: every tile of every in-flight frame could be queued at once in the worst case
+  uint64_t tiles_per_frame = 0;
+  for (const NodeDesc& n : p.nodes) tiles_per_frame += n.n_tiles;
+  uint64_t want = tiles_per_frame * (uint64_t)p.n_inst + 1024;
+  int cap = 1 << 12;
+  while ((uint64_t)cap < want && cap < (1 << 24)) cap <<= 1;
+  p.q_capacity = cap;
+  p.off_q_entries = place(sizeof(QueueEntry) * (uint64_t)cap * N_CLASSES);
+  p.off_q_seq = place(sizeof(unsigned long long) * (uint64_t)cap * N_CLASSES);
+  p.admit_capacity = 1;
+  while (p.admit_capacity < 2 * p.n_inst) p.admit_capacity <<= 1;
+  p.off_admit = place(sizeof(AdmitRec) * p.admit_capacity);
+  p.off_dep = place(sizeof(int32_t) * (uint64_t)nn * p.n_inst);
+  p.off_tiles_done = place(sizeof(int32_t) * (uint64_t)nn * p.n_inst);
+  p.off_inst_frame = place(sizeof(uint64_t) * p.n_inst);
+  p.off_slot_base = place(sizeof(uint64_t) * p.n_inst);
+  p.trace_capacity = o.trace_capacity;
+  p.off_trace = place(sizeof(TraceRec) * (uint64_t)std::max<uint32_t>(o.trace_capacity, 1));
+  p.off_tmaps = place(128ull * std::max<size_t>(p.tmaps.size() + 1, 1), 128);
+  p.slot_bytes = align_up(b.slot_cursor, 4096);
+  p.off_slots = place(p.slot_bytes * p.n_inst, 4096);
+  p.arena_bytes = align_up(cur, 4096);
+  return true;
+}
+
+}  // namespace vla

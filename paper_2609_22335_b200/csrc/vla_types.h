@@ -1,0 +1,207 @@
+// Shared host/device data structures of the tile program and the dispatcher.
+#pragma once
+#include <stdint.h>
+
+namespace vla {
+
+// ---- operations a node can be (each node splits into n_tiles independent tiles)
+enum Op : int32_t {
+  OP_GEMM = 0,      // out = epilogue(A[M,K] * W[N,K]^T), bf16 operands, fp32 accumulate
+  OP_RMSNORM = 1,   // bf16 out = rmsnorm(x fp32) * g (optionally * (1+gamma) + beta, optional pixel-shuffle scatter)
+  OP_ATTN = 2,      // fused softmax(QK^T/sqrt(hd))V over up to two K/V segments
+  OP_PATCHIFY = 3,  // image fp32 -> bf16 patch rows
+  OP_EMBED = 4,     // text-embedding gather (+ position table) into the fp32 residual stream
+  OP_ROPE = 5,      // fp32 q|k|v rows -> bf16 with rotary embedding on the q and k heads
+  OP_ADDROWS = 6,   // out fp32 [M,N] = in fp32 (+ vec) (+ table)
+  OP_TIMEEMB = 7,   // sinusoidal timestep embedding rows -> bf16
+  OP_EMIT = 8,      // copy the finished chunk to the host-visible ring and publish its frame id
+  OP_COUNT = 9
+};
+
+enum Kind : int32_t { KIND_GEMM = 0, KIND_ATTN = 1, KIND_ELEM = 2 };
+enum Phase : int32_t { PHASE_VLM = 0, PHASE_ACT = 1 };
+constexpr int N_CLASSES = 6;  // phase * 3 + kind
+
+enum Act : int32_t { ACT_NONE = 0, ACT_GELU = 1, ACT_SILU = 2 };
+
+// A device address inside the arena: byte offset, bit 63 set when relative to the
+// frame slot (instance) base rather than the arena base.  0 = null.
+typedef uint64_t Ref;
+constexpr Ref REF_SLOT = 1ull << 63;
+
+constexpr int GEMM_BM = 128;   // output features per GEMM tile (the MMA M dimension)
+constexpr int GEMM_BK = 64;    // K elements per pipeline stage (one 128-byte swizzle row of bf16)
+constexpr int WORKER_THREADS = 128;
+constexpr int GEMM_TOK_CHUNK = 32;   // tokens accumulated per pass of the GEMM body
+constexpr int GEMM_SMEM_BYTES = (GEMM_BM * (GEMM_BK + 4) + GEMM_TOK_CHUNK * GEMM_BK) * 4;
+
+struct GemmArgs {
+  Ref A, W, W2;        // A bf16 [M,lda]; W (and W2 when dual) bf16 [N,Kp]
+  Ref X;               // optional fp32 addend [M,ldx], scaled by c_x
+  Ref vec;             // optional fp32 [N], broadcast over rows
+  Ref tab, tab2;       // optional fp32 tables [M,ldtab] added row by row
+  Ref out32, out16;    // fp32 and/or bf16 outputs [M,ld]
+  int32_t lda, ldx, ldtab, ldtab2, ldo32, ldo16;
+  int32_t M, N, Kp;    // tokens, output features, padded reduction length (multiple of GEMM_BK)
+  int32_t bt, tiles_t; // tokens per tile, number of token tiles
+  int32_t act, dual;   // activation; dual: out = act(A W^T) * (A W2^T)
+  float c_acc, c_x;    // out = c_x * X + c_acc * acc + vec + tab + tab2
+  int32_t amap_inst, wmap;  // tensor-map indices (per-instance A map base, shared W map)
+};
+
+struct NormArgs {
+  Ref x, g, mod, out;  // x fp32 [M,ldx]; g fp32 [d]; mod fp32 [2d] (gamma;beta) or null; out bf16
+  int32_t M, d, ldx, ldo;
+  int32_t rows_per_tile;
+  int32_t shuffle, grid;   // shuffle s>1: row r=(y,x) of a grid x grid token map goes to row (y/s,x/s), column block (y%s,x%s)
+};
+
+struct AttnArgs {
+  Ref q, k0, v0, k1, v1, out;  // bf16; segment 0 then segment 1 along the key axis
+  int32_t ldq, ldk0, ldk1, ldo;
+  int32_t tq, t0, t1;
+  int32_t hq, hkv, hd;
+  int32_t causal;
+  int32_t bq, q_blocks;        // queries per tile
+  float scale;
+};
+
+struct PatchArgs {
+  Ref img, out;        // img fp32 [3,H,W] of one camera; out bf16 [T,ldo]
+  int32_t img_side, patch, grid, ldo, rows_per_tile;
+};
+
+struct EmbedArgs {
+  Ref ids, table, pos, out;   // ids int32 [n]; table bf16 [vocab,d]; pos fp32 [n,d] or null; out fp32 rows
+  int32_t n, d, ldo, vocab, rows_per_tile, ldt;
+};
+
+struct RopeArgs {
+  Ref in, out;         // in fp32 [M,ld]; out bf16 [M,ld]
+  int32_t M, ld, n_rot_heads, n_heads, hd, pos0, rows_per_tile;
+};
+
+struct AddRowsArgs {
+  Ref in, vec, tab, out, out16;  // fp32; out16 optional bf16 copy
+  int32_t M, N, ldi, ldt, ldo, ldo16;
+};
+
+struct TimeEmbArgs {
+  Ref args, out;       // args fp32 [M] time arguments; out bf16 [M,ldo]
+  int32_t M, width, ldo;
+};
+
+struct EmitArgs {
+  Ref x;               // fp32 [H,ldx]
+  int32_t H, A, ldx;
+};
+
+struct NodeDesc {
+  int32_t op, cls, n_tiles, n_pred;
+  int32_t succ_begin, succ_count;
+  int32_t phase, step;
+  int32_t smem_bytes, tmem_cols;
+  int32_t pad0, pad1;
+  union {
+    GemmArgs gemm;
+    NormArgs norm;
+    AttnArgs attn;
+    PatchArgs patch;
+    EmbedArgs embed;
+    RopeArgs rope;
+    AddRowsArgs addrows;
+    TimeEmbArgs timeemb;
+    EmitArgs emit;
+  } u;
+};
+
+// Per-class static description used by the pick.
+struct ClassInfo {
+  int32_t tau[3];       // (TC, ALU, MEM) intensity 0..15
+  int32_t smem_units;   // shared-memory need in SMEM_UNIT chunks
+  int32_t tmem_units;   // tensor-memory need in TMEM_UNIT column chunks
+  int32_t pad[3];
+};
+
+constexpr int SMEM_UNIT = 8192;
+constexpr int TMEM_UNIT = 32;
+
+// A multi-producer multi-consumer ring of tile tickets (one per class).
+struct TileQueue {
+  unsigned long long head;     // next ticket to hand out
+  unsigned long long tail;     // next ticket to reserve for a push
+  long long avail;             // committed minus claimed (may dip below zero transiently)
+  unsigned long long pad;
+};
+
+struct QueueEntry {            // 8 bytes: one tile
+  uint32_t inst_node;          // inst << 20 | node
+  uint32_t tile;
+};
+
+struct AdmitRec {              // written by the host (copy stream), read by the dispatcher
+  uint32_t inst;
+  uint32_t pad;
+  uint64_t frame;
+};
+
+struct TraceRec {              // mirrors vla_trace_rec
+  uint32_t inst, node, tile;
+  uint16_t sm;
+  uint8_t worker, cls;
+  uint64_t frame, t_start, t_end;
+};
+
+// Host-visible completion record per instance (mapped pinned memory).
+struct DoneRec {
+  volatile uint64_t frame_plus1;   // 0 = nothing yet
+  uint64_t pad[7];
+};
+
+// Device-resident control block.
+struct Control {
+  unsigned int ctrl;             // bit 31 = exiting; low bits = frames in flight
+  unsigned int error;            // sticky error code (0 = none)
+  unsigned int error_info;
+  unsigned int stop;             // host request to exit
+  unsigned long long admit_head; // admission records consumed
+  unsigned long long admit_tail; // admission records published (written by host copies)
+  unsigned long long tiles_done;
+  unsigned long long trace_count;
+};
+
+enum DevError : uint32_t {
+  DEV_OK = 0, DEV_ERR_WAIT_QUEUE = 1, DEV_ERR_QUEUE_FULL = 2, DEV_ERR_WAIT_MBAR = 3, DEV_ERR_IDLE_LIMIT = 4,
+  DEV_ERR_BAD_OP = 5
+};
+
+// Everything a kernel needs, passed by value.
+struct DeviceCtx {
+  char* arena;
+  const NodeDesc* nodes;
+  const int32_t* succ;
+  const ClassInfo* classes;
+  Control* control;
+  TileQueue* queues;             // [N_CLASSES]
+  QueueEntry* q_entries;         // [N_CLASSES][q_capacity]
+  unsigned long long* q_seq;     // [N_CLASSES][q_capacity] ticket+1 when the entry is valid
+  AdmitRec* admit_ring;
+  int32_t* dep_count;            // [n_inst][n_nodes]
+  int32_t* tiles_done;           // [n_inst][n_nodes]
+  uint64_t* inst_frame;          // [n_inst] frame id currently owning the slot
+  const uint64_t* slot_base;     // [n_inst] arena offset of the instance's buffers
+  const int32_t* roots;          // nodes without predecessors
+  TraceRec* trace;
+  DoneRec* done_host;            // mapped pinned host memory, [n_inst]
+  float* chunk_host;             // mapped pinned host memory, [n_inst][H*A]
+  unsigned int* error_host;      // mapped pinned host memory
+  const void* tmaps;             // CUtensorMap table (128 B each)
+  int32_t n_nodes, n_inst, n_roots;
+  int32_t q_capacity, admit_capacity;
+  uint32_t trace_capacity;
+  int32_t policy, workers_per_sm;
+  uint64_t wait_limit_ns, idle_exit_ns;
+  int32_t chunk_elems;
+};
+
+}  // namespace vla
