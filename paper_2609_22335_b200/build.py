@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvla_b200.so")
 SOURCES = ["vla_api.cu", "program.cc"]
-HEADERS = ["vla_types.h", "program.h", "tiles.cuh", "dispatch.cuh", "pick.cuh", os.path.join("..", "..", "include", "vla.h")]
+HEADERS = []
 
 
 def _stale() -> bool:
@@ -32,7 +32,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
-    cmd += ["-lcudart", "-lcuda"]
+    cmd += ["-lcudart"]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         sys.stderr.write(r.stdout + r.stderr)

@@ -42,6 +42,15 @@ __device__ __forceinline__ void set_error(const DeviceCtx& ctx, unsigned code, u
   }
 }
 
+// ------------------------------------------------------------------ tensor memory (whole-warp calls)
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
 // ------------------------------------------------------------------ tile queues
 // Push n tiles of (inst, node) to the class queue.  Called by one thread.
 __device__ inline void queue_push(const DeviceCtx& ctx, int cls, uint32_t inst, uint32_t node, int n) {
@@ -268,6 +277,10 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_ke
     sm->tiles = 0;
   }
   __syncthreads();
+  if (threadIdx.x < 32) tmem_alloc(&sm->tmem_base, 512);   // the whole tensor memory of this SM, sub-allocated per tile
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
   Control* ctl = ctx.control;
   const int bar_id = worker + 1;
 
@@ -314,10 +327,13 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_ke
     tc.tid = wt;
     tc.bar_id = bar_id;
     tc.error = &ctl->error;
+    tc.tmaps = ctx.tmaps;
+    tc.amap_base = ctx.n_weight_tmaps + (int)cmd.inst * ctx.n_act_tmaps;
     const uint64_t t0 = gtimer();
     tc.deadline = t0 + ctx.wait_limit_ns;
     const uint64_t frame = *reinterpret_cast<const volatile uint64_t*>(ctx.inst_frame + cmd.inst);
     run_tile(ctx, tc, n, (int)cmd.tile, (int)cmd.inst, frame);
+    asm volatile("fence.proxy.async;" ::: "memory");   // outputs may be read by TMA on another SM
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
     if (wt == 0) {
       const uint64_t t1 = gtimer();
@@ -326,22 +342,36 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_ke
       complete_tile(ctx, cmd.inst, cmd.node, true);
     }
   }
+  tc_fence_before();
   __syncthreads();
+  if (threadIdx.x < 32) tmem_dealloc(sm->tmem_base, 512);
   if (threadIdx.x == 0) atomicAdd(&ctl->tiles_done, sm->tiles);
 }
 
 // ------------------------------------------------------------------ one node as an ordinary kernel (CTA = tile)
 __global__ void __launch_bounds__(WORKER_THREADS) vla_node_kernel(DeviceCtx ctx, const NodeDesc* nodes, int node_idx, int inst) {
   extern __shared__ __align__(1024) char smem_raw[];
+  __shared__ uint32_t tmem_base_s;
   const NodeDesc& n = nodes[node_idx];
+  uint32_t tmem_cols = 0;
+  if (n.tmem_cols > 0) {
+    tmem_cols = 32;
+    while ((int)tmem_cols < n.tmem_cols) tmem_cols <<= 1;
+    if (threadIdx.x < 32) tmem_alloc(&tmem_base_s, tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+  }
   TileCtx tc;
   tc.arena = ctx.arena;
   tc.slot_base = inst >= 0 ? ctx.slot_base[inst] : 0;
   tc.smem = smem_raw;
-  tc.tmem = 0;
+  tc.tmem = tmem_cols ? tmem_base_s : 0;
   tc.tid = threadIdx.x;
   tc.bar_id = 1;
   tc.error = &ctx.control->error;
+  tc.tmaps = ctx.tmaps;
+  tc.amap_base = ctx.n_weight_tmaps + (inst >= 0 ? inst : 0) * ctx.n_act_tmaps;
   const uint64_t t0 = gtimer();
   tc.deadline = t0 + ctx.wait_limit_ns;
   const uint64_t frame = inst >= 0 ? ctx.inst_frame[inst] : 0;
@@ -349,6 +379,11 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_node_kernel(DeviceCtx ctx,
   if (inst >= 0 && ctx.trace_capacity) {
     asm volatile("bar.sync 1, %0;" ::"r"(WORKER_THREADS) : "memory");
     if (threadIdx.x == 0) write_trace(ctx, (uint32_t)inst, (uint32_t)node_idx, blockIdx.x, 0, n.cls, frame, t0, gtimer());
+  }
+  if (tmem_cols) {
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x < 32) tmem_dealloc(tmem_base_s, tmem_cols);
   }
 }
 

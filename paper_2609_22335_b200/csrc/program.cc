@@ -200,9 +200,19 @@ class Builder {
       bt = (int)pad_to((g.M + tiles_t - 1) / tiles_t, 16);
     }
     g.bt = bt; g.tiles_t = tiles_t;
-    g.amap_inst = -1; g.wmap = -1;
+    {
+      // pipeline depth from the stage size; tensor maps for the operands
+      int stage = GEMM_BM * GEMM_BK * 2 * (g.dual ? 2 : 1) + bt * GEMM_BK * 2;
+      int S = std::max(2, std::min(4, GEMM_SMEM_BUDGET / stage));
+      S = std::min(S, std::max(1, g.Kp / GEMM_BK));
+      g.stages = S;
+      n.smem_bytes = 1024 + S * stage;
+      n.tmem_cols = (int)pad_to((int64_t)bt * (g.dual ? 2 : 1), TMEM_UNIT);
+      g.wmap = weight_map(W, N);
+      g.w2map = o.W2 >= 0 ? weight_map(o.W2, N) : 0;
+      g.amap = act_map(A, g.Kp, bt);
+    }
     n.n_tiles = (int)((g.N + GEMM_BM - 1) / GEMM_BM) * tiles_t;
-    n.smem_bytes = GEMM_SMEM_BYTES;
     int id = add(n, name, KIND_GEMM);
     read(id, A);
     if (o.X.buf >= 0) read(id, o.X);
@@ -212,6 +222,30 @@ class Builder {
       p.error = "internal: activation row pitch shorter than padded K in " + name;
     }
     return id;
+  }
+
+  int weight_map(int W, int64_t N) {
+    const DevTensor& t = p.dev_tensors[W];
+    TmapSpec sp{WEIGHT_BASE + t.offset, false, N, t.ld, t.ld, GEMM_BM};
+    for (size_t i = 0; i < p.wmaps.size(); ++i)
+      if (p.wmaps[i].offset == sp.offset && p.wmaps[i].rows == sp.rows) return (int)i;
+    p.wmaps.push_back(sp);
+    return (int)p.wmaps.size() - 1;
+  }
+  int act_map(const View& A, int64_t Kp, int bt) {
+    const BufInfo& bi = p.bufs[A.buf];
+    uint64_t off = bi.offset + (uint64_t)(A.row0 * bi.ld + A.col0) * bi.elem;
+    if (!bi.slot) off += const_base;
+    TmapSpec sp{off, bi.slot, A.rows, Kp, bi.ld, bt};
+    if (A.col0 != 0 || bi.elem != 2) p.error = "internal: GEMM activation view must be bf16 and start at column 0";
+    for (size_t i = 0; i < p.amaps.size(); ++i) {
+      const TmapSpec& q = p.amaps[i];
+      if (q.offset == sp.offset && q.slot == sp.slot && q.rows == sp.rows && q.cols == sp.cols && q.ld == sp.ld &&
+          q.box_rows == sp.box_rows)
+        return (int)i;
+    }
+    p.amaps.push_back(sp);
+    return (int)p.amaps.size() - 1;
   }
 
   int rmsnorm(const std::string& name, const View& x, int g_dev, const View& out, Ref mod = 0, int shuffle = 1,
@@ -827,6 +861,7 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     p.classes[c].pad[0] = p.classes[c].pad[1] = p.classes[c].pad[2] = 0;
   }
   for (const NodeDesc& n : p.nodes) {
+    if (n.smem_bytes > 26 * SMEM_UNIT) { set_err(p, "a tile needs more shared memory than one SM offers"); return false; }
     ClassInfo& ci = p.classes[n.cls];
     ci.smem_units = std::max(ci.smem_units, (n.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT);
     ci.tmem_units = std::max(ci.tmem_units, (n.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT);
@@ -868,7 +903,7 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   p.off_slot_base = place(sizeof(uint64_t) * p.n_inst);
   p.trace_capacity = o.trace_capacity;
   p.off_trace = place(sizeof(TraceRec) * (uint64_t)std::max<uint32_t>(o.trace_capacity, 1));
-  p.off_tmaps = place(128ull * std::max<size_t>(p.tmaps.size() + 1, 1), 128);
+  p.off_tmaps = place(128ull * (p.wmaps.size() + p.amaps.size() * (size_t)p.n_inst + 1), 128);
   p.slot_bytes = align_up(b.slot_cursor, 4096);
   p.off_slots = place(p.slot_bytes * p.n_inst, 4096);
   p.arena_bytes = align_up(cur, 4096);

@@ -61,8 +61,8 @@ struct Program {
   std::map<std::string, int> dev_index;
   std::vector<BufInfo> bufs;
   std::map<std::string, int> buf_index;
-  std::vector<TmapSpec> tmaps;          // weight maps first (shared), then per-instance activation maps
-  int n_weight_tmaps = 0, n_act_tmaps = 0;
+  std::vector<TmapSpec> wmaps;          // weight maps (shared by all frame slots)
+  std::vector<TmapSpec> amaps;          // activation maps, instantiated once per frame slot
 
   // time arguments of the denoising steps and solver coefficients
   std::vector<float> step_args, step_c_x, step_c_acc;

@@ -1,5 +1,6 @@
 // C ABI of the library (see include/vla.h): context set-up, weight upload, frame
 // submission / polling, and the three run modes built on the same tile bodies.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -96,6 +97,43 @@ int check_device_error(vla_ctx* c) {
     c->err = "device-side wait ran out (code " + std::to_string(code) + ")";
     return c->sticky;
   }
+  return VLA_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Encodes every TMA tensor map (2-D bf16, 128-byte swizzle, 64-column boxes, zero fill outside) and uploads the table.
+int build_tensor_maps(vla_ctx* c) {
+  const Program& p = c->prog;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  CU(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (!fn || qres != cudaDriverEntryPointSuccess) return fail(c, VLA_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+  EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
+  const size_t total = p.wmaps.size() + p.amaps.size() * (size_t)p.n_inst;
+  std::vector<CUtensorMap> maps(total + 1);
+  auto enc = [&](const TmapSpec& sp, char* base, CUtensorMap* out) -> bool {
+    cuuint64_t dims[2] = {(cuuint64_t)sp.cols, (cuuint64_t)sp.rows};
+    cuuint64_t strides[1] = {(cuuint64_t)sp.ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)GEMM_BK, (cuuint32_t)sp.box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+  };
+  for (size_t i = 0; i < p.wmaps.size(); ++i)
+    if (!enc(p.wmaps[i], c->arena + p.wmaps[i].offset, &maps[i])) return fail(c, VLA_ERR_CUDA, "weight tensor map %zu rejected", i);
+  for (int inst = 0; inst < p.n_inst; ++inst)
+    for (size_t i = 0; i < p.amaps.size(); ++i) {
+      const TmapSpec& sp = p.amaps[i];
+      char* base = c->arena + sp.offset + (sp.slot ? p.off_slots + (uint64_t)inst * p.slot_bytes : 0);
+      if (!enc(sp, base, &maps[p.wmaps.size() + (size_t)inst * p.amaps.size() + i]))
+        return fail(c, VLA_ERR_CUDA, "activation tensor map %zu rejected", i);
+    }
+  static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+  CU(cudaMemcpy(c->arena + p.off_tmaps, maps.data(), total * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
   return VLA_OK;
 }
 
@@ -330,6 +368,12 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
   CU(cudaHostGetDevicePointer(&dp, c->chunk_host, 0)); x.chunk_host = static_cast<float*>(dp);
   CU(cudaHostGetDevicePointer(&dp, c->error_host, 0)); x.error_host = static_cast<unsigned*>(dp);
   x.tmaps = at<char>(c, p.off_tmaps);
+  x.n_weight_tmaps = (int)p.wmaps.size();
+  x.n_act_tmaps = (int)p.amaps.size();
+  {
+    int rc = build_tensor_maps(c);
+    if (rc != VLA_OK) return rc;
+  }
   x.n_nodes = (int)p.nodes.size();
   x.n_inst = p.n_inst;
   x.n_roots = (int)p.roots.size();

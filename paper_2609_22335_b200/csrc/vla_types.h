@@ -32,8 +32,8 @@ constexpr Ref REF_SLOT = 1ull << 63;
 constexpr int GEMM_BM = 128;   // output features per GEMM tile (the MMA M dimension)
 constexpr int GEMM_BK = 64;    // K elements per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int WORKER_THREADS = 128;
-constexpr int GEMM_TOK_CHUNK = 32;   // tokens accumulated per pass of the GEMM body
-constexpr int GEMM_SMEM_BYTES = (GEMM_BM * (GEMM_BK + 4) + GEMM_TOK_CHUNK * GEMM_BK) * 4;
+constexpr int GEMM_MAX_BT = 256;     // most tokens per GEMM tile (MMA N)
+constexpr int GEMM_SMEM_BUDGET = 80 * 1024;  // stage memory a GEMM tile aims for (at least two stages are always taken)
 
 struct GemmArgs {
   Ref A, W, W2;        // A bf16 [M,lda]; W (and W2 when dual) bf16 [N,Kp]
@@ -46,7 +46,8 @@ struct GemmArgs {
   int32_t bt, tiles_t; // tokens per tile, number of token tiles
   int32_t act, dual;   // activation; dual: out = act(A W^T) * (A W2^T)
   float c_acc, c_x;    // out = c_x * X + c_acc * acc + vec + tab + tab2
-  int32_t amap_inst, wmap;  // tensor-map indices (per-instance A map base, shared W map)
+  int32_t wmap, w2map, amap;  // tensor-map indices: shared weight maps, activation map relative to the slot's first
+  int32_t stages;             // TMA pipeline depth
 };
 
 struct NormArgs {
@@ -195,7 +196,8 @@ struct DeviceCtx {
   DoneRec* done_host;            // mapped pinned host memory, [n_inst]
   float* chunk_host;             // mapped pinned host memory, [n_inst][H*A]
   unsigned int* error_host;      // mapped pinned host memory
-  const void* tmaps;             // CUtensorMap table (128 B each)
+  const void* tmaps;             // CUtensorMap table (128 B each): weight maps, then n_act_tmaps per frame slot
+  int32_t n_weight_tmaps, n_act_tmaps;
   int32_t n_nodes, n_inst, n_roots;
   int32_t q_capacity, admit_capacity;
   uint32_t trace_capacity;
