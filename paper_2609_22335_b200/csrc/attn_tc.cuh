@@ -1,0 +1,215 @@
+// Fused attention tile on tcgen05 / tensor memory.
+//
+// One tile = one query head x 128 queries.  Per block of bn keys:
+//   S = Q K^T          tcgen05.mma, Q and K tiles K-major (head dim contiguous), S in TMEM
+//   online softmax     one thread per query row reads its S row from TMEM (no shuffles),
+//                      writes P as bf16 into 128-byte-swizzled shared memory
+//   O += P V           tcgen05.mma, P from shared memory, V consumed from its transposed
+//                      copy V^T [head dim, tokens] so that it too is K-major; O in TMEM,
+//                      rescaled in place when a row maximum moves
+// Keys come from up to two segments (cached prefix K/V, then the head's own K/V); blocks
+// never straddle segments.  Head dims are handled in 16-wide K steps, so a head padded to
+// a multiple of 16 (72 -> 80) costs only its padding.  All waits are bounded.
+#pragma once
+#include "gemm_tc.cuh"
+
+namespace vla {
+
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t umma_idesc_bf16_n(int n) { return umma_idesc_bf16(n); }
+
+constexpr int ATTN_BQ = 128;
+
+// Barrier over the worker's threads that also ANDs a predicate, so every thread takes the same exit.
+__device__ __forceinline__ bool worker_all(const TileCtx& c, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %3, 0;\n\t"
+      "barrier.cta.red.and.pred p, %1, %2, q;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(c.bar_id), "r"(WORKER_THREADS), "r"((uint32_t)pred)
+      : "memory");
+  return r != 0;
+}
+
+__device__ void tile_attention(const TileCtx& c, const AttnArgs& a, int tile) {
+  const int warp = c.tid >> 5, lane = c.tid & 31;
+  const int head = tile / a.q_blocks, qb = tile % a.q_blocks;
+  const int g = (head * a.hkv) / a.hq;
+  const int q0 = qb * ATTN_BQ;
+  const int hs = a.hs, bn = a.bn;
+  const int nbox = (hs + 63) / 64;          // 64-column boxes covering one head
+  const int kchunks = hs / 16;              // 16-wide K steps of Q K^T
+  const int nsub = bn / 64;                 // 64-key sub-tiles of P and V^T
+
+  // shared-memory carve-up (all tile bases 1024-byte aligned)
+  const uint32_t base = smem_u32(c.smem);
+  const uint32_t bar_q = base, bar_k = base + 8, bar_v = base + 16, bar_s = base + 24, bar_o = base + 32;
+  const uint32_t Qs = base + 1024;
+  const uint32_t Ks = Qs + (uint32_t)nbox * (ATTN_BQ * 128);
+  const uint32_t Vs = Ks + (uint32_t)nbox * (uint32_t)(bn * 128);
+  const uint32_t Ps = Vs + (uint32_t)nsub * (uint32_t)(hs * 128);
+  char* Ps_gen = c.smem + (Ps - base);
+
+  if (c.tid == 0) {
+    mbar_init(bar_q, 1); mbar_init(bar_k, 1); mbar_init(bar_v, 1); mbar_init(bar_s, 1); mbar_init(bar_o, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  worker_sync(c);
+
+  const uint32_t tmem_s = c.tmem;                       // S: columns [0, bn)
+  const uint32_t tmem_o = c.tmem + (uint32_t)bn;        // O: columns [bn, bn + hs)
+  const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+  const char* tm = reinterpret_cast<const char*>(c.tmaps);
+  auto map_ptr = [&](int idx) { return reinterpret_cast<const void*>(tm + (size_t)(c.amap_base + idx) * 128); };
+  const uint32_t idesc_s = umma_idesc_bf16(bn), idesc_o = umma_idesc_bf16(hs);
+
+  if (c.tid == 0) {
+    asm volatile("fence.proxy.async;" ::: "memory");
+    mbar_expect_tx(bar_q, (uint32_t)nbox * (ATTN_BQ * 128));
+    for (int b = 0; b < nbox; ++b) tma_load_2d(Qs + (uint32_t)b * (ATTN_BQ * 128), map_ptr(a.qmap), bar_q, head * hs + b * 64, q0);
+  }
+
+  const int row = q0 + warp * 32 + lane;                // this thread's query
+  float m_run = -INFINITY, l_run = 0.f;
+  int blk = 0;
+  bool ok = true;
+  for (int seg = 0; seg < 2 && ok; ++seg) {
+    const int L = seg == 0 ? a.t0 : a.t1;
+    const int kmap = seg == 0 ? a.k0map : a.k1map, vmap = seg == 0 ? a.v0map : a.v1map;
+    for (int kv0 = 0; kv0 < L && ok; kv0 += bn, ++blk) {
+      if (a.causal && kv0 > q0 + ATTN_BQ - 1) break;    // whole block above the diagonal
+      const uint32_t ph = (uint32_t)blk & 1u;
+      if (c.tid == 0) {
+        // K and V^T of this block (single-buffered: the previous block's MMAs have completed)
+        mbar_expect_tx(bar_k, (uint32_t)nbox * (uint32_t)(bn * 128));
+        for (int b = 0; b < nbox; ++b) tma_load_2d(Ks + (uint32_t)b * (uint32_t)(bn * 128), map_ptr(kmap), bar_k, g * hs + b * 64, kv0);
+        mbar_expect_tx(bar_v, (uint32_t)nsub * (uint32_t)(hs * 128));
+        for (int j = 0; j < nsub; ++j) tma_load_2d(Vs + (uint32_t)j * (uint32_t)(hs * 128), map_ptr(vmap), bar_v, kv0 + j * 64, g * hs);
+        ok = (blk > 0 || mbar_wait(c, bar_q, 0u)) && mbar_wait(c, bar_k, ph);
+        if (ok) {
+          tc_fence_after();
+          for (int kc = 0; kc < kchunks; ++kc) {
+            const uint64_t qd = umma_desc_sw128(Qs + (uint32_t)(kc >> 2) * (ATTN_BQ * 128)) + 2u * (kc & 3);
+            const uint64_t kd = umma_desc_sw128(Ks + (uint32_t)(kc >> 2) * (uint32_t)(bn * 128)) + 2u * (kc & 3);
+            umma_bf16(tmem_s, qd, kd, idesc_s, kc != 0 ? 1u : 0u);
+          }
+          umma_commit(bar_s);
+        }
+      }
+      // ---- softmax of this block, one thread per query row
+      ok = worker_all(c, mbar_wait(c, bar_s, ph));
+      tc_fence_after();
+      if (!ok) break;
+      const int valid = min(bn, L - kv0);
+      const int lim = a.causal ? min(valid, row - kv0 + 1) : valid;   // keys [0, lim) of the block are visible to this row
+      float mx = m_run;
+      for (int c0 = 0; c0 < bn; c0 += 16) {
+        float s[16];
+        tmem_ld16(tmem_s + lane_off + (uint32_t)c0, s);
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (c0 + j < lim) mx = fmaxf(mx, s[j]);
+      }
+      const float alpha = (m_run == -INFINITY) ? 0.f : exp2f((m_run - mx) * a.scale_log2e);
+      float sum = 0.f;
+      for (int c0 = 0; c0 < bn; c0 += 16) {
+        float s[16];
+        tmem_ld16(tmem_s + lane_off + (uint32_t)c0, s);
+        uint32_t packed[8];
+#pragma unroll
+        for (int j = 0; j < 16; j += 2) {
+          float p0 = (c0 + j < lim) ? exp2f((s[j] - mx) * a.scale_log2e) : 0.f;
+          float p1 = (c0 + j + 1 < lim) ? exp2f((s[j + 1] - mx) * a.scale_log2e) : 0.f;
+          // the row sum uses the bf16-rounded probabilities the MMA will see
+          __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+          sum += __low2float(pk) + __high2float(pk);
+          packed[j >> 1] = *reinterpret_cast<uint32_t*>(&pk);
+        }
+        // two 16-byte chunks of this row in the swizzled P tile
+        const int r = warp * 32 + lane;
+        const int sub = c0 >> 6, ch = (c0 & 63) >> 3;
+        char* prow = Ps_gen + (size_t)sub * (ATTN_BQ * 128) + (size_t)r * 128;
+        *reinterpret_cast<uint4*>(prow + (((ch) ^ (r & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        *reinterpret_cast<uint4*>(prow + (((ch + 1) ^ (r & 7)) << 4)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+      }
+      l_run = l_run * alpha + sum;
+      m_run = mx;
+      // rescale O where a row maximum moved (warp-uniform decision: the TMEM accesses are warp-wide)
+      if (blk > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
+        for (int c0 = 0; c0 < hs; c0 += 16) {
+          float o[16];
+          tmem_ld16(tmem_o + lane_off + (uint32_t)c0, o);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) o[j] *= alpha;
+          tmem_st16(tmem_o + lane_off + (uint32_t)c0, o);
+        }
+        tmem_st_wait();
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P written by generic stores, read by the MMA
+      tc_fence_before();
+      worker_sync(c);
+      if (c.tid == 0) {
+        ok = mbar_wait(c, bar_v, ph);
+        if (ok) {
+          tc_fence_after();
+          for (int kc = 0; kc < bn / 16; ++kc) {
+            const uint64_t pd = umma_desc_sw128(Ps + (uint32_t)(kc >> 2) * (ATTN_BQ * 128)) + 2u * (kc & 3);
+            const uint64_t vd = umma_desc_sw128(Vs + (uint32_t)(kc >> 2) * (uint32_t)(hs * 128)) + 2u * (kc & 3);
+            umma_bf16(tmem_o, pd, vd, idesc_o, (blk | kc) != 0 ? 1u : 0u);
+          }
+          umma_commit(bar_o);
+          ok = mbar_wait(c, bar_o, ph);     // K, V^T and P buffers are free again
+        }
+      }
+    }
+  }
+  // ---- epilogue: O / l -> bf16
+  worker_sync(c);    // thread 0 has seen the last P V complete
+  tc_fence_after();
+  const bool failed = *reinterpret_cast<volatile unsigned*>(c.error) != 0u;
+  if (!failed && blk > 0) {
+    unsigned short* O = resolve<unsigned short>(c, a.out);
+    const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
+    for (int c0 = 0; c0 < hs; c0 += 16) {
+      float o[16];
+      tmem_ld16(tmem_o + lane_off + (uint32_t)c0, o);
+      if (row < a.tq) {
+        uint32_t pk[8];
+#pragma unroll
+        for (int j = 0; j < 16; j += 2) {
+          __nv_bfloat162 v = __floats2bfloat162_rn(o[j] * inv, o[j + 1] * inv);
+          pk[j >> 1] = *reinterpret_cast<uint32_t*>(&v);
+        }
+        unsigned short* dst = O + (size_t)row * a.ldo + head * a.hd + c0;
+        if (c0 + 16 <= a.hd) {
+          *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          *reinterpret_cast<uint4*>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+        } else {
+          for (int j = 0; j < 16 && c0 + j < a.hd; ++j)
+            dst[j] = (unsigned short)((j & 1) ? (pk[j >> 1] >> 16) : (pk[j >> 1] & 0xFFFFu));
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  worker_sync(c);
+  if (c.tid == 0) {
+    mbar_inval(bar_q); mbar_inval(bar_k); mbar_inval(bar_v); mbar_inval(bar_s); mbar_inval(bar_o);
+  }
+}
+
+}  // namespace vla

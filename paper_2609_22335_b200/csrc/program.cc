@@ -102,6 +102,26 @@ class Builder {
     return d;
   }
   int matrix1(const std::string& name, int64_t rows, int64_t cols) { return matrix(name, {name}, {rows}, cols); }
+  // stacked per-head projections whose heads are padded from hd to hs rows (padding rows stay zero)
+  int matrix_heads(const std::string& dev_name, const std::vector<std::string>& parts, const std::vector<int64_t>& part_heads,
+                   int64_t hd, int64_t hs, int64_t cols) {
+    if (hd == hs) {
+      std::vector<int64_t> r;
+      for (auto h : part_heads) r.push_back(h * hd);
+      return matrix(dev_name, parts, r, cols);
+    }
+    int64_t heads = 0;
+    for (auto h : part_heads) heads += h;
+    int d = dev_tensor(dev_name, heads * hs, cols, true);
+    int64_t off = 0;
+    for (size_t i = 0; i < parts.size(); ++i) {
+      source(parts[i], part_heads[i] * hd, cols, d, off);
+      p.sources.back().group_rows = hd;
+      p.sources.back().group_stride = hs;
+      off += part_heads[i] * hs;
+    }
+    return d;
+  }
   int table(const std::string& name, int64_t rows, int64_t cols) {   // fp32 position table
     int d = dev_tensor(name, rows, cols, false);
     source(name, rows, cols, d, 0);
@@ -171,7 +191,8 @@ class Builder {
     Ref vec = 0;
     Ref tab = 0; int ldtab = 0;
     Ref tab2 = 0; int ldtab2 = 0;
-    View out32, out16;
+    View out32, out16, outT;
+    int t_col0 = 0;
     int act = ACT_NONE;
     int W2 = -1;
     int64_t w_row0 = 0;
@@ -192,6 +213,7 @@ class Builder {
     g.vec = o.vec; g.tab = o.tab; g.ldtab = o.ldtab; g.tab2 = o.tab2; g.ldtab2 = o.ldtab2;
     g.out32 = ref(o.out32); g.ldo32 = o.out32.buf >= 0 ? (int)ld(o.out32) : 0;
     g.out16 = ref(o.out16); g.ldo16 = o.out16.buf >= 0 ? (int)ld(o.out16) : 0;
+    g.outT = ref(o.outT); g.ldoT = o.outT.buf >= 0 ? (int)ld(o.outT) : 0; g.t_col0 = o.t_col0;
     g.act = o.act;
     int tiles_t = (int)((g.M + 255) / 256);
     int bt = (int)pad_to((g.M + tiles_t - 1) / tiles_t, 16);
@@ -218,6 +240,7 @@ class Builder {
     if (o.X.buf >= 0) read(id, o.X);
     if (o.out32.buf >= 0) write(id, o.out32);
     if (o.out16.buf >= 0) write(id, o.out16);
+    if (o.outT.buf >= 0) write(id, o.outT);
     if (A.rows * 1 > 0 && p.bufs[A.buf].ld < wt.ld && !init_mode) {
       p.error = "internal: activation row pitch shorter than padded K in " + name;
     }
@@ -232,12 +255,12 @@ class Builder {
     p.wmaps.push_back(sp);
     return (int)p.wmaps.size() - 1;
   }
-  int act_map(const View& A, int64_t Kp, int bt) {
+  int act_map(const View& A, int64_t cols, int box_rows) {
     const BufInfo& bi = p.bufs[A.buf];
     uint64_t off = bi.offset + (uint64_t)(A.row0 * bi.ld + A.col0) * bi.elem;
     if (!bi.slot) off += const_base;
-    TmapSpec sp{off, bi.slot, A.rows, Kp, bi.ld, bt};
-    if (A.col0 != 0 || bi.elem != 2) p.error = "internal: GEMM activation view must be bf16 and start at column 0";
+    TmapSpec sp{off, bi.slot, A.rows, cols, bi.ld, box_rows};
+    if ((A.col0 * 2) % 16 != 0 || bi.elem != 2) p.error = "internal: TMA view must be bf16 and start on a 16-byte boundary";
     for (size_t i = 0; i < p.amaps.size(); ++i) {
       const TmapSpec& q = p.amaps[i];
       if (q.offset == sp.offset && q.slot == sp.slot && q.rows == sp.rows && q.cols == sp.cols && q.ld == sp.ld &&
@@ -264,26 +287,79 @@ class Builder {
     return id;
   }
 
-  int attention(const std::string& name, const View& q, const View& k0, const View& v0, int t0, const View& k1,
-                const View& v1, int t1, const View& out, int hq, int hkv, int hd, bool causal) {
+  // A projected q|k buffer plus the transposed V buffer of one attention input.
+  struct QKV {
+    int qk = -1, vt = -1;      // qk bf16 [T, (hq+hkv)*hs]; vt bf16 [hkv*hs, pad64(T)]
+    int T = 0, hq = 0, hkv = 0, hs = 0;
+  };
+  QKV make_qkv(const std::string& name, int T, int hq, int hkv, int hs) {
+    QKV q;
+    q.T = T; q.hq = hq; q.hkv = hkv; q.hs = hs;
+    q.qk = buf(name + ".qk", T, (int64_t)(hq + hkv) * hs, 2);
+    q.vt = buf(name + ".vt", (int64_t)hkv * hs, pad_to(T, 64), 2);
+    return q;
+  }
+
+  // Fused attention of the queries in `q` (rows [0,tq), head h at column h*hs) over the keys/values of
+  // kv0 (all its T tokens) and then, optionally, kv1.
+  int attention(const std::string& name, const View& q, int tq, const QKV& kv0, const QKV* kv1, const View& out, int hq,
+                int hkv, int hd, int hs, bool causal) {
     NodeDesc n;
     std::memset(&n, 0, sizeof(n));
     n.op = OP_ATTN;
     AttnArgs& a = n.u.attn;
-    a.q = ref(q); a.k0 = ref(k0); a.v0 = ref(v0); a.k1 = ref(k1); a.v1 = ref(v1); a.out = ref(out);
-    a.ldq = (int)ld(q); a.ldk0 = k0.buf >= 0 ? (int)ld(k0) : 0; a.ldk1 = k1.buf >= 0 ? (int)ld(k1) : 0;
-    a.ldo = (int)ld(out);
-    a.tq = (int)q.rows; a.t0 = t0; a.t1 = t1; a.hq = hq; a.hkv = hkv; a.hd = hd; a.causal = causal;
-    a.bq = 16; a.q_blocks = (a.tq + a.bq - 1) / a.bq;
-    a.scale = 1.0f / std::sqrt((float)hd);
+    a.out = ref(out); a.ldo = (int)ld(out);
+    a.tq = tq; a.t0 = kv0.T; a.t1 = kv1 ? kv1->T : 0;
+    a.hq = hq; a.hkv = hkv; a.hd = hd; a.hs = hs; a.causal = causal;
+    a.bn = hs <= 64 ? 128 : 64;
+    a.q_blocks = (tq + 127) / 128;
+    a.scale_log2e = 1.4426950408889634f / std::sqrt((float)hd);
+    const int nbox = (hs + 63) / 64, nsub = a.bn / 64;
+    n.smem_bytes = 1024 + nbox * 128 * 128 + nbox * a.bn * 128 + nsub * hs * 128 + nsub * 128 * 128;
+    n.tmem_cols = (int)pad_to(a.bn + hs, TMEM_UNIT);
     n.n_tiles = hq * a.q_blocks;
-    n.smem_bytes = 4 * (hd + t0 + t1) * 4 + 256;
+    // tensor maps: Q rows in 128-row boxes, K rows in bn-row boxes, V^T in hs-row boxes of 64 tokens
+    const int64_t qcols = ld(q) - q.col0;
+    a.qmap = act_map(q, qcols, 128);
+    auto kview = [&](const QKV& s_) { return rows(s_.qk, 0, s_.T, (int64_t)s_.hq * s_.hs); };
+    a.k0map = act_map(kview(kv0), (int64_t)kv0.hkv * kv0.hs, a.bn);
+    a.v0map = act_map(all(kv0.vt), kv0.T, hs);
+    if (kv1) {
+      a.k1map = act_map(kview(*kv1), (int64_t)kv1->hkv * kv1->hs, a.bn);
+      a.v1map = act_map(all(kv1->vt), kv1->T, hs);
+    }
     int id = add(n, name, KIND_ATTN);
     read(id, q);
-    if (k0.buf >= 0) { read(id, k0); if (v0.buf != k0.buf) read(id, v0); }
-    if (k1.buf >= 0 && k1.buf != q.buf) { read(id, k1); if (v1.buf != k1.buf) read(id, v1); }
+    read(id, all(kv0.qk)); read(id, all(kv0.vt));
+    if (kv1) { read(id, all(kv1->qk)); read(id, all(kv1->vt)); }
     write(id, out);
     return id;
+  }
+
+  // q|k|v projection of `A` into `dst`: one GEMM whose V columns are written transposed; with RoPE the
+  // GEMM writes fp32 and a rotary tile produces the bf16 q|k and V^T.
+  void qkv_project(const std::string& name, const View& A, int W, const QKV& dst, int hd, int scratch32, int pos0) {
+    const int64_t nqk = (int64_t)(dst.hq + dst.hkv) * dst.hs, nall = nqk + (int64_t)dst.hkv * dst.hs;
+    if (scratch32 >= 0) {
+      GemmOpt gq; gq.out32 = all(scratch32);
+      gemm(name + "qkv", A, W, nall, gq);
+      NodeDesc n;
+      std::memset(&n, 0, sizeof n);
+      n.op = OP_ROPE;
+      RopeArgs& r = n.u.rope;
+      r.in = ref(all(scratch32)); r.out = ref(all(dst.qk)); r.outT = ref(all(dst.vt));
+      r.M = dst.T; r.ld = (int)nall; r.ldo = (int)nqk; r.ldoT = (int)p.bufs[dst.vt].ld;
+      r.n_rot_heads = dst.hq + dst.hkv; r.n_heads = dst.hq + 2 * dst.hkv; r.hd = hd; r.pos0 = pos0;
+      r.rows_per_tile = 4;
+      n.n_tiles = (dst.T + 3) / 4;
+      int id = add(n, name + "rope", KIND_ELEM);
+      read(id, all(scratch32));
+      write(id, all(dst.qk));
+      write(id, all(dst.vt));
+    } else {
+      GemmOpt gq; gq.out16 = all(dst.qk); gq.outT = all(dst.vt); gq.t_col0 = (int)nqk;
+      gemm(name + "qkv", A, W, nall, gq);
+    }
   }
 
   int elem_node(NodeDesc& n, const std::string& name) { return add(n, name, KIND_ELEM); }
@@ -382,7 +458,10 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   const bool head_pos = !(d.head == VLA_HEAD_B && d.rope);
   const bool gated = d.mlp_kind != VLA_MLP_GELU, agated = d.act_mlp_kind != VLA_MLP_GELU;
   const int hvd = d.vis_heads * d.vis_hd;
-  const int nq = d.hq * d.hd, nkv = d.hkv * d.hd, nqkv = nq + 2 * nkv;
+  const int vhs = (int)pad_to(std::max(d.vis_hd, 1), 16);          // vision head stride (72 -> 80)
+  const int lhs = (int)pad_to(d.hd, 16);                            // LLM head stride
+  const int nq = d.hq * d.hd, nkv = d.hkv * d.hd, nqkv = (d.hq + 2 * d.hkv) * lhs;
+  if (lhs != d.hd) { set_err(p, "LLM head dimension must be a multiple of 16"); return false; }
   auto P64 = [](int64_t x) { return pad_to(x, GEMM_BK); };
   char nm[96];
   auto N_ = [&](const char* fmt, int a = 0, int c = 0) { std::snprintf(nm, sizeof nm, fmt, a, c); return std::string(nm); };
@@ -395,7 +474,8 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   for (int i = 0; i < d.vis_layers; ++i) {
     std::string pre = N_("vis.L%d.", i);
     venc[i].n1 = b.gain(pre + "n1", dv);
-    venc[i].wqkv = b.matrix(pre + "wqkv", {pre + "wq", pre + "wk", pre + "wv"}, {hvd, hvd, hvd}, dv);
+    venc[i].wqkv = b.matrix_heads(pre + "wqkv", {pre + "wq", pre + "wk", pre + "wv"},
+                                  {d.vis_heads, d.vis_heads, d.vis_heads}, d.vis_hd, vhs, dv);
     venc[i].wo = b.matrix1(pre + "wo", dv, hvd);
     venc[i].n2 = b.gain(pre + "n2", dv);
     venc[i].w1 = b.matrix1(pre + "w1", d.vis_mlp, dv);
@@ -547,15 +627,16 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   int x = b.buf("llm.x", S, D, 4);
   int h = b.buf("llm.h", S, P64(D), 2);
   int qkv32 = d.rope ? b.buf("llm.qkv32", S, nqkv, 4) : -1;
-  std::vector<int> qkv(d.llm_layers);
+  std::vector<Builder::QKV> lq(d.llm_layers);
   {
-    int shared = -1;
+    bool have_shared = false;
+    Builder::QKV shared;
     for (int i = 0; i < d.llm_layers; ++i) {
       bool own = d.handoff == VLA_HANDOFF_KV_ALL || (d.handoff == VLA_HANDOFF_KV_LAST && i == d.llm_layers - 1);
-      if (own) qkv[i] = b.buf(N_("llm.qkv.%d", i), S, nqkv, 2);
+      if (own) lq[i] = b.make_qkv(N_("llm.qkv.%d", i), S, d.hq, d.hkv, lhs);
       else {
-        if (shared < 0) shared = b.buf("llm.qkv", S, nqkv, 2);
-        qkv[i] = shared;
+        if (!have_shared) { shared = b.make_qkv("llm.qkv", S, d.hq, d.hkv, lhs); have_shared = true; }
+        lq[i] = shared;
       }
     }
   }
@@ -592,7 +673,8 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     }
     int xv = b.buf(N_("vis%d.x", c), T, dv, 4);
     int hv = b.buf(N_("vis%d.h", c), T, P64(dv), 2);
-    int vqkv = d.vis_layers > 0 ? b.buf(N_("vis%d.qkv", c), T, 3 * hvd, 2) : -1;
+    Builder::QKV vq;
+    if (d.vis_layers > 0) vq = b.make_qkv(N_("vis%d.qkv", c), T, d.vis_heads, d.vis_heads, vhs);
     int vatt = d.vis_layers > 0 ? b.buf(N_("vis%d.att", c), T, P64(hvd), 2) : -1;
     int vmid = d.vis_layers > 0 ? b.buf(N_("vis%d.mid", c), T, P64(d.vis_mlp), 2) : -1;
     int shuf = b.buf(N_("vis%d.shuf", c), tpc, P64((int64_t)d.shuffle * d.shuffle * dv), 2);
@@ -604,10 +686,9 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     }
     for (int i = 0; i < d.vis_layers; ++i) {
       b.rmsnorm(N_("vis%d.L%d.n1", c, i), b.all(xv), venc[i].n1, b.all(hv));
-      Builder::GemmOpt gq; gq.out16 = b.all(vqkv);
-      b.gemm(N_("vis%d.L%d.qkv", c, i), b.all(hv), venc[i].wqkv, 3 * hvd, gq);
-      b.attention(N_("vis%d.L%d.attn", c, i), b.rows(vqkv, 0, T, 0), b.rows(vqkv, 0, T, hvd), b.rows(vqkv, 0, T, 2 * hvd),
-                  T, View(), View(), 0, b.all(vatt), d.vis_heads, d.vis_heads, d.vis_hd, false);
+      b.qkv_project(N_("vis%d.L%d.", c, i), b.all(hv), venc[i].wqkv, vq, d.vis_hd, -1, 0);
+      b.attention(N_("vis%d.L%d.attn", c, i), b.rows(vq.qk, 0, T, 0), T, vq, nullptr, b.all(vatt), d.vis_heads, d.vis_heads,
+                  d.vis_hd, vhs, false);
       Builder::GemmOpt go; go.X = b.all(xv); go.out32 = b.all(xv);
       b.gemm(N_("vis%d.L%d.wo", c, i), b.all(vatt), venc[i].wo, dv, go);
       b.rmsnorm(N_("vis%d.L%d.n2", c, i), b.all(xv), venc[i].n2, b.all(hv));
@@ -642,26 +723,9 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   }
   for (int i = 0; i < d.llm_layers; ++i) {
     b.rmsnorm(N_("llm.L%d.n1", i), b.all(x), lw[i].n1, b.all(h));
-    if (d.rope) {
-      Builder::GemmOpt gq; gq.out32 = b.all(qkv32);
-      b.gemm(N_("llm.L%d.qkv", i), b.all(h), lw[i].wqkv, nqkv, gq);
-      NodeDesc n;
-      std::memset(&n, 0, sizeof n);
-      n.op = OP_ROPE;
-      RopeArgs& a = n.u.rope;
-      a.in = b.ref(b.all(qkv32)); a.out = b.ref(b.all(qkv[i]));
-      a.M = S; a.ld = nqkv; a.n_rot_heads = d.hq + d.hkv; a.n_heads = d.hq + 2 * d.hkv; a.hd = d.hd; a.pos0 = 0;
-      a.rows_per_tile = 4;
-      n.n_tiles = (S + 3) / 4;
-      int id = b.add(n, N_("llm.L%d.rope", i), KIND_ELEM);
-      b.read(id, b.all(qkv32));
-      b.write(id, b.all(qkv[i]));
-    } else {
-      Builder::GemmOpt gq; gq.out16 = b.all(qkv[i]);
-      b.gemm(N_("llm.L%d.qkv", i), b.all(h), lw[i].wqkv, nqkv, gq);
-    }
-    b.attention(N_("llm.L%d.attn", i), b.rows(qkv[i], 0, S, 0), b.rows(qkv[i], 0, S, nq), b.rows(qkv[i], 0, S, nq + nkv), S,
-                View(), View(), 0, b.all(att), d.hq, d.hkv, d.hd, d.causal != 0);
+    b.qkv_project(N_("llm.L%d.", i), b.all(h), lw[i].wqkv, lq[i], d.hd, qkv32, 0);
+    b.attention(N_("llm.L%d.attn", i), b.rows(lq[i].qk, 0, S, 0), S, lq[i], nullptr, b.all(att), d.hq, d.hkv, d.hd, lhs,
+                d.causal != 0);
     Builder::GemmOpt go; go.X = b.all(x); go.out32 = b.all(x);
     b.gemm(N_("llm.L%d.wo", i), b.all(att), lw[i].wo, D, go);
     b.rmsnorm(N_("llm.L%d.n2", i), b.all(x), lw[i].n2, b.all(h));
@@ -678,25 +742,26 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     b.gemm(N_("llm.L%d.w2", i), b.all(mid), gated ? lw[i].wd : lw[i].w2, D, g2);
   }
   b.rmsnorm("llm.norm", b.all(x), w_lnorm, b.all(hidden));
-  std::vector<int> ckv(d.act_layers, -1);
+  const int ahd = d.head == VLA_HEAD_B ? d.hd : da / d.act_heads;
+  const int ahs = (int)pad_to(ahd, 16);
+  if (ahs != ahd) { set_err(p, "action-head head dimension must be a multiple of 16"); return false; }
+  std::vector<Builder::QKV> ckv(d.act_layers);
   if (d.head == VLA_HEAD_C)
     for (int i = 1; i < d.act_layers; i += 2) {
-      ckv[i] = b.buf(N_("act.ckv.%d", i), S, 2 * da, 2);
-      Builder::GemmOpt g; g.out16 = b.all(ckv[i]);
-      b.gemm(N_("act.L%d.ckv", i), b.all(hidden), aw[i].ckv, 2 * da, g);
+      ckv[i] = b.make_qkv(N_("act.ckv.%d", i), S, 0, d.act_heads, ahs);
+      b.qkv_project(N_("act.L%d.c", i), b.all(hidden), aw[i].ckv, ckv[i], ahd, -1, 0);
     }
 
   // ================================================================== action-head phase
   b.phase = PHASE_ACT;
   b.step = -1;
-  const int ahd = d.head == VLA_HEAD_B ? d.hd : da / d.act_heads;
-  const int a_nq = d.head == VLA_HEAD_B ? nq : da, a_nkv = d.head == VLA_HEAD_B ? nkv : da;
-  const int a_nqkv = a_nq + 2 * a_nkv;
+  const int a_hq = d.head == VLA_HEAD_B ? d.hq : d.act_heads, a_hkv = d.head == VLA_HEAD_B ? d.hkv : d.act_heads;
+  const int a_nq = a_hq * ahs, a_nqkv = (a_hq + 2 * a_hkv) * ahs;
   int xs = b.buf("act.x", d.horizon, d.act_dim, 4);
   int xbf = b.buf("act.xbf", d.horizon, P64(d.act_dim), 2);
   int z = b.buf("act.z", Ta, da, 4);
   int hz = b.buf("act.h", Ta, P64(da), 2);
-  int aqkv = b.buf("act.qkv", Ta, a_nqkv, 2);
+  Builder::QKV aq = b.make_qkv("act.qkv", Ta, a_hq, a_hkv, ahs);
   int aqkv32 = (d.head == VLA_HEAD_B && d.rope) ? b.buf("act.qkv32", Ta, a_nqkv, 4) : -1;
   int aatt = b.buf("act.att", Ta, P64(std::max(a_nq, nq)), 2);
   int aqc = (d.head == VLA_HEAD_A || d.head == VLA_HEAD_C) ? b.buf("act.qc", Ta, d.head == VLA_HEAD_A ? nq : da, 2) : -1;
@@ -740,32 +805,12 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
       b.rmsnorm(NN("n1"), b.all(z), a.n1, b.all(hz), mod1);
       bool cross_only = d.head == VLA_HEAD_C && (i % 2 == 1);
       if (!cross_only) {
-        if (aqkv32 >= 0) {
-          Builder::GemmOpt gq; gq.out32 = b.all(aqkv32);
-          b.gemm(NN("qkv"), b.all(hz), a.wqkv, a_nqkv, gq);
-          NodeDesc n;
-          std::memset(&n, 0, sizeof n);
-          n.op = OP_ROPE;
-          RopeArgs& r = n.u.rope;
-          r.in = b.ref(b.all(aqkv32)); r.out = b.ref(b.all(aqkv));
-          r.M = Ta; r.ld = a_nqkv; r.n_rot_heads = d.hq + d.hkv; r.n_heads = d.hq + 2 * d.hkv; r.hd = d.hd; r.pos0 = S;
-          r.rows_per_tile = 4;
-          n.n_tiles = (Ta + 3) / 4;
-          int id = b.add(n, NN("rope"), KIND_ELEM);
-          b.read(id, b.all(aqkv32));
-          b.write(id, b.all(aqkv));
-        } else {
-          Builder::GemmOpt gq; gq.out16 = b.all(aqkv);
-          b.gemm(NN("qkv"), b.all(hz), a.wqkv, a_nqkv, gq);
-        }
+        b.qkv_project(NN(""), b.all(hz), a.wqkv, aq, ahd, aqkv32, S);
         View att_out = b.rows(aatt, 0, Ta);
-        if (d.head == VLA_HEAD_B) {
-          b.attention(NN("attn"), b.rows(aqkv, 0, Ta, 0), b.rows(qkv[i], 0, S, nq), b.rows(qkv[i], 0, S, nq + nkv), S,
-                      b.rows(aqkv, 0, Ta, a_nq), b.rows(aqkv, 0, Ta, a_nq + a_nkv), Ta, att_out, d.hq, d.hkv, d.hd, false);
-        } else {
-          b.attention(NN("attn"), b.rows(aqkv, 0, Ta, 0), b.rows(aqkv, 0, Ta, a_nq), b.rows(aqkv, 0, Ta, a_nq + a_nkv), Ta,
-                      View(), View(), 0, att_out, d.act_heads, d.act_heads, ahd, false);
-        }
+        if (d.head == VLA_HEAD_B)
+          b.attention(NN("attn"), b.rows(aq.qk, 0, Ta, 0), Ta, lq[i], &aq, att_out, d.hq, d.hkv, d.hd, lhs, false);
+        else
+          b.attention(NN("attn"), b.rows(aq.qk, 0, Ta, 0), Ta, aq, nullptr, att_out, d.act_heads, d.act_heads, ahd, ahs, false);
         Builder::GemmOpt go; go.X = b.all(z); go.out32 = b.all(z);
         b.gemm(NN("wo"), b.all(aatt), a.wo, da, go);
       }
@@ -773,17 +818,14 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
         b.rmsnorm(NN("n2"), b.all(z), a.n2, b.all(hz));
         Builder::GemmOpt gq; gq.out16 = b.all(aqc);
         b.gemm(NN("cq"), b.all(hz), a.cq, nq, gq);
-        int kvb = qkv[d.llm_layers - 1];
-        b.attention(NN("xattn"), b.all(aqc), b.rows(kvb, 0, S, nq), b.rows(kvb, 0, S, nq + nkv), S, View(), View(), 0,
-                    b.all(aatt), d.hq, d.hkv, d.hd, false);
+        b.attention(NN("xattn"), b.all(aqc), Ta, lq[d.llm_layers - 1], nullptr, b.all(aatt), d.hq, d.hkv, d.hd, lhs, false);
         Builder::GemmOpt go; go.X = b.all(z); go.out32 = b.all(z);
         b.gemm(NN("co"), b.all(aatt), a.co, da, go);
         b.rmsnorm(NN("n3"), b.all(z), a.n3, b.all(hz));
       } else if (cross_only) {
         Builder::GemmOpt gq; gq.out16 = b.all(aqc);
         b.gemm(NN("cq"), b.all(hz), a.cq, da, gq);
-        b.attention(NN("xattn"), b.all(aqc), b.rows(ckv[i], 0, S, 0), b.rows(ckv[i], 0, S, da), S, View(), View(), 0,
-                    b.all(aatt), d.act_heads, d.act_heads, ahd, false);
+        b.attention(NN("xattn"), b.all(aqc), Ta, ckv[i], nullptr, b.all(aatt), d.act_heads, d.act_heads, ahd, ahs, false);
         Builder::GemmOpt go; go.X = b.all(z); go.out32 = b.all(z);
         b.gemm(NN("co"), b.all(aatt), a.co, da, go);
         b.rmsnorm(NN("n2"), b.all(z), a.n2, b.all(hz), mod2);
@@ -877,7 +919,7 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   };
   p.off_weights = Builder::WEIGHT_BASE;
   p.off_consts = b.const_base;
-  p.zero_bytes_begin = b.const_base;
+  p.zero_bytes_begin = 0;   // the whole arena starts zeroed: weight padding rows and columns rely on it
   p.off_nodes = place(sizeof(NodeDesc) * p.nodes.size());
   p.off_init_nodes = place(sizeof(NodeDesc) * p.init_program.size());
   p.off_succ = place(sizeof(int32_t) * std::max<size_t>(p.succ.size(), 1));

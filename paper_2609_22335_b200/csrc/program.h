@@ -16,6 +16,8 @@ struct SourceTensor {
   int64_t rows, cols;       // cols == 0: a vector of `rows` elements
   int dev;                  // index into Program::dev_tensors
   int64_t row_offset;       // first row inside the device tensor
+  int64_t group_rows = 0;   // > 0: rows arrive in groups of group_rows (one head) placed group_stride rows apart
+  int64_t group_stride = 0;
   bool loaded = false;
 };
 

@@ -1,6 +1,7 @@
 // Tile bodies other than the GEMM (see gemm_tc.cuh): RMSNorm, fused attention, and the
 // elementwise / gather tiles, plus the dispatch switch.
 #pragma once
+#include "attn_tc.cuh"
 #include "gemm_tc.cuh"
 #include "tiles_common.cuh"
 
@@ -30,65 +31,6 @@ __device__ void tile_rmsnorm(const TileCtx& c, const NormArgs& a, int tile) {
     float v = ld_act(x + i) * inv * g[i];
     if (mod) v = v * (1.0f + mod[i]) + mod[a.d + i];
     o[i] = f32_to_bf16_bits(v);
-  }
-}
-
-// ------------------------------------------------------------------ attention tile
-// One tile = one query head x bq queries; each warp walks its queries one at a time:
-// scores for all keys (lanes over keys), softmax in fp32, then P.V (lanes over head dims).
-__device__ void tile_attention(const TileCtx& c, const AttnArgs& a, int tile) {
-  const int warp = c.tid >> 5, lane = c.tid & 31;
-  const int head = tile / a.q_blocks, qb = tile % a.q_blocks;
-  const int g = (head * a.hkv) / a.hq;
-  const int tkv = a.t0 + a.t1;
-  const unsigned short* Q = resolve<const unsigned short>(c, a.q);
-  const unsigned short* K0 = resolve<const unsigned short>(c, a.k0);
-  const unsigned short* V0 = resolve<const unsigned short>(c, a.v0);
-  const unsigned short* K1 = resolve<const unsigned short>(c, a.k1);
-  const unsigned short* V1 = resolve<const unsigned short>(c, a.v1);
-  unsigned short* O = resolve<unsigned short>(c, a.out);
-  float* qv = reinterpret_cast<float*>(c.smem) + warp * (a.hd + tkv);
-  float* sc = qv + a.hd;
-  const int per_warp = a.bq / 4;
-  for (int qi = 0; qi < per_warp; ++qi) {
-    const int q = qb * a.bq + warp * per_warp + qi;
-    if (q >= a.tq) break;
-    __syncwarp();
-    for (int i = lane; i < a.hd; i += 32) qv[i] = bf16_bits_to_f32(ld_act(Q + (size_t)q * a.ldq + head * a.hd + i));
-    __syncwarp();
-    const int nk = a.causal ? (q + 1) : tkv;
-    float mx = -INFINITY;
-    for (int j = lane; j < nk; j += 32) {
-      const unsigned short* kr = j < a.t0 ? (K0 + (size_t)j * a.ldk0 + g * a.hd) : (K1 + (size_t)(j - a.t0) * a.ldk1 + g * a.hd);
-      float s = 0.f;
-      for (int d0 = 0; d0 < a.hd; d0 += 8) {
-        float k8[8];
-        unpack8(ld_act(reinterpret_cast<const uint4*>(kr + d0)), k8);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) s = fmaf(qv[d0 + i], k8[i], s);
-      }
-      s *= a.scale;
-      sc[j] = s;
-      mx = fmaxf(mx, s);
-    }
-    mx = warp_max(mx);
-    float sum = 0.f;
-    for (int j = lane; j < nk; j += 32) {
-      float p = expf(sc[j] - mx);
-      sc[j] = p;
-      sum += p;
-    }
-    sum = warp_sum(sum);
-    __syncwarp();
-    const float inv = 1.0f / sum;
-    for (int d0 = lane; d0 < a.hd; d0 += 32) {
-      float o = 0.f;
-      for (int j = 0; j < nk; ++j) {
-        const unsigned short* vr = j < a.t0 ? (V0 + (size_t)j * a.ldk0 + g * a.hd) : (V1 + (size_t)(j - a.t0) * a.ldk1 + g * a.hd);
-        o = fmaf(sc[j], bf16_bits_to_f32(ld_act(vr + d0)), o);
-      }
-      O[(size_t)q * a.ldo + head * a.hd + d0] = f32_to_bf16_bits(o * inv);
-    }
   }
 }
 
@@ -128,7 +70,8 @@ __device__ void tile_rope(const TileCtx& c, const RopeArgs& a, int tile) {
   const int r = tile * a.rows_per_tile + warp;
   if (warp >= a.rows_per_tile || r >= a.M) return;
   const float* in = resolve<const float>(c, a.in) + (size_t)r * a.ld;
-  unsigned short* out = resolve<unsigned short>(c, a.out) + (size_t)r * a.ld;
+  unsigned short* out = resolve<unsigned short>(c, a.out) + (size_t)r * a.ldo;
+  unsigned short* outT = resolve<unsigned short>(c, a.outT);
   const int half = a.hd / 2;
   const float pos = (float)(a.pos0 + r);
   const float lnb = 9.210340371976184f;   // ln(10000)
@@ -142,7 +85,8 @@ __device__ void tile_rope(const TileCtx& c, const RopeArgs& a, int tile) {
       out[hh * a.hd + half + i] = f32_to_bf16_bits(x2 * cs + x1 * sn);
     }
   }
-  for (int e = a.n_rot_heads * a.hd + lane; e < a.n_heads * a.hd; e += 32) out[e] = f32_to_bf16_bits(ld_act(in + e));
+  const int v0 = a.n_rot_heads * a.hd;
+  for (int e = v0 + lane; e < a.n_heads * a.hd; e += 32) outT[(size_t)(e - v0) * a.ldoT + r] = f32_to_bf16_bits(ld_act(in + e));
 }
 
 __device__ void tile_addrows(const TileCtx& c, const AddRowsArgs& a, int) {

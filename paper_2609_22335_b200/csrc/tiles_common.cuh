@@ -75,13 +75,14 @@ __device__ __forceinline__ float warp_max(float v) {
 // ------------------------------------------------------------------ GEMM epilogue (one output element)
 struct GemmPtrs {
   const float* X; const float* vec; const float* tab; const float* tab2;
-  float* out32; unsigned short* out16;
+  float* out32; unsigned short* out16; unsigned short* outT;
 };
 __device__ __forceinline__ GemmPtrs gemm_ptrs(const TileCtx& c, const GemmArgs& g) {
   GemmPtrs p;
   p.X = resolve<const float>(c, g.X); p.vec = resolve<const float>(c, g.vec);
   p.tab = resolve<const float>(c, g.tab); p.tab2 = resolve<const float>(c, g.tab2);
   p.out32 = resolve<float>(c, g.out32); p.out16 = resolve<unsigned short>(c, g.out16);
+  p.outT = resolve<unsigned short>(c, g.outT);
   return p;
 }
 // out[r][f] = c_x X[r][f] + c_acc * (act(acc) [* acc2]) + vec[f] + tab[r][f] + tab2[r][f]
@@ -94,7 +95,8 @@ __device__ __forceinline__ void gemm_store(const GemmArgs& g, const GemmPtrs& p,
   if (p.tab) v += p.tab[(size_t)r * g.ldtab + f];
   if (p.tab2) v += p.tab2[(size_t)r * g.ldtab2 + f];
   if (p.out32) p.out32[(size_t)r * g.ldo32 + f] = v;
-  if (p.out16) p.out16[(size_t)r * g.ldo16 + f] = f32_to_bf16_bits(v);
+  if (p.outT && f >= g.t_col0) p.outT[(size_t)(f - g.t_col0) * g.ldoT + r] = f32_to_bf16_bits(v);
+  else if (p.out16) p.out16[(size_t)r * g.ldo16 + f] = f32_to_bf16_bits(v);
 }
 
 }  // namespace vla

@@ -436,9 +436,15 @@ int vla_load_weights(vla_ctx* c, const vla_tensor* tensors, size_t n, int32_t fi
       } else if (t.dtype != 1) {
         return fail(c, VLA_ERR_INVALID, "tensor '%s': unknown dtype", t.name);
       }
-      // padding columns [cols, ld) must be zero: clear the rows first when padded
-      if (dt.ld != s.cols) CU(cudaMemset(dst, 0, (size_t)s.rows * dt.ld * 2));
-      CU(cudaMemcpy2D(dst, (size_t)dt.ld * 2, src, (size_t)s.cols * 2, (size_t)s.cols * 2, (size_t)s.rows, cudaMemcpyHostToDevice));
+      // padding columns [cols, ld) and padding rows between heads stay zero (the arena was cleared at init)
+      if (s.group_rows > 0) {
+        for (int64_t g0 = 0, gi = 0; g0 < s.rows; g0 += s.group_rows, ++gi)
+          CU(cudaMemcpy2D(dst + (size_t)gi * s.group_stride * dt.ld * 2, (size_t)dt.ld * 2,
+                          static_cast<const char*>(src) + (size_t)g0 * s.cols * 2, (size_t)s.cols * 2, (size_t)s.cols * 2,
+                          (size_t)s.group_rows, cudaMemcpyHostToDevice));
+      } else {
+        CU(cudaMemcpy2D(dst, (size_t)dt.ld * 2, src, (size_t)s.cols * 2, (size_t)s.cols * 2, (size_t)s.rows, cudaMemcpyHostToDevice));
+      }
     }
     s.loaded = true;
   }

@@ -41,7 +41,8 @@ struct GemmArgs {
   Ref vec;             // optional fp32 [N], broadcast over rows
   Ref tab, tab2;       // optional fp32 tables [M,ldtab] added row by row
   Ref out32, out16;    // fp32 and/or bf16 outputs [M,ld]
-  int32_t lda, ldx, ldtab, ldtab2, ldo32, ldo16;
+  Ref outT;            // optional transposed bf16 output: features >= t_col0 go to outT[f - t_col0][token]
+  int32_t lda, ldx, ldtab, ldtab2, ldo32, ldo16, ldoT, t_col0;
   int32_t M, N, Kp;    // tokens, output features, padded reduction length (multiple of GEMM_BK)
   int32_t bt, tiles_t; // tokens per tile, number of token tiles
   int32_t act, dual;   // activation; dual: out = act(A W^T) * (A W2^T)
@@ -58,13 +59,14 @@ struct NormArgs {
 };
 
 struct AttnArgs {
-  Ref q, k0, v0, k1, v1, out;  // bf16; segment 0 then segment 1 along the key axis
-  int32_t ldq, ldk0, ldk1, ldo;
-  int32_t tq, t0, t1;
-  int32_t hq, hkv, hd;
+  Ref out;                     // bf16 [tq, ldo], head h at columns h*hd
+  int32_t qmap, k0map, v0map, k1map, v1map;   // activation tensor maps: Q and K [tokens, heads*hs], V^T [heads*hs, tokens]
+  int32_t ldo;
+  int32_t tq, t0, t1;          // queries; keys of segment 0 and segment 1
+  int32_t hq, hkv, hd, hs;     // hs = head stride (hd padded to a multiple of 16)
   int32_t causal;
-  int32_t bq, q_blocks;        // queries per tile
-  float scale;
+  int32_t bn, q_blocks;        // keys per block; 128-query blocks
+  float scale_log2e;           // log2(e) / sqrt(hd)
 };
 
 struct PatchArgs {
@@ -78,8 +80,8 @@ struct EmbedArgs {
 };
 
 struct RopeArgs {
-  Ref in, out;         // in fp32 [M,ld]; out bf16 [M,ld]
-  int32_t M, ld, n_rot_heads, n_heads, hd, pos0, rows_per_tile;
+  Ref in, out, outT;   // in fp32 [M,ld]; out bf16 [M,ldo] (rotated q and k heads); outT bf16 [v features, ldoT] = V^T
+  int32_t M, ld, ldo, ldoT, n_rot_heads, n_heads, hd, pos0, rows_per_tile;
 };
 
 struct AddRowsArgs {

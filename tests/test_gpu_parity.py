@@ -143,9 +143,12 @@ def test_stage_localisation_cfg1():
         assert np.max(np.abs(hidden - vlm["hidden"])) < 5e-2
         assert np.linalg.norm(hidden - vlm["hidden"]) / np.linalg.norm(vlm["hidden"]) < 1e-2
         nq, nkv = m.hq * m.hd, m.hkv * m.hd
-        qkv = eng.debug_fetch(0, 0, f"llm.qkv.{m.llm_layers - 1}").reshape(m.prefix_len, nq + 2 * nkv)
+        qk = eng.debug_fetch(0, 0, f"llm.qkv.{m.llm_layers - 1}.qk").reshape(m.prefix_len, nq + nkv)
         k_ref = vlm["kv"][-1][0].reshape(m.prefix_len, nkv)
-        assert np.linalg.norm(qkv[:, nq:nq + nkv] - k_ref) / np.linalg.norm(k_ref) < 1e-2
+        assert np.linalg.norm(qk[:, nq:] - k_ref) / np.linalg.norm(k_ref) < 1e-2
+        vt = eng.debug_fetch(0, 0, f"llm.qkv.{m.llm_layers - 1}.vt").reshape(nkv, -1)[:, :m.prefix_len]
+        v_ref = vlm["kv"][-1][1].reshape(m.prefix_len, nkv)
+        assert np.linalg.norm(vt.T - v_ref) / np.linalg.norm(v_ref) < 1e-2
         ct = eng.debug_fetch(0, 0, "const.ct").reshape(m.n_steps, m.act_d)
         for k in range(m.n_steps):
             ref = O.time_condition(m, w, 1000.0 * k / m.n_steps, np.float64)
