@@ -248,6 +248,9 @@ class Engine:
         """frames[r][n] -> chunks[r][n]; submits as fast as the rings accept and polls in frame order."""
         import time
         R = len(frames)
+        if not hasattr(self, "_frames_done"):
+            self._frames_done = [0] * self.n_streams
+        base = list(self._frames_done)
         nxt = [0] * R
         got = [[None] * len(frames[r]) for r in range(R)]
         remaining = sum(len(f) for f in frames)
@@ -266,7 +269,8 @@ class Engine:
                     if res is None:
                         break
                     chunk, fid = res
-                    got[r][fid] = chunk
+                    got[r][fid - base[r]] = chunk
+                    self._frames_done[r] += 1
                     remaining -= 1
                     progressed = True
             if not progressed:

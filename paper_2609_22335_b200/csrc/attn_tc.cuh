@@ -93,7 +93,8 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a, int tile) {
     for (int kv0 = 0; kv0 < L && ok; kv0 += bn, ++blk) {
       if (a.causal && kv0 > q0 + ATTN_BQ - 1) break;    // whole block above the diagonal
       const uint32_t ph = (uint32_t)blk & 1u;
-      if (c.tid == 0) {
+      if (warp == 0) {           // lanes 1..31 park at the __syncwarp below instead of spinning beside the issuing lane
+      if (lane == 0) {
         // K and V^T of this block (single-buffered: the previous block's MMAs have completed)
         mbar_expect_tx(bar_k, (uint32_t)nbox * (uint32_t)(bn * 128));
         for (int b = 0; b < nbox; ++b) tma_load_2d(Ks + (uint32_t)b * (uint32_t)(bn * 128), map_ptr(kmap), bar_k, g * hs + b * 64, kv0);
@@ -109,6 +110,8 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a, int tile) {
           }
           umma_commit(bar_s);
         }
+      }
+      __syncwarp();
       }
       // ---- softmax of this block, one thread per query row
       ok = worker_all(c, mbar_wait(c, bar_s, ph));
@@ -162,7 +165,8 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a, int tile) {
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P written by generic stores, read by the MMA
       tc_fence_before();
       worker_sync(c);
-      if (c.tid == 0) {
+      if (warp == 0) {
+      if (lane == 0) {
         ok = mbar_wait(c, bar_v, ph);
         if (ok) {
           tc_fence_after();
@@ -174,6 +178,8 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a, int tile) {
           umma_commit(bar_o);
           ok = mbar_wait(c, bar_o, ph);     // K, V^T and P buffers are free again
         }
+      }
+      __syncwarp();
       }
     }
   }

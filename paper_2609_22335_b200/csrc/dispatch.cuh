@@ -8,7 +8,7 @@ namespace vla {
 
 constexpr unsigned CTRL_EXITING = 0x80000000u;
 constexpr int MAX_WORKERS = 4;
-constexpr int SM_STATE_BYTES = 1024;
+constexpr int SM_STATE_BYTES = 2048;
 
 __device__ __forceinline__ uint64_t gtimer() {
   uint64_t t;
@@ -52,28 +52,40 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
 }
 
 // ------------------------------------------------------------------ tile queues
-// Push n tiles of (inst, node) to the class queue.  Called by one thread.
-__device__ inline void queue_push(const DeviceCtx& ctx, int cls, uint32_t inst, uint32_t node, int n) {
+// Pushing tiles is split in three so a whole worker can fill the entries in parallel:
+// reserve (one thread), fill (any threads, entry i of the range), commit (one thread, after a barrier).
+__device__ inline unsigned long long queue_reserve(const DeviceCtx& ctx, int cls, int n) {
   TileQueue* q = ctx.queues + cls;
   const unsigned long long base = atomicAdd(&q->tail, (unsigned long long)n);
   const unsigned long long head = ld_volatile_u64(&q->head);
-  if (base + n - head > (unsigned long long)ctx.q_capacity) {
-    set_error(ctx, DEV_ERR_QUEUE_FULL, cls);
-    return;
-  }
+  if (base + n - head > (unsigned long long)ctx.q_capacity) set_error(ctx, DEV_ERR_QUEUE_FULL, cls);
+  return base;
+}
+__device__ inline void queue_fill(const DeviceCtx& ctx, int cls, unsigned long long base, uint32_t inst, uint32_t node, int first,
+                                  int count, int stride) {
   const unsigned long long mask = (unsigned long long)ctx.q_capacity - 1;
   QueueEntry* ent = ctx.q_entries + (size_t)cls * ctx.q_capacity;
   unsigned long long* seq = ctx.q_seq + (size_t)cls * ctx.q_capacity;
-  for (int i = 0; i < n; ++i) {
-    unsigned long long t = base + i;
+  for (int i = first; i < count; i += stride) {
     QueueEntry e;
     e.inst_node = (inst << 20) | node;
     e.tile = (uint32_t)i;
-    ent[t & mask] = e;
-    st_release_u64(seq + (t & mask), t + 1);
+    ent[(base + i) & mask] = e;
   }
+  __threadfence();   // entries before their sequence words
+  for (int i = first; i < count; i += stride)
+    *reinterpret_cast<volatile unsigned long long*>(seq + ((base + i) & mask)) = base + i + 1;
+}
+__device__ inline void queue_commit(const DeviceCtx& ctx, int cls, int n) {
   __threadfence();
-  atomicAdd(reinterpret_cast<unsigned long long*>(&q->avail), (unsigned long long)n);
+  atomicAdd(reinterpret_cast<unsigned long long*>(&ctx.queues[cls].avail), (unsigned long long)n);
+  atomicAdd(&ctx.control->doorbell, 1ull);
+}
+// One thread pushes everything (admission of a frame's root tiles).
+__device__ inline void queue_push(const DeviceCtx& ctx, int cls, uint32_t inst, uint32_t node, int n) {
+  const unsigned long long base = queue_reserve(ctx, cls, n);
+  queue_fill(ctx, cls, base, inst, node, 0, n, 1);
+  queue_commit(ctx, cls, n);
 }
 
 // Claim one tile if any is committed.  Bounded wait for the claimed ticket's entry to land.
@@ -99,11 +111,19 @@ __device__ inline bool queue_try_pop(const DeviceCtx& ctx, int cls, QueueEntry& 
 }
 
 // ------------------------------------------------------------------ per-SM state of the persistent kernel
+constexpr int MAX_READY = 6;
+struct ReadyItem {
+  unsigned long long base;   // reserved queue range
+  uint32_t node;
+  int n_tiles, cls;
+};
 struct WorkerCmd {
   int kind;            // 0 run, 1 exit
   uint32_t inst, node, tile;
   int cls;
   int smem_unit0, smem_units, tmem_unit0, tmem_units;
+  int n_ready;         // successors released by the tile just finished (filled by the leader)
+  ReadyItem ready[MAX_READY];
 };
 
 struct SmState {
@@ -126,9 +146,12 @@ __device__ __forceinline__ int find_free(unsigned mask, int need, int total) {
   return -1;
 }
 
-// Tile finished: bump the node's counter; the last tile releases the successors.
-__device__ inline void complete_tile(const DeviceCtx& ctx, uint32_t inst, uint32_t node_idx, bool persistent) {
+// Tile finished: bump the node's counter; the last tile of a node releases its successors.
+// Released successors get their queue range reserved here and are returned in `cmd->ready`
+// (the whole worker then fills the entries); without `cmd` they are pushed on the spot.
+__device__ inline void complete_tile(const DeviceCtx& ctx, uint32_t inst, uint32_t node_idx, bool persistent, WorkerCmd* cmd) {
   const NodeDesc& n = ctx.nodes[node_idx];
+  if (cmd) cmd->n_ready = 0;
   __threadfence();
   int* cnt = ctx.tiles_done + (size_t)inst * ctx.n_nodes + node_idx;
   int done = atomicAdd(cnt, 1) + 1;
@@ -142,8 +165,13 @@ __device__ inline void complete_tile(const DeviceCtx& ctx, uint32_t inst, uint32
     if (left == 0) {
       const NodeDesc& sn = ctx.nodes[s];
       *dep = sn.n_pred;
-      __threadfence();
-      queue_push(ctx, sn.cls, inst, (uint32_t)s, sn.n_tiles);
+      if (cmd && cmd->n_ready < MAX_READY) {
+        ReadyItem& it = cmd->ready[cmd->n_ready++];
+        it.base = queue_reserve(ctx, sn.cls, sn.n_tiles);
+        it.node = (uint32_t)s; it.n_tiles = sn.n_tiles; it.cls = sn.cls;
+      } else {
+        queue_push(ctx, sn.cls, inst, (uint32_t)s, sn.n_tiles);
+      }
     }
   }
   if (persistent && n.op == OP_EMIT) atomicSub(&ctx.control->ctrl, 1u);
@@ -289,35 +317,45 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_ke
       WorkerCmd& cmd = sm->cur[worker];
       const uint64_t wait_start = gtimer();
       uint64_t idle_start = 0;
-      unsigned backoff = 32;
+      unsigned backoff = 64, polls = 0;
+      unsigned long long bell_seen = ~0ull;
       cmd.kind = 1;
       for (;;) {
-        if (ld_volatile_u32(&ctl->error) != 0u || ld_volatile_u32(&ctl->stop) != 0u) break;
-        if (ld_volatile_u32(&ctl->ctrl) & CTRL_EXITING) break;
-        try_admit(ctx);
-        if (try_pick(ctx, sm, worker, wait_start + ctx.wait_limit_ns)) break;   // cmd.kind = 0 now
-        const uint64_t now = gtimer();
-        const unsigned cw = ld_volatile_u32(&ctl->ctrl);
-        if (cw & CTRL_EXITING) break;
-        const bool none = cw == 0u && ld_volatile_u64(&ctl->admit_head) >= ld_volatile_u64(&ctl->admit_tail);
-        if (none) {
-          if (idle_start == 0) idle_start = now;
-          else if (now - idle_start > ctx.idle_exit_ns) atomicCAS(&ctl->ctrl, 0u, CTRL_EXITING);
-        } else {
-          idle_start = 0;
-          if (now - wait_start > ctx.wait_limit_ns) {   // frames in flight but nothing runnable for too long
-            set_error(ctx, DEV_ERR_IDLE_LIMIT, (unsigned)blockIdx.x);
-            break;
+        // An idle leader polls one word (the doorbell); the queues are scanned only when it moved.
+        const unsigned long long bell = ld_volatile_u64(&ctl->doorbell);
+        const bool slow = (polls++ & 15u) == 0;
+        if (slow) {
+          if (ld_volatile_u32(&ctl->error) != 0u || ld_volatile_u32(&ctl->stop) != 0u) break;
+          if (ld_volatile_u32(&ctl->ctrl) & CTRL_EXITING) break;
+          try_admit(ctx);
+        }
+        if (bell != bell_seen || slow) {
+          bell_seen = bell;
+          if (try_pick(ctx, sm, worker, wait_start + ctx.wait_limit_ns)) break;   // cmd.kind = 0 now
+        }
+        if (slow) {
+          const uint64_t now = gtimer();
+          const unsigned cw = ld_volatile_u32(&ctl->ctrl);
+          if (cw & CTRL_EXITING) break;
+          const bool none = cw == 0u && ld_volatile_u64(&ctl->admit_head) >= ld_volatile_u64(&ctl->admit_tail);
+          if (none) {
+            if (idle_start == 0) idle_start = now;
+            else if (now - idle_start > ctx.idle_exit_ns) atomicCAS(&ctl->ctrl, 0u, CTRL_EXITING);
+          } else {
+            idle_start = 0;
+            if (now - wait_start > ctx.wait_limit_ns) {   // frames in flight but nothing runnable for too long
+              set_error(ctx, DEV_ERR_IDLE_LIMIT, (unsigned)blockIdx.x);
+              break;
+            }
           }
         }
         __nanosleep(backoff);
-        if (backoff < 1024) backoff <<= 1;
+        if (backoff < 2048) backoff <<= 1;
       }
     }
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
     const WorkerCmd cmd = sm->cur[worker];
     if (cmd.kind != 0) break;
-    __threadfence();   // acquire side: tile inputs were released by other SMs
     const NodeDesc& n = ctx.nodes[cmd.node];
     TileCtx tc;
     tc.arena = ctx.arena;
@@ -328,6 +366,8 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_ke
     tc.bar_id = bar_id;
     tc.error = &ctl->error;
     tc.tmaps = ctx.tmaps;
+    tc.dbg = ctl->dbg;
+    tc.inputs = ctx.input_ptrs + (size_t)cmd.inst * N_FRAME_INPUTS;
     tc.amap_base = ctx.n_weight_tmaps + (int)cmd.inst * ctx.n_act_tmaps;
     const uint64_t t0 = gtimer();
     tc.deadline = t0 + ctx.wait_limit_ns;
@@ -339,7 +379,18 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_ke
       const uint64_t t1 = gtimer();
       write_trace(ctx, cmd.inst, cmd.node, cmd.tile, worker, cmd.cls, frame, t0, t1);
       release_resources(ctx, sm, cmd);
-      complete_tile(ctx, cmd.inst, cmd.node, true);
+      complete_tile(ctx, cmd.inst, cmd.node, true, &sm->cur[worker]);
+    }
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
+    const int n_ready = sm->cur[worker].n_ready;
+    if (n_ready > 0) {
+      for (int i = 0; i < n_ready; ++i) {
+        const ReadyItem it = sm->cur[worker].ready[i];
+        queue_fill(ctx, it.cls, it.base, cmd.inst, it.node, wt, it.n_tiles, WORKER_THREADS);
+      }
+      asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
+      if (wt == 0)
+        for (int i = 0; i < n_ready; ++i) queue_commit(ctx, sm->cur[worker].ready[i].cls, sm->cur[worker].ready[i].n_tiles);
     }
   }
   tc_fence_before();
@@ -371,6 +422,8 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_node_kernel(DeviceCtx ctx,
   tc.bar_id = 1;
   tc.error = &ctx.control->error;
   tc.tmaps = ctx.tmaps;
+  tc.dbg = ctx.control->dbg;
+  tc.inputs = ctx.input_ptrs + (size_t)(inst >= 0 ? inst : 0) * N_FRAME_INPUTS;
   tc.amap_base = ctx.n_weight_tmaps + (inst >= 0 ? inst : 0) * ctx.n_act_tmaps;
   const uint64_t t0 = gtimer();
   tc.deadline = t0 + ctx.wait_limit_ns;

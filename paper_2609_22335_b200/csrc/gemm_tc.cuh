@@ -135,7 +135,13 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   worker_sync(c);
 
   const uint32_t tmem_d = c.tmem;                 // accumulator columns [0, bt) (and [bt, 2 bt) when dual)
-  if (warp == 0 && lane == 0) {
+#ifdef VLA_TILE_TIMING
+  uint64_t tt0; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt0));
+#endif
+  // Whole warps take a role: lanes 1..31 of the producer and MMA warps park at __syncwarp (they must not
+  // spin on a barrier, which would stall the issuing lane of the same warp).
+  if (warp == 0) {
+    if (lane == 0) {
     // ---------------- TMA producer
     asm volatile("fence.proxy.async;" ::: "memory");   // operands were written by generic stores on other SMs
     const char* tm = reinterpret_cast<const char*>(c.tmaps);
@@ -152,7 +158,10 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       if (g.dual) tma_load_2d(dst + GEMM_W_STAGE_BYTES, w2map, full_bar(s), kb * GEMM_BK, f0);
       tma_load_2d(dst + GEMM_W_STAGE_BYTES * (g.dual ? 2 : 1), amap, full_bar(s), kb * GEMM_BK, t0);
     }
-  } else if (warp == 1 && lane == 0) {
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
     // ---------------- MMA issuer
     const uint32_t idesc = umma_idesc_bf16(g.bt);
     bool ok = true;
@@ -161,6 +170,9 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       const uint32_t ph = (uint32_t)(kb / S) & 1u;
       ok = mbar_wait(c, full_bar(s), ph);
       if (!ok) break;
+#ifdef VLA_TILE_TIMING
+      if (kb == 0 && g.M > 512) { uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); atomicAdd(c.dbg + 0, t - tt0); }
+#endif
       tc_fence_after();
       const uint32_t wsm = stage0 + (uint32_t)(s * stage_bytes);
       const uint32_t asm_ = wsm + GEMM_W_STAGE_BYTES * (g.dual ? 2 : 1);
@@ -175,30 +187,45 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       umma_commit(empty_bar(s));        // stage reusable once these MMAs have read it
     }
     if (ok) umma_commit(accum_bar);     // accumulators complete
+    }
+    __syncwarp();
   }
-  __syncwarp();
 
   // ---------------- epilogue: warp w owns TMEM lanes 32w..32w+31 = features f0+32w..
   const bool ready = mbar_wait(c, accum_bar, 0u);
   __syncwarp();
   tc_fence_after();
+#ifdef VLA_TILE_TIMING
+  uint64_t tt1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt1));
+#endif
   if (ready) {
     GemmPtrs ptrs = gemm_ptrs(c, g);
     const int f = f0 + warp * 32 + lane;
+    const bool fok = f < g.N;
+    const float vecf = (ptrs.vec && fok) ? ptrs.vec[f] : 0.f;
     const uint32_t lane_base = tmem_d + ((uint32_t)(warp * 32) << 16);
     for (int c0 = 0; c0 < nt; c0 += 16) {
       float a[16], b[16];
       tmem_ld16(lane_base + (uint32_t)c0, a);
       if (g.dual) tmem_ld16(lane_base + (uint32_t)(g.bt + c0), b);
-      if (f < g.N) {
-#pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (c0 + j < nt) gemm_store(g, ptrs, t0 + c0 + j, f, a[j], g.dual ? b[j] : 0.f);
-      }
+      if (!fok) continue;
+      const int n = min(16, nt - c0), r0 = t0 + c0;
+      if (g.dual) {
+        if (g.act == ACT_SILU) gemm_store16<ACT_SILU, true>(g, ptrs, r0, n, f, vecf, a, b);
+        else gemm_store16<ACT_GELU, true>(g, ptrs, r0, n, f, vecf, a, b);
+      } else if (g.act == ACT_GELU) gemm_store16<ACT_GELU, false>(g, ptrs, r0, n, f, vecf, a, b);
+      else if (g.act == ACT_SILU) gemm_store16<ACT_SILU, false>(g, ptrs, r0, n, f, vecf, a, b);
+      else gemm_store16<ACT_NONE, false>(g, ptrs, r0, n, f, vecf, a, b);
     }
   }
   tc_fence_before();
   worker_sync(c);
+#ifdef VLA_TILE_TIMING
+  if (c.tid == 64 && g.M > 512) {
+    uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    atomicAdd(c.dbg + 1, tt1 - tt0); atomicAdd(c.dbg + 2, t - tt1); atomicAdd(c.dbg + 3, 1ull); atomicAdd(c.dbg + 4, (unsigned long long)nkb);
+  }
+#endif
   if (c.tid == 0) {
     for (int s = 0; s < 2 * S + 1; ++s) mbar_inval(bar0 + 8u * s);
   }

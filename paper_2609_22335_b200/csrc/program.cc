@@ -57,6 +57,7 @@ class Builder {
     acc.emplace_back();
     return (int)p.bufs.size() - 1;
   }
+  static Ref in_ref(int idx, uint64_t byte_off = 0) { return REF_INPUT | ((uint64_t)idx << 56) | byte_off; }
   View all(int b) const { return View{b, 0, p.bufs[b].rows, 0}; }
   View rows(int b, int64_t r0, int64_t n, int64_t c0 = 0) const { return View{b, r0, n, c0}; }
   int64_t ld(const View& v) const { return p.bufs[v.buf].ld; }
@@ -279,7 +280,8 @@ class Builder {
     NormArgs& a = n.u.norm;
     a.x = ref(x); a.g = wref(g_dev); a.mod = mod; a.out = ref(out);
     a.M = (int)x.rows; a.d = (int)p.dev_tensors[g_dev].cols; a.ldx = (int)ld(x); a.ldo = (int)ld(out);
-    a.rows_per_tile = 4; a.shuffle = shuffle; a.grid = grid;
+    a.rows_per_tile = 16; a.shuffle = shuffle; a.grid = grid;
+    if (a.d % 4) p.error = "model widths must be multiples of 4";
     n.n_tiles = (a.M + a.rows_per_tile - 1) / a.rows_per_tile;
     int id = add(n, name, KIND_ELEM);
     read(id, x);
@@ -350,8 +352,8 @@ class Builder {
       r.in = ref(all(scratch32)); r.out = ref(all(dst.qk)); r.outT = ref(all(dst.vt));
       r.M = dst.T; r.ld = (int)nall; r.ldo = (int)nqk; r.ldoT = (int)p.bufs[dst.vt].ld;
       r.n_rot_heads = dst.hq + dst.hkv; r.n_heads = dst.hq + 2 * dst.hkv; r.hd = hd; r.pos0 = pos0;
-      r.rows_per_tile = 4;
-      n.n_tiles = (dst.T + 3) / 4;
+      r.rows_per_tile = 16;
+      n.n_tiles = (dst.T + 15) / 16;
       int id = add(n, name + "rope", KIND_ELEM);
       read(id, all(scratch32));
       write(id, all(dst.qk));
@@ -654,12 +656,11 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
       std::memset(&n, 0, sizeof n);
       n.op = OP_PATCHIFY;
       PatchArgs& a = n.u.patch;
-      a.img = b.ref(b.rows(in_img, c, 1));
+      a.img = Builder::in_ref(0, (uint64_t)c * 3 * d.img * d.img * 4);
       a.out = b.ref(b.all(patches));
-      a.img_side = d.img; a.patch = d.patch; a.grid = grid; a.ldo = (int)P64(patch_k); a.rows_per_tile = 4;
-      n.n_tiles = (T + 3) / 4;
+      a.img_side = d.img; a.patch = d.patch; a.grid = grid; a.ldo = (int)P64(patch_k); a.rows_per_tile = 16;
+      n.n_tiles = (T + 15) / 16;
       int id = b.add(n, N_("vis%d.patchify", c), KIND_ELEM);
-      b.read(id, b.rows(in_img, c, 1));
       b.write(id, b.all(patches));
     }
     if (d.vis_layers == 0 && !d.connector) {
@@ -711,14 +712,13 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     std::memset(&n, 0, sizeof n);
     n.op = OP_EMBED;
     EmbedArgs& a = n.u.embed;
-    a.ids = b.ref(b.all(in_txt));
+    a.ids = Builder::in_ref(1);
     a.table = b.wref(w_emb);
     a.pos = w_lpos >= 0 ? b.wref(w_lpos, n_img) : 0;
     a.out = b.ref(b.rows(x, n_img, d.n_text));
-    a.n = d.n_text; a.d = D; a.ldo = D; a.vocab = d.vocab; a.rows_per_tile = 4; a.ldt = (int)P64(D);
-    n.n_tiles = (d.n_text + 3) / 4;
+    a.n = d.n_text; a.d = D; a.ldo = D; a.vocab = d.vocab; a.rows_per_tile = 16; a.ldt = (int)P64(D);
+    n.n_tiles = (d.n_text + 15) / 16;
     int id = b.add(n, "llm.embed", KIND_ELEM);
-    b.read(id, b.all(in_txt));
     b.write(id, b.rows(x, n_img, d.n_text));
   }
   for (int i = 0; i < d.llm_layers; ++i) {
@@ -770,7 +770,7 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   int state_bf = has_state ? b.buf("act.state_bf", 1, P64(d.state_dim), 2) : -1;
 
   if (has_state) {
-    b.addrows("act.state_cvt", b.all(in_state), 0, 0, 1, d.state_dim, 0, 0, 0, View(), b.all(state_bf));
+    b.addrows("act.state_cvt", View(), Builder::in_ref(2), d.state_dim, 1, d.state_dim, 0, 0, 0, View(), b.all(state_bf));
     Builder::GemmOpt g;
     if (head_pos) { g.tab = b.wref(w_apos, 0); g.ldtab = da; }
     g.out32 = b.all(tok0);
@@ -781,7 +781,7 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     g.out32 = b.all(tok0);
     b.gemm("act.cond_tok", b.rows(hidden, S - 1, 1), w_acond, da, g);
   }
-  b.addrows("act.x_init", b.all(in_noise), 0, 0, d.horizon, d.act_dim, 0, 0, 0, b.all(xs), b.all(xbf));
+  b.addrows("act.x_init", View(), Builder::in_ref(3), d.act_dim, d.horizon, d.act_dim, 0, 0, 0, b.all(xs), b.all(xbf));
 
   for (int k = 0; k < ns; ++k) {
     b.step = k;
@@ -943,6 +943,7 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   p.off_tiles_done = place(sizeof(int32_t) * (uint64_t)nn * p.n_inst);
   p.off_inst_frame = place(sizeof(uint64_t) * p.n_inst);
   p.off_slot_base = place(sizeof(uint64_t) * p.n_inst);
+  p.off_input_ptrs = place(sizeof(uint64_t) * N_FRAME_INPUTS * p.n_inst);
   p.trace_capacity = o.trace_capacity;
   p.off_trace = place(sizeof(TraceRec) * (uint64_t)std::max<uint32_t>(o.trace_capacity, 1));
   p.off_tmaps = place(128ull * (p.wmaps.size() + p.amaps.size() * (size_t)p.n_inst + 1), 128);

@@ -7,86 +7,137 @@
 
 namespace vla {
 
-// ------------------------------------------------------------------ RMSNorm tile (one warp per row)
+// ------------------------------------------------------------------ RMSNorm tile (one warp per row, float4 lanes)
+// Rows up to 2048 wide are read once and held in registers; wider rows take a second pass through L2.
 __device__ void tile_rmsnorm(const TileCtx& c, const NormArgs& a, int tile) {
+  constexpr int MAXV = 16;
   const int warp = c.tid >> 5, lane = c.tid & 31;
-  const int r = tile * a.rows_per_tile + warp;
-  if (warp >= a.rows_per_tile || r >= a.M) return;
-  const float* x = resolve<const float>(c, a.x) + (size_t)r * a.ldx;
-  const float* g = resolve<const float>(c, a.g);
+  const float4* g4 = reinterpret_cast<const float4*>(resolve<const float>(c, a.g));
   const float* mod = resolve<const float>(c, a.mod);
   unsigned short* out = resolve<unsigned short>(c, a.out);
-  float ss = 0.f;
-  for (int i = lane; i < a.d; i += 32) { float v = ld_act(x + i); ss = fmaf(v, v, ss); }
-  ss = warp_sum(ss);
-  const float inv = 1.0f / sqrtf(ss / (float)a.d + 1e-6f);
-  size_t orow = r, ocol0 = 0;
-  if (a.shuffle > 1) {
-    int y = r / a.grid, xx = r % a.grid, s = a.shuffle;
-    orow = (size_t)(y / s) * (a.grid / s) + (xx / s);
-    ocol0 = (size_t)((y % s) * s + (xx % s)) * a.d;
-  }
-  unsigned short* o = out + orow * a.ldo + ocol0;
-  for (int i = lane; i < a.d; i += 32) {
-    float v = ld_act(x + i) * inv * g[i];
-    if (mod) v = v * (1.0f + mod[i]) + mod[a.d + i];
-    o[i] = f32_to_bf16_bits(v);
+  const float* xbase = resolve<const float>(c, a.x);
+  const int d4 = a.d >> 2;                      // widths are multiples of 4
+  const bool in_regs = d4 <= 32 * MAXV;
+  for (int rr = warp; rr < a.rows_per_tile; rr += WORKER_THREADS / 32) {
+    const int r = tile * a.rows_per_tile + rr;
+    if (r >= a.M) break;
+    const float4* x4 = reinterpret_cast<const float4*>(xbase + (size_t)r * a.ldx);
+    float4 v[MAXV];
+    float ss = 0.f;
+    if (in_regs) {
+#pragma unroll
+      for (int k = 0; k < MAXV; ++k) {
+        const int i = lane + 32 * k;
+        v[k] = i < d4 ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int k = 0; k < MAXV; ++k) {
+        ss = fmaf(v[k].x, v[k].x, ss); ss = fmaf(v[k].y, v[k].y, ss); ss = fmaf(v[k].z, v[k].z, ss); ss = fmaf(v[k].w, v[k].w, ss);
+      }
+    } else {
+      for (int i = lane; i < d4; i += 32) {
+        float4 t = __ldcg(x4 + i);
+        ss = fmaf(t.x, t.x, ss); ss = fmaf(t.y, t.y, ss); ss = fmaf(t.z, t.z, ss); ss = fmaf(t.w, t.w, ss);
+      }
+    }
+    ss = warp_sum(ss);
+    const float inv = 1.0f / sqrtf(ss / (float)a.d + 1e-6f);
+    size_t orow = r, ocol0 = 0;
+    if (a.shuffle > 1) {
+      int y = r / a.grid, xx = r % a.grid, s = a.shuffle;
+      orow = (size_t)(y / s) * (a.grid / s) + (xx / s);
+      ocol0 = (size_t)((y % s) * s + (xx % s)) * a.d;
+    }
+    uint2* o2 = reinterpret_cast<uint2*>(out + orow * a.ldo + ocol0);
+    auto emit = [&](int i, float4 t) {
+      float4 gg = g4[i];
+      float y0 = t.x * inv * gg.x, y1 = t.y * inv * gg.y, y2 = t.z * inv * gg.z, y3 = t.w * inv * gg.w;
+      if (mod) {
+        float4 ga = reinterpret_cast<const float4*>(mod)[i], be = reinterpret_cast<const float4*>(mod + a.d)[i];
+        y0 = y0 * (1.0f + ga.x) + be.x; y1 = y1 * (1.0f + ga.y) + be.y;
+        y2 = y2 * (1.0f + ga.z) + be.z; y3 = y3 * (1.0f + ga.w) + be.w;
+      }
+      __nv_bfloat162 lo = __floats2bfloat162_rn(y0, y1), hi = __floats2bfloat162_rn(y2, y3);
+      o2[i] = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+    };
+    if (in_regs) {
+#pragma unroll
+      for (int k = 0; k < MAXV; ++k) {
+        const int i = lane + 32 * k;
+        if (i < d4) emit(i, v[k]);
+      }
+    } else {
+      for (int i = lane; i < d4; i += 32) emit(i, __ldcg(x4 + i));
+    }
   }
 }
 
 // ------------------------------------------------------------------ elementwise tiles
 __device__ void tile_patchify(const TileCtx& c, const PatchArgs& a, int tile) {
   const int warp = c.tid >> 5, lane = c.tid & 31;
-  const int p = tile * a.rows_per_tile + warp;
-  if (warp >= a.rows_per_tile || p >= a.grid * a.grid) return;
   const float* img = resolve<const float>(c, a.img);
-  unsigned short* out = resolve<unsigned short>(c, a.out) + (size_t)p * a.ldo;
-  const int py = p / a.grid, px = p % a.grid, P = a.patch, pk = 3 * P * P;
-  for (int e = lane; e < pk; e += 32) {
-    int ch = e / (P * P), rem = e % (P * P), yy = rem / P, xx = rem % P;
-    float v = ld_act(img + ((size_t)ch * a.img_side + (py * P + yy)) * a.img_side + px * P + xx);
-    out[e] = f32_to_bf16_bits(v);
+  unsigned short* obase = resolve<unsigned short>(c, a.out);
+  const int P = a.patch, pk = 3 * P * P;
+  for (int rr = warp; rr < a.rows_per_tile; rr += WORKER_THREADS / 32) {
+    const int p = tile * a.rows_per_tile + rr;
+    if (p >= a.grid * a.grid) break;
+    unsigned short* out = obase + (size_t)p * a.ldo;
+    const int py = p / a.grid, px = p % a.grid;
+    for (int e = lane; e < pk; e += 32) {
+      int ch = e / (P * P), rem = e % (P * P), yy = rem / P, xx = rem % P;
+      float v = ld_act(img + ((size_t)ch * a.img_side + (py * P + yy)) * a.img_side + px * P + xx);
+      out[e] = f32_to_bf16_bits(v);
+    }
   }
 }
 
 __device__ void tile_embed(const TileCtx& c, const EmbedArgs& a, int tile) {
   const int warp = c.tid >> 5, lane = c.tid & 31;
-  const int r = tile * a.rows_per_tile + warp;
-  if (warp >= a.rows_per_tile || r >= a.n) return;
-  int id = ld_act(resolve<const int>(c, a.ids) + r);
-  id = min(max(id, 0), a.vocab - 1);
-  const unsigned short* row = resolve<const unsigned short>(c, a.table) + (size_t)id * a.ldt;
+  const int* ids = resolve<const int>(c, a.ids);
+  const unsigned short* table = resolve<const unsigned short>(c, a.table);
   const float* pos = resolve<const float>(c, a.pos);
-  float* out = resolve<float>(c, a.out) + (size_t)r * a.ldo;
-  for (int i = lane; i < a.d; i += 32) {
-    float v = bf16_bits_to_f32(row[i]);
-    if (pos) v += pos[(size_t)r * a.d + i];
-    out[i] = v;
+  float* obase = resolve<float>(c, a.out);
+  for (int rr = warp; rr < a.rows_per_tile; rr += WORKER_THREADS / 32) {
+    const int r = tile * a.rows_per_tile + rr;
+    if (r >= a.n) break;
+    int id = ld_act(ids + r);
+    id = min(max(id, 0), a.vocab - 1);
+    const unsigned short* row = table + (size_t)id * a.ldt;
+    float* out = obase + (size_t)r * a.ldo;
+    for (int i = lane; i < a.d; i += 32) {
+      float v = bf16_bits_to_f32(row[i]);
+      if (pos) v += pos[(size_t)r * a.d + i];
+      out[i] = v;
+    }
   }
 }
 
 __device__ void tile_rope(const TileCtx& c, const RopeArgs& a, int tile) {
   const int warp = c.tid >> 5, lane = c.tid & 31;
-  const int r = tile * a.rows_per_tile + warp;
-  if (warp >= a.rows_per_tile || r >= a.M) return;
-  const float* in = resolve<const float>(c, a.in) + (size_t)r * a.ld;
-  unsigned short* out = resolve<unsigned short>(c, a.out) + (size_t)r * a.ldo;
+  const float* ibase = resolve<const float>(c, a.in);
+  unsigned short* obase = resolve<unsigned short>(c, a.out);
   unsigned short* outT = resolve<unsigned short>(c, a.outT);
   const int half = a.hd / 2;
-  const float pos = (float)(a.pos0 + r);
   const float lnb = 9.210340371976184f;   // ln(10000)
-  for (int i = lane; i < half; i += 32) {
-    float inv = expf(-lnb * (2.0f * (float)i) / (float)a.hd);
-    float sn, cs;
-    sincosf(pos * inv, &sn, &cs);
-    for (int hh = 0; hh < a.n_rot_heads; ++hh) {
-      float x1 = ld_act(in + hh * a.hd + i), x2 = ld_act(in + hh * a.hd + half + i);
-      out[hh * a.hd + i] = f32_to_bf16_bits(x1 * cs - x2 * sn);
-      out[hh * a.hd + half + i] = f32_to_bf16_bits(x2 * cs + x1 * sn);
+  for (int rr = warp; rr < a.rows_per_tile; rr += WORKER_THREADS / 32) {
+    const int r = tile * a.rows_per_tile + rr;
+    if (r >= a.M) break;
+    const float* in = ibase + (size_t)r * a.ld;
+    unsigned short* out = obase + (size_t)r * a.ldo;
+    const float pos = (float)(a.pos0 + r);
+    for (int i = lane; i < half; i += 32) {
+      float inv = expf(-lnb * (2.0f * (float)i) / (float)a.hd);
+      float sn, cs;
+      sincosf(pos * inv, &sn, &cs);
+      for (int hh = 0; hh < a.n_rot_heads; ++hh) {
+        float x1 = ld_act(in + hh * a.hd + i), x2 = ld_act(in + hh * a.hd + half + i);
+        out[hh * a.hd + i] = f32_to_bf16_bits(x1 * cs - x2 * sn);
+        out[hh * a.hd + half + i] = f32_to_bf16_bits(x2 * cs + x1 * sn);
+      }
     }
+    const int v0 = a.n_rot_heads * a.hd;
+    for (int e = v0 + lane; e < a.n_heads * a.hd; e += 32) outT[(size_t)(e - v0) * a.ldoT + r] = f32_to_bf16_bits(ld_act(in + e));
   }
-  const int v0 = a.n_rot_heads * a.hd;
-  for (int e = v0 + lane; e < a.n_heads * a.hd; e += 32) outT[(size_t)(e - v0) * a.ldoT + r] = f32_to_bf16_bits(ld_act(in + e));
 }
 
 __device__ void tile_addrows(const TileCtx& c, const AddRowsArgs& a, int) {

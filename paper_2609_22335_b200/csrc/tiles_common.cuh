@@ -21,6 +21,8 @@ struct TileCtx {
   int bar_id;           // named barrier of this worker
   uint64_t deadline;    // %globaltimer value after which bounded waits give up
   unsigned int* error;  // sticky device error word
+  const uint64_t* inputs;  // this frame slot's input pointer table
+  unsigned long long* dbg; // bring-up counters (VLA_TILE_TIMING builds only)
   const void* tmaps;    // tensor-map table (128 bytes per entry)
   int amap_base;        // index of this frame slot's first activation map
 };
@@ -28,6 +30,10 @@ struct TileCtx {
 template <typename T>
 __device__ __forceinline__ T* resolve(const TileCtx& c, Ref r) {
   if (r == 0) return nullptr;
+  if (r & REF_INPUT) {
+    const unsigned long long p = __ldcg(reinterpret_cast<const unsigned long long*>(c.inputs) + ((r >> 56) & 0xF));
+    return reinterpret_cast<T*>(p + (r & ((1ull << 56) - 1)));
+  }
   return reinterpret_cast<T*>(c.arena + (r & ~REF_SLOT) + ((r & REF_SLOT) ? c.slot_base : 0ull));
 }
 
@@ -52,11 +58,22 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
   f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xFFFF0000u);
 }
 
+// Activations use the hardware approximations (tanh.approx, ex2.approx): their error (~2^-11 relative)
+// is below the bf16 rounding of the values they produce.
+__device__ __forceinline__ float tanh_fast(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ float gelu_tanh_f(float x) {
   const float c = 0.7978845608028654f;
-  return 0.5f * x * (1.0f + tanhf(c * (x + 0.044715f * x * x * x)));
+  return 0.5f * x * (1.0f + tanh_fast(c * (x + 0.044715f * x * x * x)));
 }
-__device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x)); }
+__device__ __forceinline__ float silu_f(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
+template <int ACT>
+__device__ __forceinline__ float apply_act_t(float v) {
+  return ACT == ACT_GELU ? gelu_tanh_f(v) : (ACT == ACT_SILU ? silu_f(v) : v);
+}
 __device__ __forceinline__ float apply_act(int act, float v) {
   return act == ACT_GELU ? gelu_tanh_f(v) : (act == ACT_SILU ? silu_f(v) : v);
 }
@@ -85,18 +102,71 @@ __device__ __forceinline__ GemmPtrs gemm_ptrs(const TileCtx& c, const GemmArgs& 
   p.outT = resolve<unsigned short>(c, g.outT);
   return p;
 }
-// out[r][f] = c_x X[r][f] + c_acc * (act(acc) [* acc2]) + vec[f] + tab[r][f] + tab2[r][f]
-__device__ __forceinline__ void gemm_store(const GemmArgs& g, const GemmPtrs& p, int r, int f, float acc, float acc2) {
-  float v = apply_act(g.act, acc);
-  if (g.dual) v *= acc2;
-  v *= g.c_acc;
-  if (p.X) v += g.c_x * ld_act(p.X + (size_t)r * g.ldx + f);
-  if (p.vec) v += p.vec[f];
-  if (p.tab) v += p.tab[(size_t)r * g.ldtab + f];
-  if (p.tab2) v += p.tab2[(size_t)r * g.ldtab2 + f];
-  if (p.out32) p.out32[(size_t)r * g.ldo32 + f] = v;
-  if (p.outT && f >= g.t_col0) p.outT[(size_t)(f - g.t_col0) * g.ldoT + r] = f32_to_bf16_bits(v);
-  else if (p.out16) p.out16[(size_t)r * g.ldo16 + f] = f32_to_bf16_bits(v);
+// Epilogue of one thread's 16 consecutive tokens of one output feature f:
+//   out[r][f] = c_x X[r][f] + c_acc * (act(acc) [* acc2]) + vec[f] + tab[r][f] + tab2[r][f]
+// Loads are issued for all 16 tokens before any arithmetic or store so that they overlap
+// (X and the fp32 output may be the same buffer, which would otherwise serialise them).
+template <int ACT, bool DUAL>
+__device__ __forceinline__ void gemm_store16(const GemmArgs& g, const GemmPtrs& p, int r0, int n, int f, float vecf,
+                                             const float* a, const float* b) {
+  float v[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    float t = apply_act_t<ACT>(a[j]);
+    if (DUAL) t *= b[j];
+    v[j] = t * g.c_acc + vecf;
+  }
+  if (p.X) {
+    const float* xp = p.X + (size_t)r0 * g.ldx + f;
+    float x[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) x[j] = j < n ? __ldcg(xp + (size_t)j * g.ldx) : 0.f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = fmaf(g.c_x, x[j], v[j]);
+  }
+  if (p.tab) {
+    const float* tp = p.tab + (size_t)r0 * g.ldtab + f;
+    float x[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) x[j] = j < n ? tp[(size_t)j * g.ldtab] : 0.f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] += x[j];
+  }
+  if (p.tab2) {
+    const float* tp = p.tab2 + (size_t)r0 * g.ldtab2 + f;
+    float x[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) x[j] = j < n ? tp[(size_t)j * g.ldtab2] : 0.f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] += x[j];
+  }
+  if (p.out32) {
+    float* op = p.out32 + (size_t)r0 * g.ldo32 + f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (j < n) op[(size_t)j * g.ldo32] = v[j];
+  }
+  if (p.outT && f >= g.t_col0) {
+    // transposed output: this thread's 16 tokens are contiguous in row f - t_col0
+    unsigned short* op = p.outT + (size_t)(f - g.t_col0) * g.ldoT + r0;
+    uint32_t pk[8];
+#pragma unroll
+    for (int j = 0; j < 16; j += 2) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(v[j], v[j + 1]);
+      pk[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    if (n == 16) {
+      *reinterpret_cast<uint4*>(op) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      *reinterpret_cast<uint4*>(op + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+    } else {
+      for (int j = 0; j < n; ++j) op[j] = (unsigned short)((j & 1) ? (pk[j >> 1] >> 16) : (pk[j >> 1] & 0xFFFFu));
+    }
+  } else if (p.out16) {
+    unsigned short* op = p.out16 + (size_t)r0 * g.ldo16 + f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (j < n) op[(size_t)j * g.ldo16] = f32_to_bf16_bits(v[j]);
+  }
 }
 
 }  // namespace vla

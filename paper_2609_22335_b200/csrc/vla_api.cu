@@ -8,6 +8,7 @@
 #include <chrono>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <string>
 #include <thread>
@@ -46,6 +47,7 @@ struct vla_ctx {
   AdmitRec* admit_pinned = nullptr; // ring of admission records (source of the device copies)
   unsigned long long* tail_pinned = nullptr;
   unsigned* zero_pinned = nullptr;
+  uint64_t* inptr_pinned = nullptr; // [n_inst][N_FRAME_INPUTS] source of the input pointer table copies
   unsigned long long n_admitted = 0;
   std::vector<InstHost> inst;
   std::vector<uint64_t> next_submit, next_poll;   // per request stream frame counters
@@ -211,11 +213,11 @@ int submit_common(vla_ctx* c, int32_t stream, const float* image, const int32_t*
   if (ih.state != 0) return fail(c, VLA_ERR_BUSY, "frame ring of stream %d is full", stream);
 
   char* slot_dev = c->arena + p.off_slots + (uint64_t)inst * p.slot_bytes;
+  uint64_t* ip = c->inptr_pinned + (size_t)inst * N_FRAME_INPUTS;
   if (device_inputs) {
-    CU(cudaMemcpyAsync(slot_dev + p.in_image, image, p.image_bytes, cudaMemcpyDeviceToDevice, c->scopy));
-    CU(cudaMemcpyAsync(slot_dev + p.in_text, text_ids, p.text_bytes, cudaMemcpyDeviceToDevice, c->scopy));
-    if (d.state_dim > 0) CU(cudaMemcpyAsync(slot_dev + p.in_state, state, p.state_bytes, cudaMemcpyDeviceToDevice, c->scopy));
-    CU(cudaMemcpyAsync(slot_dev + p.in_noise, noise, p.noise_bytes, cudaMemcpyDeviceToDevice, c->scopy));
+    // resident inputs are read in place: only their addresses travel
+    ip[0] = reinterpret_cast<uint64_t>(image); ip[1] = reinterpret_cast<uint64_t>(text_ids);
+    ip[2] = reinterpret_cast<uint64_t>(state); ip[3] = reinterpret_cast<uint64_t>(noise);
   } else {
     char* st = c->staging + (size_t)inst * c->staging_bytes;
     std::memcpy(st + (p.in_image - c->in_lo), image, p.image_bytes);
@@ -223,7 +225,11 @@ int submit_common(vla_ctx* c, int32_t stream, const float* image, const int32_t*
     if (d.state_dim > 0) std::memcpy(st + (p.in_state - c->in_lo), state, p.state_bytes);
     std::memcpy(st + (p.in_noise - c->in_lo), noise, p.noise_bytes);
     CU(cudaMemcpyAsync(slot_dev + c->in_lo, st, c->staging_bytes, cudaMemcpyHostToDevice, c->scopy));
+    ip[0] = reinterpret_cast<uint64_t>(slot_dev + p.in_image); ip[1] = reinterpret_cast<uint64_t>(slot_dev + p.in_text);
+    ip[2] = reinterpret_cast<uint64_t>(slot_dev + p.in_state); ip[3] = reinterpret_cast<uint64_t>(slot_dev + p.in_noise);
   }
+  CU(cudaMemcpyAsync(const_cast<uint64_t*>(c->dctx.input_ptrs) + (size_t)inst * N_FRAME_INPUTS, ip,
+                     sizeof(uint64_t) * N_FRAME_INPUTS, cudaMemcpyHostToDevice, c->scopy));
   ih.state = 1;
   ih.frame = f;
   c->done_host[inst].frame_plus1 = 0;
@@ -343,6 +349,7 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
   *c->error_host = 0;
   CU(cudaHostAlloc(&c->admit_pinned, sizeof(AdmitRec) * p.admit_capacity, cudaHostAllocDefault));
   CU(cudaHostAlloc(&c->tail_pinned, sizeof(unsigned long long) * p.admit_capacity, cudaHostAllocDefault));
+  CU(cudaHostAlloc(&c->inptr_pinned, sizeof(uint64_t) * N_FRAME_INPUTS * p.n_inst, cudaHostAllocDefault));
   CU(cudaHostAlloc(&c->zero_pinned, 64, cudaHostAllocDefault));
   std::memset(c->zero_pinned, 0, 64);
 
@@ -361,6 +368,7 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
   x.tiles_done = at<int32_t>(c, p.off_tiles_done);
   x.inst_frame = at<uint64_t>(c, p.off_inst_frame);
   x.slot_base = at<uint64_t>(c, p.off_slot_base);
+  x.input_ptrs = at<uint64_t>(c, p.off_input_ptrs);
   x.roots = at<int32_t>(c, p.off_roots);
   x.trace = at<TraceRec>(c, p.off_trace);
   void* dp = nullptr;
@@ -594,6 +602,10 @@ int vla_get_counters(vla_ctx* c, uint64_t* tiles, uint64_t* kernel_launches, uin
     Control ctl;
     CU(cudaMemcpy(&ctl, c->dctx.control, sizeof ctl, cudaMemcpyDeviceToHost));
     *tiles = ctl.tiles_done;
+    if (getenv("VLA_PRINT_DBG"))
+      fprintf(stderr, "dbg: first_full %.2f us  mainloop %.2f us  epilogue %.2f us  tiles %llu  kb/tile %.1f\n",
+              ctl.dbg[3] ? ctl.dbg[0] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3] ? ctl.dbg[1] / 1e3 / ctl.dbg[3] : 0.0,
+              ctl.dbg[3] ? ctl.dbg[2] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3], ctl.dbg[3] ? (double)ctl.dbg[4] / ctl.dbg[3] : 0.0);
   }
   if (kernel_launches) *kernel_launches = c->n_kernel_launches;
   if (persistent_launches) *persistent_launches = c->n_persistent_launches;
@@ -661,6 +673,7 @@ int vla_destroy(vla_ctx* c) {
   if (c->admit_pinned) cudaFreeHost(c->admit_pinned);
   if (c->tail_pinned) cudaFreeHost(c->tail_pinned);
   if (c->zero_pinned) cudaFreeHost(c->zero_pinned);
+  if (c->inptr_pinned) cudaFreeHost(c->inptr_pinned);
   delete c;
   return VLA_OK;
 }

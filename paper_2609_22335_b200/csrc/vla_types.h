@@ -28,6 +28,10 @@ enum Act : int32_t { ACT_NONE = 0, ACT_GELU = 1, ACT_SILU = 2 };
 // frame slot (instance) base rather than the arena base.  0 = null.
 typedef uint64_t Ref;
 constexpr Ref REF_SLOT = 1ull << 63;
+// Bit 62: one of the frame's input arrays (index in bits 56..59: 0 image, 1 text ids, 2 state, 3 noise),
+// reached through the per-slot input pointer table so resident inputs are read in place.
+constexpr Ref REF_INPUT = 1ull << 62;
+constexpr int N_FRAME_INPUTS = 4;
 
 constexpr int GEMM_BM = 128;   // output features per GEMM tile (the MMA M dimension)
 constexpr int GEMM_BK = 64;    // K elements per pipeline stage (one 128-byte swizzle row of bf16)
@@ -130,11 +134,11 @@ constexpr int SMEM_UNIT = 8192;
 constexpr int TMEM_UNIT = 32;
 
 // A multi-producer multi-consumer ring of tile tickets (one per class).
-struct TileQueue {
+struct TileQueue {             // one 128-byte line per queue
   unsigned long long head;     // next ticket to hand out
   unsigned long long tail;     // next ticket to reserve for a push
   long long avail;             // committed minus claimed (may dip below zero transiently)
-  unsigned long long pad;
+  unsigned long long pad[13];
 };
 
 struct QueueEntry {            // 8 bytes: one tile
@@ -162,15 +166,20 @@ struct DoneRec {
 };
 
 // Device-resident control block.
-struct Control {
+struct Control {                 // polled words and hot counters live on separate 128-byte lines
   unsigned int ctrl;             // bit 31 = exiting; low bits = frames in flight
   unsigned int error;            // sticky error code (0 = none)
   unsigned int error_info;
   unsigned int stop;             // host request to exit
+  unsigned int pad0[28];
   unsigned long long admit_head; // admission records consumed
   unsigned long long admit_tail; // admission records published (written by host copies)
+  unsigned long long pad1[14];
+  unsigned long long doorbell;   // bumped whenever tiles are committed to any queue
+  unsigned long long pad2[15];
   unsigned long long tiles_done;
   unsigned long long trace_count;
+  unsigned long long dbg[14];    // scratch counters for kernel bring-up (see VLA_TILE_TIMING)
 };
 
 enum DevError : uint32_t {
@@ -193,6 +202,7 @@ struct DeviceCtx {
   int32_t* tiles_done;           // [n_inst][n_nodes]
   uint64_t* inst_frame;          // [n_inst] frame id currently owning the slot
   const uint64_t* slot_base;     // [n_inst] arena offset of the instance's buffers
+  const uint64_t* input_ptrs;    // [n_inst][N_FRAME_INPUTS] device addresses of the frame's input arrays
   const int32_t* roots;          // nodes without predecessors
   TraceRec* trace;
   DoneRec* done_host;            // mapped pinned host memory, [n_inst]
