@@ -176,6 +176,25 @@ int vla_get_counters(vla_ctx* ctx, uint64_t* tiles, uint64_t* kernel_launches, u
 int vla_policy_probe(int32_t n_cls, const int32_t* taus /*[n_cls*3]*/, const int32_t* pending, const int32_t* feasible,
                      int32_t* cta_count, int32_t* u /*[3]*/, int32_t rr_start, int32_t* picked, int32_t* phase);
 
+/* ---- stand-alone operators: the engine's tile bodies on caller-owned DEVICE tensors ------------------------
+ * Both run asynchronously on `stream` (a cudaStream_t; NULL = default stream). */
+
+/* Fused attention, softmax(Q K^T / sqrt(hd)) V per head with grouped KV heads -- the attention of the VLM
+ * decoder layers and of the action head (Section 2.1, Figure 1).  q [tq, hq*hd], k and v [tkv, hkv*hd],
+ * out [tq, hq*hd]: bf16, row-major, DEVICE, 16-byte aligned.  hd a multiple of 16, at most 256; hq a
+ * multiple of hkv; causal (key j visible to query i iff j <= i) needs tq == tkv.
+ * scratch: DEVICE, 256-byte aligned, at least vla_op_attention_scratch_bytes(); the call writes an error
+ * word and the transposed copy of v there, so calls sharing a scratch buffer must not overlap on the GPU. */
+int vla_op_attention_scratch_bytes(int32_t tkv, int32_t hkv, int32_t hd, size_t* out_bytes);
+int vla_op_attention(const void* q, const void* k, const void* v, void* out, int32_t tq, int32_t tkv, int32_t hq,
+                     int32_t hkv, int32_t hd, int32_t causal, void* scratch, size_t scratch_bytes, void* stream);
+
+/* Linear layer y = act(x W^T) -- the dense contractions of both phases (Section 2.1; Section 2.3 calls them the
+ * VLM's "large GEMMs").  a [m,k] and w [n,k] bf16 row-major DEVICE; k a multiple of 8; fp32 accumulation.
+ * out32 (fp32 [m,n]) and/or out16 (bf16 [m,n]) DEVICE, either may be NULL.  act: 0 none, 1 GeLU (tanh form), 2 SiLU. */
+int vla_op_linear(const void* a, const void* w, float* out32, void* out16, int32_t m, int32_t n, int32_t k, int32_t act,
+                  void* stream);
+
 const char* vla_last_error(vla_ctx* ctx);
 int vla_destroy(vla_ctx* ctx);
 

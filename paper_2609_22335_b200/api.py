@@ -25,7 +25,8 @@ _SOLVER = {"euler": 0, "ddim": 1}
 
 EXPORTS = ["vla_required_arena_bytes", "vla_init", "vla_load_weights", "vla_submit_frame", "vla_submit_frame_device",
            "vla_poll_actions", "vla_wait_idle", "vla_get_trace", "vla_reset_trace", "vla_program_info", "vla_debug_fetch",
-           "vla_get_counters", "vla_policy_probe", "vla_last_error", "vla_destroy"]
+           "vla_get_counters", "vla_policy_probe", "vla_last_error", "vla_destroy",
+           "vla_op_attention_scratch_bytes", "vla_op_attention", "vla_op_linear"]
 
 
 class vla_model_desc(C.Structure):
@@ -87,6 +88,9 @@ def load_library() -> C.CDLL:
     lib.vla_get_counters.argtypes = [C.c_void_p, P(C.c_uint64), P(C.c_uint64), P(C.c_uint64)]
     lib.vla_policy_probe.argtypes = [C.c_int32, P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32),
                                      C.c_int32, P(C.c_int32), P(C.c_int32)]
+    lib.vla_op_attention_scratch_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, P(C.c_size_t)]
+    lib.vla_op_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 6 + [C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.vla_op_linear.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 4 + [C.c_void_p]
     lib.vla_last_error.argtypes = [C.c_void_p]
     lib.vla_last_error.restype = C.c_char_p
     lib.vla_destroy.argtypes = [C.c_void_p]
@@ -340,3 +344,42 @@ def policy_probe(taus, pending, feasible, cta_count, u, rr_start=0):
     if rc != VLA_OK:
         raise VlaError(rc, "policy probe failed")
     return picked.value, phase.value, list(cc), list(uu)
+
+
+def _stream_ptr(stream):
+    return None if stream is None else stream.cuda_stream
+
+
+def op_attention_scratch_bytes(tkv, hkv, hd) -> int:
+    out = C.c_size_t(0)
+    rc = load_library().vla_op_attention_scratch_bytes(tkv, hkv, hd, C.byref(out))
+    if rc != VLA_OK:
+        raise VlaError(rc, "bad attention shape")
+    return out.value
+
+
+def op_attention(q, k, v, hq, hkv, hd, causal=False, scratch=None, stream=None):
+    """q [tq, hq*hd], k/v [tkv, hkv*hd]: CUDA bf16 torch tensors.  Returns out [tq, hq*hd] bf16."""
+    import torch
+    tq, tkv = q.shape[0], k.shape[0]
+    out = torch.empty_like(q)
+    if scratch is None:
+        scratch = torch.empty(op_attention_scratch_bytes(tkv, hkv, hd), dtype=torch.uint8, device=q.device)
+    rc = load_library().vla_op_attention(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), tq, tkv, hq, hkv, hd,
+                                         int(causal), scratch.data_ptr(), scratch.numel(), _stream_ptr(stream))
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_op_attention failed")
+    return out
+
+
+def op_linear(a, w, act=0, out_bf16=False, stream=None):
+    """a [m,k], w [n,k]: CUDA bf16 torch tensors.  Returns act(a w^T) as fp32 (or bf16) [m,n]."""
+    import torch
+    m, k = a.shape
+    n = w.shape[0]
+    out = torch.empty((m, n), dtype=torch.bfloat16 if out_bf16 else torch.float32, device=a.device)
+    rc = load_library().vla_op_linear(a.data_ptr(), w.data_ptr(), None if out_bf16 else out.data_ptr(),
+                                      out.data_ptr() if out_bf16 else None, m, n, k, act, _stream_ptr(stream))
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_op_linear failed")
+    return out

@@ -679,3 +679,5 @@ int vla_destroy(vla_ctx* c) {
 }
 
 }  // extern "C"
+
+#include "ops_api.cuh"
