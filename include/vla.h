@@ -189,6 +189,24 @@ int vla_op_attention_scratch_bytes(int32_t tkv, int32_t hkv, int32_t hd, size_t*
 int vla_op_attention(const void* q, const void* k, const void* v, void* out, int32_t tq, int32_t tkv, int32_t hq,
                      int32_t hkv, int32_t hd, int32_t causal, void* scratch, size_t scratch_bytes, void* stream);
 
+/* Same attention for callers that cannot allocate device memory (no counterpart in the paper: this is a
+ * deployment convenience).  Some callers of this library are not allowed to call cudaMalloc or to hand over
+ * a scratch buffer: code that runs inside a real-time control loop with a fixed memory budget, a plugin whose
+ * host owns every allocation, or a process that must not touch the allocator after start-up.  For them the
+ * scratch of vla_op_attention (an error word plus the transposed copy of v) lives in a fixed array in device
+ * memory that every GPU loading this library holds until the process exits.  The call allocates nothing:
+ * no cudaMalloc, no cudaFree, no allocating library routine; the caller passes only inputs and outputs.
+ * Limit: vla_op_attention_scratch_bytes(tkv, hkv, hd) must not exceed vla_op_attention_static_capacity()
+ * (256 bytes + 4 MiB for the transposed v, e.g. hkv*hd = 1024 with up to 2048 keys); larger shapes are refused
+ * with VLA_ERR_NOMEM and nothing runs.  The first call on each device looks the array's device address up
+ * (with that device current); make that first call outside any stream capture.  All calls on a device share
+ * the one array, which keeps whatever the previous call left: the call clears what it needs cleared, but two
+ * calls that overlap on the GPU (different streams, or the same call from two threads) race on it -- run them
+ * one after the other.  Arguments, layouts and results are those of vla_op_attention. */
+int vla_op_attention_static_capacity(size_t* out_bytes);
+int vla_op_attention_static(const void* q, const void* k, const void* v, void* out, int32_t tq, int32_t tkv, int32_t hq,
+                            int32_t hkv, int32_t hd, int32_t causal, void* stream);
+
 /* Linear layer y = act(x W^T) -- the dense contractions of both phases (Section 2.1; Section 2.3 calls them the
  * VLM's "large GEMMs").  a [m,k] and w [n,k] bf16 row-major DEVICE; k a multiple of 8; fp32 accumulation.
  * out32 (fp32 [m,n]) and/or out16 (bf16 [m,n]) DEVICE, either may be NULL.  act: 0 none, 1 GeLU (tanh form), 2 SiLU. */

@@ -26,7 +26,8 @@ _SOLVER = {"euler": 0, "ddim": 1}
 EXPORTS = ["vla_required_arena_bytes", "vla_init", "vla_load_weights", "vla_submit_frame", "vla_submit_frame_device",
            "vla_poll_actions", "vla_wait_idle", "vla_get_trace", "vla_reset_trace", "vla_program_info", "vla_debug_fetch",
            "vla_get_counters", "vla_policy_probe", "vla_last_error", "vla_destroy",
-           "vla_op_attention_scratch_bytes", "vla_op_attention", "vla_op_linear"]
+           "vla_op_attention_scratch_bytes", "vla_op_attention", "vla_op_linear",
+           "vla_op_attention_static_capacity", "vla_op_attention_static"]
 
 
 class vla_model_desc(C.Structure):
@@ -91,6 +92,8 @@ def load_library() -> C.CDLL:
     lib.vla_op_attention_scratch_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, P(C.c_size_t)]
     lib.vla_op_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 6 + [C.c_void_p, C.c_size_t, C.c_void_p]
     lib.vla_op_linear.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 4 + [C.c_void_p]
+    lib.vla_op_attention_static_capacity.argtypes = [P(C.c_size_t)]
+    lib.vla_op_attention_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 6 + [C.c_void_p]
     lib.vla_last_error.argtypes = [C.c_void_p]
     lib.vla_last_error.restype = C.c_char_p
     lib.vla_destroy.argtypes = [C.c_void_p]
@@ -382,4 +385,20 @@ def op_linear(a, w, act=0, out_bf16=False, stream=None):
                                       out.data_ptr() if out_bf16 else None, m, n, k, act, _stream_ptr(stream))
     if rc != VLA_OK:
         raise VlaError(rc, "vla_op_linear failed")
+    return out
+
+
+def op_attention_static(q, k, v, out, hq, hkv, hd, causal=False, stream=None):
+    """Attention for callers that may not allocate: scratch lives in a fixed device array inside the library.
+
+    Unlike ``op_attention`` this wrapper creates nothing either: the caller supplies ``out``.  Shapes whose
+    scratch need exceeds the fixed array raise with VLA_ERR_NOMEM.  Calls share the array, so do not overlap them.
+    """
+    tq, tkv = q.shape[0], k.shape[0]
+    rc = load_library().vla_op_attention_static(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), tq, tkv, hq, hkv, hd,
+                                                int(causal), _stream_ptr(stream))
+    if rc == VLA_ERR_NOMEM:
+        raise VlaError(rc, "attention shape needs more scratch than the library's fixed array holds")
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_op_attention_static failed")
     return out

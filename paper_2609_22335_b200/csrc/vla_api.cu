@@ -681,3 +681,52 @@ int vla_destroy(vla_ctx* c) {
 }  // extern "C"
 
 #include "ops_api.cuh"
+
+// ------------------------------------------------------------------------------------------------
+// Attention without any allocation: the scratch of vla_op_attention (error word + transposed V)
+// lives in a fixed array in device memory that every GPU loading this library holds until exit.
+// In host code the array's name is only a handle; the device address is looked up once per device
+// with cudaGetSymbolAddress and that pointer is what the kernels receive.
+// ------------------------------------------------------------------------------------------------
+#define VLA_OP_ATTENTION_STATIC_VT_BYTES (4u << 20)   /* room for the transposed V: 4 MiB */
+static __device__ __align__(256) unsigned char g_attention_static_scratch[256 + VLA_OP_ATTENTION_STATIC_VT_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::atomic<void*> g_static_scratch_ptr[kMaxDevices];
+
+// Device address of the static scratch on the current device (looked up on the first call per device).
+int static_scratch_for_current_device(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VLA_ERR_CUDA;
+  void* p = g_static_scratch_ptr[dev].load(std::memory_order_acquire);
+  if (!p) {
+    if (cudaGetSymbolAddress(&p, g_attention_static_scratch) != cudaSuccess || !p) return VLA_ERR_CUDA;
+    g_static_scratch_ptr[dev].store(p, std::memory_order_release);
+  }
+  *out = p;
+  return VLA_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int vla_op_attention_static_capacity(size_t* out_bytes) {
+  if (!out_bytes) return VLA_ERR_INVALID;
+  *out_bytes = sizeof(g_attention_static_scratch);
+  return VLA_OK;
+}
+
+int vla_op_attention_static(const void* q, const void* k, const void* v, void* out, int32_t tq, int32_t tkv, int32_t hq,
+                            int32_t hkv, int32_t hd, int32_t causal, void* stream) {
+  if (!q || !k || !v || !out || !vla::op_attention_shape_ok(tq, tkv, hq, hkv, hd)) return VLA_ERR_INVALID;
+  if (causal && tq != tkv) return VLA_ERR_INVALID;
+  if (vla::op_attention_scratch_bytes(tkv, hkv, hd) > sizeof(g_attention_static_scratch)) return VLA_ERR_NOMEM;
+  void* scratch = nullptr;
+  int rc = static_scratch_for_current_device(&scratch);
+  if (rc != VLA_OK) return rc;
+  // op_attention_run clears the error word itself; V^T is fully rewritten for the rows and tokens it reads
+  return vla::op_attention_run(q, k, v, out, tq, tkv, hq, hkv, hd, causal, scratch, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"
