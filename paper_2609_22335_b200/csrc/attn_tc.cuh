@@ -29,7 +29,8 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 
 __device__ __forceinline__ uint32_t umma_idesc_bf16_n(int n) { return umma_idesc_bf16(n); }
 
-constexpr int ATTN_BQ = 128;
+constexpr int ATTN_BQ = 128;   // queries per tile (MMA M)
+constexpr int ATTN_BN = 64;    // keys per block (MMA N of S, MMA K of P V; one 128-byte swizzle row of P)
 
 // Barrier over the worker's threads that also ANDs a predicate, so every thread takes the same exit.
 __device__ __forceinline__ bool worker_all(const TileCtx& c, bool pred) {
@@ -45,23 +46,62 @@ __device__ __forceinline__ bool worker_all(const TileCtx& c, bool pred) {
   return r != 0;
 }
 
+__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float exp2_fast(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Key blocks of a tile: segment 0 (cached prefix) then segment 1 (the head's own keys), 64 keys each,
+// never straddling a segment; with a causal mask the walk stops at the diagonal.
+struct KvBlock {
+  int seg, kv0;
+  bool valid;
+};
+__device__ __forceinline__ KvBlock kv_first(const AttnArgs& a) {
+  KvBlock b;
+  b.seg = a.t0 > 0 ? 0 : 1;
+  b.kv0 = 0;
+  b.valid = (a.t0 > 0 || a.t1 > 0);
+  return b;
+}
+__device__ __forceinline__ KvBlock kv_next(const AttnArgs& a, KvBlock b, int q_last) {
+  b.kv0 += ATTN_BN;
+  const int L = b.seg == 0 ? a.t0 : a.t1;
+  if (b.kv0 >= L) {
+    if (b.seg == 0 && a.t1 > 0) { b.seg = 1; b.kv0 = 0; }
+    else b.valid = false;
+  }
+  if (a.causal && b.kv0 > q_last) b.valid = false;
+  return b;
+}
+
 __device__ void tile_attention(const TileCtx& c, const AttnArgs& a, int tile) {
   const int warp = c.tid >> 5, lane = c.tid & 31;
   const int head = tile / a.q_blocks, qb = tile % a.q_blocks;
   const int g = (head * a.hkv) / a.hq;
   const int q0 = qb * ATTN_BQ;
-  const int hs = a.hs, bn = a.bn;
+  const int hs = a.hs;
   const int nbox = (hs + 63) / 64;          // 64-column boxes covering one head
   const int kchunks = hs / 16;              // 16-wide K steps of Q K^T
-  const int nsub = bn / 64;                 // 64-key sub-tiles of P and V^T
 
   // shared-memory carve-up (all tile bases 1024-byte aligned)
   const uint32_t base = smem_u32(c.smem);
   const uint32_t bar_q = base, bar_k = base + 8, bar_v = base + 16, bar_s = base + 24, bar_o = base + 32;
   const uint32_t Qs = base + 1024;
   const uint32_t Ks = Qs + (uint32_t)nbox * (ATTN_BQ * 128);
-  const uint32_t Vs = Ks + (uint32_t)nbox * (uint32_t)(bn * 128);
-  const uint32_t Ps = Vs + (uint32_t)nsub * (uint32_t)(hs * 128);
+  const uint32_t Vs = Ks + (uint32_t)nbox * (ATTN_BN * 128);
+  const uint32_t Ps = Vs + (uint32_t)(hs * 128);
   char* Ps_gen = c.smem + (Ps - base);
 
   if (c.tid == 0) {
@@ -70,124 +110,137 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a, int tile) {
   }
   worker_sync(c);
 
-  const uint32_t tmem_s = c.tmem;                       // S: columns [0, bn)
-  const uint32_t tmem_o = c.tmem + (uint32_t)bn;        // O: columns [bn, bn + hs)
+  const uint32_t tmem_s = c.tmem;                            // S: columns [0, 64)
+  const uint32_t tmem_o = c.tmem + (uint32_t)ATTN_BN;        // O: columns [64, 64 + hs)
   const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
   const char* tm = reinterpret_cast<const char*>(c.tmaps);
   auto map_ptr = [&](int idx) { return reinterpret_cast<const void*>(tm + (size_t)(c.amap_base + idx) * 128); };
-  const uint32_t idesc_s = umma_idesc_bf16(bn), idesc_o = umma_idesc_bf16(hs);
+  const uint32_t idesc_s = umma_idesc_bf16(ATTN_BN), idesc_o = umma_idesc_bf16(hs);
+  const bool issuer = c.tid == 0;
+  auto load_k = [&](const KvBlock& b) {
+    mbar_expect_tx(bar_k, (uint32_t)nbox * (ATTN_BN * 128));
+    const void* m = map_ptr(b.seg == 0 ? a.k0map : a.k1map);
+    for (int i = 0; i < nbox; ++i) tma_load_2d(Ks + (uint32_t)i * (ATTN_BN * 128), m, bar_k, g * hs + i * 64, b.kv0);
+  };
+  auto load_v = [&](const KvBlock& b) {
+    mbar_expect_tx(bar_v, (uint32_t)(hs * 128));
+    tma_load_2d(Vs, map_ptr(b.seg == 0 ? a.v0map : a.v1map), bar_v, b.kv0, g * hs);
+  };
 
-  if (c.tid == 0) {
+  KvBlock cur = kv_first(a);
+  if (issuer) {
     asm volatile("fence.proxy.async;" ::: "memory");
     mbar_expect_tx(bar_q, (uint32_t)nbox * (ATTN_BQ * 128));
     for (int b = 0; b < nbox; ++b) tma_load_2d(Qs + (uint32_t)b * (ATTN_BQ * 128), map_ptr(a.qmap), bar_q, head * hs + b * 64, q0);
+    if (cur.valid) load_k(cur);
   }
 
   const int row = q0 + warp * 32 + lane;                // this thread's query
+  const int r_in = warp * 32 + lane;
   float m_run = -INFINITY, l_run = 0.f;
   int blk = 0;
   bool ok = true;
-  for (int seg = 0; seg < 2 && ok; ++seg) {
-    const int L = seg == 0 ? a.t0 : a.t1;
-    const int kmap = seg == 0 ? a.k0map : a.k1map, vmap = seg == 0 ? a.v0map : a.v1map;
-    for (int kv0 = 0; kv0 < L && ok; kv0 += bn, ++blk) {
-      if (a.causal && kv0 > q0 + ATTN_BQ - 1) break;    // whole block above the diagonal
-      const uint32_t ph = (uint32_t)blk & 1u;
-      if (warp == 0) {           // lanes 1..31 park at the __syncwarp below instead of spinning beside the issuing lane
+  while (cur.valid) {
+    const KvBlock nxt = kv_next(a, cur, q0 + ATTN_BQ - 1);
+    const uint32_t ph = (uint32_t)blk & 1u;
+    // ---- S = Q K^T of this block (issued by one lane; its warp mates park at the __syncwarp)
+    if (warp == 0) {
       if (lane == 0) {
-        // K and V^T of this block (single-buffered: the previous block's MMAs have completed)
-        mbar_expect_tx(bar_k, (uint32_t)nbox * (uint32_t)(bn * 128));
-        for (int b = 0; b < nbox; ++b) tma_load_2d(Ks + (uint32_t)b * (uint32_t)(bn * 128), map_ptr(kmap), bar_k, g * hs + b * 64, kv0);
-        mbar_expect_tx(bar_v, (uint32_t)nsub * (uint32_t)(hs * 128));
-        for (int j = 0; j < nsub; ++j) tma_load_2d(Vs + (uint32_t)j * (uint32_t)(hs * 128), map_ptr(vmap), bar_v, kv0 + j * 64, g * hs);
-        ok = (blk > 0 || mbar_wait(c, bar_q, 0u)) && mbar_wait(c, bar_k, ph);
-        if (ok) {
+        bool go = (blk > 0 || mbar_wait(c, bar_q, 0u)) && mbar_wait(c, bar_k, ph);
+        if (go) {
           tc_fence_after();
           for (int kc = 0; kc < kchunks; ++kc) {
             const uint64_t qd = umma_desc_sw128(Qs + (uint32_t)(kc >> 2) * (ATTN_BQ * 128)) + 2u * (kc & 3);
-            const uint64_t kd = umma_desc_sw128(Ks + (uint32_t)(kc >> 2) * (uint32_t)(bn * 128)) + 2u * (kc & 3);
+            const uint64_t kd = umma_desc_sw128(Ks + (uint32_t)(kc >> 2) * (ATTN_BN * 128)) + 2u * (kc & 3);
             umma_bf16(tmem_s, qd, kd, idesc_s, kc != 0 ? 1u : 0u);
           }
           umma_commit(bar_s);
         }
       }
       __syncwarp();
-      }
-      // ---- softmax of this block, one thread per query row
-      ok = worker_all(c, mbar_wait(c, bar_s, ph));
-      tc_fence_after();
-      if (!ok) break;
-      const int valid = min(bn, L - kv0);
-      const int lim = a.causal ? min(valid, row - kv0 + 1) : valid;   // keys [0, lim) of the block are visible to this row
-      float mx = m_run;
-      for (int c0 = 0; c0 < bn; c0 += 16) {
-        float s[16];
-        tmem_ld16(tmem_s + lane_off + (uint32_t)c0, s);
-#pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (c0 + j < lim) mx = fmaxf(mx, s[j]);
-      }
-      const float alpha = (m_run == -INFINITY) ? 0.f : exp2f((m_run - mx) * a.scale_log2e);
-      float sum = 0.f;
-      for (int c0 = 0; c0 < bn; c0 += 16) {
-        float s[16];
-        tmem_ld16(tmem_s + lane_off + (uint32_t)c0, s);
-        uint32_t packed[8];
-#pragma unroll
-        for (int j = 0; j < 16; j += 2) {
-          float p0 = (c0 + j < lim) ? exp2f((s[j] - mx) * a.scale_log2e) : 0.f;
-          float p1 = (c0 + j + 1 < lim) ? exp2f((s[j + 1] - mx) * a.scale_log2e) : 0.f;
-          // the row sum uses the bf16-rounded probabilities the MMA will see
-          __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-          sum += __low2float(pk) + __high2float(pk);
-          packed[j >> 1] = *reinterpret_cast<uint32_t*>(&pk);
-        }
-        // two 16-byte chunks of this row in the swizzled P tile
-        const int r = warp * 32 + lane;
-        const int sub = c0 >> 6, ch = (c0 & 63) >> 3;
-        char* prow = Ps_gen + (size_t)sub * (ATTN_BQ * 128) + (size_t)r * 128;
-        *reinterpret_cast<uint4*>(prow + (((ch) ^ (r & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-        *reinterpret_cast<uint4*>(prow + (((ch + 1) ^ (r & 7)) << 4)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
-      }
-      l_run = l_run * alpha + sum;
-      m_run = mx;
-      // rescale O where a row maximum moved (warp-uniform decision: the TMEM accesses are warp-wide)
-      if (blk > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
-        for (int c0 = 0; c0 < hs; c0 += 16) {
-          float o[16];
-          tmem_ld16(tmem_o + lane_off + (uint32_t)c0, o);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) o[j] *= alpha;
-          tmem_st16(tmem_o + lane_off + (uint32_t)c0, o);
-        }
-        tmem_st_wait();
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P written by generic stores, read by the MMA
-      tc_fence_before();
-      worker_sync(c);
-      if (warp == 0) {
+    }
+    ok = worker_all(c, mbar_wait(c, bar_s, ph));
+    tc_fence_after();
+    if (!ok) break;
+    // S(blk) complete implies P V(blk-1) complete: K, V^T and P buffers are free.  Fetch the next K and
+    // this block's V^T now; both loads hide behind the softmax below.
+    if (warp == 0) {
       if (lane == 0) {
-        ok = mbar_wait(c, bar_v, ph);
-        if (ok) {
+        if (nxt.valid) load_k(nxt);
+        load_v(cur);
+      }
+      __syncwarp();
+    }
+    // ---- softmax of this block: one thread per query row, the 64 scores held in registers
+    const int L = cur.seg == 0 ? a.t0 : a.t1;
+    const int valid = min(ATTN_BN, L - cur.kv0);
+    const int lim = a.causal ? min(valid, row - cur.kv0 + 1) : valid;   // keys [0, lim) of the block are visible to this row
+    uint32_t sr[ATTN_BN];
+    tmem_ld16_nowait(tmem_s + lane_off + 0u, sr + 0);
+    tmem_ld16_nowait(tmem_s + lane_off + 16u, sr + 16);
+    tmem_ld16_nowait(tmem_s + lane_off + 32u, sr + 32);
+    tmem_ld16_nowait(tmem_s + lane_off + 48u, sr + 48);
+    tmem_ld_wait();
+    float mx = m_run;
+#pragma unroll
+    for (int j = 0; j < ATTN_BN; ++j)
+      if (j < lim) mx = fmaxf(mx, __uint_as_float(sr[j]));
+    const float alpha = (m_run == -INFINITY) ? 0.f : exp2_fast((m_run - mx) * a.scale_log2e);
+    const float mb = mx * a.scale_log2e;
+    float sum = 0.f;
+    char* prow = Ps_gen + (size_t)r_in * 128;
+#pragma unroll
+    for (int ch = 0; ch < ATTN_BN / 8; ++ch) {
+      uint32_t pk[4];
+#pragma unroll
+      for (int j = 0; j < 8; j += 2) {
+        const int jj = ch * 8 + j;
+        float p0 = (jj < lim) ? exp2_fast(fmaf(__uint_as_float(sr[jj]), a.scale_log2e, -mb)) : 0.f;
+        float p1 = (jj + 1 < lim) ? exp2_fast(fmaf(__uint_as_float(sr[jj + 1]), a.scale_log2e, -mb)) : 0.f;
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);     // the row sum uses the rounded probabilities the MMA sees
+        sum += __low2float(h2) + __high2float(h2);
+        pk[j >> 1] = *reinterpret_cast<uint32_t*>(&h2);
+      }
+      *reinterpret_cast<uint4*>(prow + ((ch ^ (r_in & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+    l_run = l_run * alpha + sum;
+    m_run = mx;
+    // rescale O where a row maximum moved (warp-uniform decision: the TMEM accesses are warp-wide)
+    if (blk > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
+      for (int c0 = 0; c0 < hs; c0 += 16) {
+        float o[16];
+        tmem_ld16(tmem_o + lane_off + (uint32_t)c0, o);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) o[j] *= alpha;
+        tmem_st16(tmem_o + lane_off + (uint32_t)c0, o);
+      }
+      tmem_st_wait();
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P written by generic stores, read by the MMA
+    tc_fence_before();
+    worker_sync(c);
+    // ---- O += P V
+    if (warp == 0) {
+      if (lane == 0) {
+        if (mbar_wait(c, bar_v, ph)) {
           tc_fence_after();
-          for (int kc = 0; kc < bn / 16; ++kc) {
-            const uint64_t pd = umma_desc_sw128(Ps + (uint32_t)(kc >> 2) * (ATTN_BQ * 128)) + 2u * (kc & 3);
-            const uint64_t vd = umma_desc_sw128(Vs + (uint32_t)(kc >> 2) * (uint32_t)(hs * 128)) + 2u * (kc & 3);
+          for (int kc = 0; kc < ATTN_BN / 16; ++kc) {
+            const uint64_t pd = umma_desc_sw128(Ps) + 2u * kc;
+            const uint64_t vd = umma_desc_sw128(Vs) + 2u * kc;
             umma_bf16(tmem_o, pd, vd, idesc_o, (blk | kc) != 0 ? 1u : 0u);
           }
           umma_commit(bar_o);
-          ok = mbar_wait(c, bar_o, ph);     // K, V^T and P buffers are free again
         }
       }
       __syncwarp();
-      }
     }
+    cur = nxt;
+    ++blk;
   }
-  // ---- epilogue: O / l -> bf16
-  worker_sync(c);    // thread 0 has seen the last P V complete
+  // ---- epilogue: O / l -> bf16 (after the last P V has landed)
+  if (ok && blk > 0) ok = worker_all(c, mbar_wait(c, bar_o, (uint32_t)(blk - 1) & 1u));
   tc_fence_after();
-  const bool failed = *reinterpret_cast<volatile unsigned*>(c.error) != 0u;
-  if (!failed && blk > 0) {
+  if (ok && blk > 0) {
     unsigned short* O = resolve<unsigned short>(c, a.out);
     const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
     for (int c0 = 0; c0 < hs; c0 += 16) {

@@ -128,19 +128,22 @@ struct WorkerCmd {
 
 struct SmState {
   unsigned lock;
-  unsigned smem_mask, tmem_mask;   // bit i set = unit i in use
+  unsigned long long smem_mask;    // bit i set = shared-memory unit i in use
+  unsigned tmem_mask;              // bit i set = tensor-memory unit i in use
   int n_smem_units, n_tmem_units;
   PickState pick;
+  int waiter;                      // worker holding a tile while it waits for room (-1: none)
   unsigned tmem_base;
   unsigned long long tiles;        // tiles this SM ran (added to the global counter at exit)
   WorkerCmd cur[MAX_WORKERS];
 };
 static_assert(sizeof(SmState) <= SM_STATE_BYTES, "SM state too large");
 
-__device__ __forceinline__ int find_free(unsigned mask, int need, int total) {
+__device__ __forceinline__ unsigned long long unit_bits(int n) { return n >= 64 ? ~0ull : ((1ull << n) - 1ull); }
+__device__ __forceinline__ int find_free(unsigned long long mask, int need, int total) {
   if (need == 0) return 0;
   if (need > total) return -1;
-  unsigned want = (need >= 32) ? 0xffffffffu : ((1u << need) - 1u);
+  const unsigned long long want = unit_bits(need);
   for (int i = 0; i + need <= total; ++i)
     if (((mask >> i) & want) == 0) return i;
   return -1;
@@ -218,6 +221,10 @@ __device__ inline void try_admit(const DeviceCtx& ctx) {
 }
 
 // Leader of a worker: find the next tile for this worker under the pick policy.
+// Feasibility is tested with each class's smallest footprint; the tile actually claimed is then
+// given its exact shared-memory and tensor-memory need.  If that does not fit yet, the worker keeps
+// the tile and waits (bounded) for co-resident tiles to finish; meanwhile it is the SM's only
+// "waiter" and the other workers admit nothing that needs shared or tensor memory.
 __device__ inline bool try_pick(const DeviceCtx& ctx, SmState* sm, int worker, uint64_t deadline) {
   unsigned pending = 0;
   for (int c = 0; c < N_CLASSES; ++c)
@@ -229,40 +236,62 @@ __device__ inline bool try_pick(const DeviceCtx& ctx, SmState* sm, int worker, u
     if ((++spins & 255u) == 0 && gtimer() > deadline) return false;
   }
   bool got = false;
-  int tau[N_CLASSES * 3];
-  for (int c = 0; c < N_CLASSES; ++c)
+  int tau[N_CLASSES * 3], group[N_CLASSES];
+  for (int c = 0; c < N_CLASSES; ++c) {
     for (int x = 0; x < 3; ++x) tau[c * 3 + x] = ctx.classes[c].tau[x];
+    group[c] = ctx.classes[c].group;
+  }
+  const bool blocked = sm->waiter >= 0 && sm->waiter != worker;
+  WorkerCmd& cmd = sm->cur[worker];
   for (int attempt = 0; attempt < N_CLASSES && pending; ++attempt) {
     unsigned feasible = 0;
     for (int c = 0; c < N_CLASSES; ++c) {
-      if (find_free(sm->smem_mask, ctx.classes[c].smem_units, sm->n_smem_units) >= 0 &&
-          find_free(sm->tmem_mask, ctx.classes[c].tmem_units, sm->n_tmem_units) >= 0)
+      const int su = ctx.classes[c].smem_units, tu = ctx.classes[c].tmem_units;
+      if (blocked && (su > 0 || tu > 0)) continue;
+      if (find_free(sm->smem_mask, su, sm->n_smem_units) >= 0 && find_free(sm->tmem_mask, tu, sm->n_tmem_units) >= 0)
         feasible |= 1u << c;
     }
     int phase;
-    int k = pick_choose(N_CLASSES, tau, pending, feasible, sm->pick, sm->pick.rr, ctx.policy, &phase);
+    int k = pick_choose(N_CLASSES, tau, group, pending, feasible, sm->pick, sm->pick.rr, ctx.policy, &phase);
     if (k < 0) break;
     QueueEntry e;
     if (!queue_try_pop(ctx, k, e, deadline)) {
       pending &= ~(1u << k);
       continue;
     }
-    WorkerCmd& cmd = sm->cur[worker];
     cmd.kind = 0;
     cmd.inst = e.inst_node >> 20;
     cmd.node = e.inst_node & 0xFFFFFu;
     cmd.tile = e.tile;
     cmd.cls = k;
-    cmd.smem_units = ctx.classes[k].smem_units;
-    cmd.tmem_units = ctx.classes[k].tmem_units;
-    cmd.smem_unit0 = find_free(sm->smem_mask, cmd.smem_units, sm->n_smem_units);
-    cmd.tmem_unit0 = find_free(sm->tmem_mask, cmd.tmem_units, sm->n_tmem_units);
-    if (cmd.smem_units) sm->smem_mask |= ((cmd.smem_units >= 32 ? 0xffffffffu : ((1u << cmd.smem_units) - 1u)) << cmd.smem_unit0);
-    if (cmd.tmem_units) sm->tmem_mask |= ((cmd.tmem_units >= 32 ? 0xffffffffu : ((1u << cmd.tmem_units) - 1u)) << cmd.tmem_unit0);
+    const NodeDesc& nd = ctx.nodes[cmd.node];
+    cmd.smem_units = (nd.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT;
+    cmd.tmem_units = (nd.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT;
     pick_commit(sm->pick, k, tau);
     sm->pick.rr = (k + 1) % N_CLASSES;
     got = true;
     break;
+  }
+  if (got) {
+    // exact allocation; hold the tile and wait when the SM is too full right now
+    for (;;) {
+      cmd.smem_unit0 = find_free(sm->smem_mask, cmd.smem_units, sm->n_smem_units);
+      cmd.tmem_unit0 = find_free((unsigned long long)sm->tmem_mask, cmd.tmem_units, sm->n_tmem_units);
+      if (cmd.smem_unit0 >= 0 && cmd.tmem_unit0 >= 0) break;
+      sm->waiter = worker;
+      __threadfence_block();
+      atomicExch(&sm->lock, 0u);
+      __nanosleep(200);
+      if (gtimer() > deadline || ld_volatile_u32(&ctx.control->error) != 0u) {
+        set_error(ctx, DEV_ERR_IDLE_LIMIT, 0x1000u + (unsigned)blockIdx.x);
+        cmd.kind = 1;
+        return true;    // leave: kind = exit
+      }
+      while (atomicCAS(&sm->lock, 0u, 1u) != 0u) __nanosleep(32);
+    }
+    if (sm->waiter == worker) sm->waiter = -1;
+    if (cmd.smem_units) sm->smem_mask |= unit_bits(cmd.smem_units) << cmd.smem_unit0;
+    if (cmd.tmem_units) sm->tmem_mask |= (unsigned)(unit_bits(cmd.tmem_units) << cmd.tmem_unit0);
   }
   __threadfence_block();
   atomicExch(&sm->lock, 0u);
@@ -271,8 +300,8 @@ __device__ inline bool try_pick(const DeviceCtx& ctx, SmState* sm, int worker, u
 
 __device__ inline void release_resources(const DeviceCtx& ctx, SmState* sm, const WorkerCmd& cmd) {
   while (atomicCAS(&sm->lock, 0u, 1u) != 0u) __nanosleep(32);
-  if (cmd.smem_units) sm->smem_mask &= ~((cmd.smem_units >= 32 ? 0xffffffffu : ((1u << cmd.smem_units) - 1u)) << cmd.smem_unit0);
-  if (cmd.tmem_units) sm->tmem_mask &= ~((cmd.tmem_units >= 32 ? 0xffffffffu : ((1u << cmd.tmem_units) - 1u)) << cmd.tmem_unit0);
+  if (cmd.smem_units) sm->smem_mask &= ~(unit_bits(cmd.smem_units) << cmd.smem_unit0);
+  if (cmd.tmem_units) sm->tmem_mask &= ~(unsigned)(unit_bits(cmd.tmem_units) << cmd.tmem_unit0);
   int tau[3] = {ctx.classes[cmd.cls].tau[0], ctx.classes[cmd.cls].tau[1], ctx.classes[cmd.cls].tau[2]};
   sm->pick.cta_count[cmd.cls] -= 1;
   for (int x = 0; x < 3; ++x) sm->pick.u[x] -= tau[x];
@@ -296,12 +325,13 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_ke
     sm->smem_mask = 0;
     sm->tmem_mask = 0;
     int units = (dyn_smem_bytes - SM_STATE_BYTES) / SMEM_UNIT;
-    sm->n_smem_units = units > 32 ? 32 : units;
+    sm->n_smem_units = units > 64 ? 64 : units;
     sm->n_tmem_units = 512 / TMEM_UNIT;
     for (int c = 0; c < PICK_MAX_CLASSES; ++c) sm->pick.cta_count[c] = 0;
     sm->pick.u[0] = sm->pick.u[1] = sm->pick.u[2] = 0;
     sm->pick.rr = (int)(blockIdx.x % N_CLASSES);
     sm->tmem_base = 0;
+    sm->waiter = -1;
     sm->tiles = 0;
   }
   __syncthreads();
@@ -331,7 +361,14 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_ke
         }
         if (bell != bell_seen || slow) {
           bell_seen = bell;
+#ifdef VLA_TILE_TIMING
+          const uint64_t tp0 = gtimer();
+          const bool hit = try_pick(ctx, sm, worker, wait_start + ctx.wait_limit_ns);
+          atomicAdd(ctl->dbg + (hit ? 5 : 7), gtimer() - tp0); atomicAdd(ctl->dbg + (hit ? 6 : 8), 1ull);
+          if (hit) break;
+#else
           if (try_pick(ctx, sm, worker, wait_start + ctx.wait_limit_ns)) break;   // cmd.kind = 0 now
+#endif
         }
         if (slow) {
           const uint64_t now = gtimer();
@@ -380,6 +417,9 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_ke
       write_trace(ctx, cmd.inst, cmd.node, cmd.tile, worker, cmd.cls, frame, t0, t1);
       release_resources(ctx, sm, cmd);
       complete_tile(ctx, cmd.inst, cmd.node, true, &sm->cur[worker]);
+#ifdef VLA_TILE_TIMING
+      atomicAdd(ctl->dbg + 9, gtimer() - t1); atomicAdd(ctl->dbg + 10, 1ull);
+#endif
     }
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
     const int n_ready = sm->cur[worker].n_ready;
@@ -444,7 +484,9 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_node_kernel(DeviceCtx ctx,
 __global__ void vla_pick_probe_kernel(int n_cls, const int* tau, unsigned pending, unsigned feasible, PickState* st,
                                       int rr_start, int policy, int* out) {
   int phase;
-  int k = pick_choose(n_cls, tau, pending, feasible, *st, rr_start, policy, &phase);
+  int group[PICK_MAX_CLASSES];
+  for (int i = 0; i < PICK_MAX_CLASSES; ++i) group[i] = i;   // one class per group: the paper's listing
+  int k = pick_choose(n_cls, tau, group, pending, feasible, *st, rr_start, policy, &phase);
   if (k >= 0) pick_commit(*st, k, tau);
   out[0] = k;
   out[1] = phase;

@@ -134,7 +134,7 @@ inline int op_attention_run(const void* q, const void* k, const void* v, void* o
   a.ldo = hq * hd;
   a.tq = tq; a.t0 = tkv; a.t1 = 0;
   a.hq = hq; a.hkv = hkv; a.hd = hd; a.hs = hd; a.causal = causal ? 1 : 0;
-  a.bn = hd <= 64 ? 128 : 64;
+  a.bn = 64;
   a.q_blocks = (tq + 127) / 128;
   a.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
   a.qmap = 0; a.k0map = 1; a.v0map = 2; a.k1map = 1; a.v1map = 2;
@@ -144,8 +144,8 @@ inline int op_attention_run(const void* q, const void* k, const void* v, void* o
       !op_encode(&maps.m[1], k, tkv, (int64_t)hkv * hd, (int64_t)hkv * hd, a.bn) ||
       !op_encode(&maps.m[2], vt, (int64_t)hkv * hd, tkv, tpad, hd))
     return VLA_ERR_CUDA;
-  const int nbox = (hd + 63) / 64, nsub = a.bn / 64;
-  const int smem = 1024 + nbox * 128 * 128 + nbox * a.bn * 128 + nsub * hd * 128 + nsub * 128 * 128;
+  const int nbox = (hd + 63) / 64;
+  const int smem = 1024 + nbox * 128 * 128 + nbox * a.bn * 128 + hd * 128 + 128 * 128;
   int tmem_cols = 32;
   while (tmem_cols < a.bn + hd) tmem_cols <<= 1;
   if (cudaFuncSetAttribute(vla_op_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
@@ -183,7 +183,7 @@ int vla_op_linear(const void* a, const void* w, float* out32, void* out16, int32
   g.out32 = reinterpret_cast<Ref>(out32); g.ldo32 = n;
   g.out16 = reinterpret_cast<Ref>(out16); g.ldo16 = n;
   g.act = act; g.c_acc = 1.f; g.c_x = 1.f;
-  g.tiles_t = (m + 255) / 256;
+  g.tiles_t = (m + GEMM_MAX_BT - 1) / GEMM_MAX_BT;
   g.bt = (int)op_pad((m + g.tiles_t - 1) / g.tiles_t, 16);
   const int stage = GEMM_BM * GEMM_BK * 2 + g.bt * GEMM_BK * 2;
   g.stages = std::max(1, std::min(std::max(2, std::min(4, GEMM_SMEM_BUDGET / stage)), g.Kp / GEMM_BK));

@@ -6,9 +6,13 @@
 // Feasible(k, j) is "the class's shared-memory and tensor-memory need fits what
 // this SM has free right now".  One call chooses at most one class.
 //
-//   Phase 1  a pending, feasible class with no tile resident on this SM wins,
-//            scanning from a rotating start (co-residency priority: a short
-//            action-head tile is never stuck behind resident VLM tiles);
+//   Phase 1  a pending, feasible class whose GROUP has no tile resident on this SM
+//            wins, scanning from a rotating start (co-residency priority: a short
+//            action-head tile is never stuck behind resident VLM tiles).  A group
+//            is what the paper calls a kernel of one stream: the engine groups the
+//            tile classes by phase (VLM stream, action-head stream: K = 2, as in
+//            the paper's evaluation); with one class per group this is the
+//            paper's listing exactly;
 //   Phase 2  otherwise the pending feasible class with the largest
 //            s = sum_x (U_max - U_x[j]) * tau_x(k); strict '>' keeps the first seen.
 //
@@ -36,8 +40,8 @@ struct PickState {
 enum PickPolicy : int { POLICY_TWO_PHASE = 0, POLICY_CLASS_ORDER = 1, POLICY_ROUND_ROBIN = 2 };
 
 // Returns the chosen class or -1; *phase = 1 or 2 (0 when nothing was chosen).
-VLA_HD inline int pick_choose(int n_cls, const int* tau /*[n_cls][3]*/, unsigned pending, unsigned feasible,
-                              const PickState& st, int rr_start, int policy, int* phase) {
+VLA_HD inline int pick_choose(int n_cls, const int* tau /*[n_cls][3]*/, const int* group /*[n_cls]*/, unsigned pending,
+                              unsigned feasible, const PickState& st, int rr_start, int policy, int* phase) {
   *phase = 0;
   unsigned ok = pending & feasible;
   if (ok == 0) return -1;
@@ -53,9 +57,12 @@ VLA_HD inline int pick_choose(int n_cls, const int* tau /*[n_cls][3]*/, unsigned
     }
     return -1;
   }
+  int resident[PICK_MAX_CLASSES];                         // tiles resident per group
+  for (int g = 0; g < PICK_MAX_CLASSES; ++g) resident[g] = 0;
+  for (int k = 0; k < n_cls; ++k) resident[group[k]] += st.cta_count[k];
   for (int i = 0; i < n_cls; ++i) {                       // Phase 1
     int k = (rr_start + i) % n_cls;
-    if ((ok & (1u << k)) && st.cta_count[k] == 0) { *phase = 1; return k; }
+    if ((ok & (1u << k)) && resident[group[k]] == 0) { *phase = 1; return k; }
   }
   int best = -1, best_score = -1;                         // Phase 2
   for (int k = 0; k < n_cls; ++k) {

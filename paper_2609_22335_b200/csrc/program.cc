@@ -216,12 +216,8 @@ class Builder {
     g.out16 = ref(o.out16); g.ldo16 = o.out16.buf >= 0 ? (int)ld(o.out16) : 0;
     g.outT = ref(o.outT); g.ldoT = o.outT.buf >= 0 ? (int)ld(o.outT) : 0; g.t_col0 = o.t_col0;
     g.act = o.act;
-    int tiles_t = (int)((g.M + 255) / 256);
+    int tiles_t = (int)((g.M + GEMM_MAX_BT - 1) / GEMM_MAX_BT);
     int bt = (int)pad_to((g.M + tiles_t - 1) / tiles_t, 16);
-    if (g.dual && bt > 128) {              // two accumulators: keep both within the tensor-memory budget of one worker
-      tiles_t = (int)((g.M + 127) / 128);
-      bt = (int)pad_to((g.M + tiles_t - 1) / tiles_t, 16);
-    }
     g.bt = bt; g.tiles_t = tiles_t;
     {
       // pipeline depth from the stage size; tensor maps for the operands
@@ -313,11 +309,11 @@ class Builder {
     a.out = ref(out); a.ldo = (int)ld(out);
     a.tq = tq; a.t0 = kv0.T; a.t1 = kv1 ? kv1->T : 0;
     a.hq = hq; a.hkv = hkv; a.hd = hd; a.hs = hs; a.causal = causal;
-    a.bn = hs <= 64 ? 128 : 64;
+    a.bn = 64;
     a.q_blocks = (tq + 127) / 128;
     a.scale_log2e = 1.4426950408889634f / std::sqrt((float)hd);
-    const int nbox = (hs + 63) / 64, nsub = a.bn / 64;
-    n.smem_bytes = 1024 + nbox * 128 * 128 + nbox * a.bn * 128 + nsub * hs * 128 + nsub * 128 * 128;
+    const int nbox = (hs + 63) / 64;
+    n.smem_bytes = 1024 + nbox * 128 * 128 + nbox * a.bn * 128 + hs * 128 + 128 * 128;
     n.tmem_cols = (int)pad_to(a.bn + hs, TMEM_UNIT);
     n.n_tiles = hq * a.q_blocks;
     // tensor maps: Q rows in 128-row boxes, K rows in bn-row boxes, V^T in hs-row boxes of 64 tokens
@@ -898,15 +894,20 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   const int taus[N_CLASSES][3] = {{15, 2, 3}, {8, 8, 2}, {0, 4, 10}, {2, 3, 12}, {1, 8, 4}, {0, 3, 6}};
   for (int c = 0; c < N_CLASSES; ++c) {
     for (int x_ = 0; x_ < 3; ++x_) p.classes[c].tau[x_] = taus[c][x_];
-    p.classes[c].smem_units = 0;
-    p.classes[c].tmem_units = 0;
-    p.classes[c].pad[0] = p.classes[c].pad[1] = p.classes[c].pad[2] = 0;
+    p.classes[c].smem_units = 1 << 20;
+    p.classes[c].tmem_units = 1 << 20;
+    p.classes[c].group = c / 3;
+    p.classes[c].pad[0] = p.classes[c].pad[1] = 0;
   }
   for (const NodeDesc& n : p.nodes) {
-    if (n.smem_bytes > 26 * SMEM_UNIT) { set_err(p, "a tile needs more shared memory than one SM offers"); return false; }
+    if (n.smem_bytes > 54 * SMEM_UNIT) { set_err(p, "a tile needs more shared memory than one SM offers"); return false; }
     ClassInfo& ci = p.classes[n.cls];
-    ci.smem_units = std::max(ci.smem_units, (n.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT);
-    ci.tmem_units = std::max(ci.tmem_units, (n.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT);
+    ci.smem_units = std::min(ci.smem_units, (n.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT);
+    ci.tmem_units = std::min(ci.tmem_units, (n.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT);
+  }
+  for (int c = 0; c < N_CLASSES; ++c) {
+    if (p.classes[c].smem_units == (1 << 20)) p.classes[c].smem_units = 0;
+    if (p.classes[c].tmem_units == (1 << 20)) p.classes[c].tmem_units = 0;
   }
 
   // ================================================================== arena layout

@@ -606,6 +606,10 @@ int vla_get_counters(vla_ctx* c, uint64_t* tiles, uint64_t* kernel_launches, uin
       fprintf(stderr, "dbg: first_full %.2f us  mainloop %.2f us  epilogue %.2f us  tiles %llu  kb/tile %.1f\n",
               ctl.dbg[3] ? ctl.dbg[0] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3] ? ctl.dbg[1] / 1e3 / ctl.dbg[3] : 0.0,
               ctl.dbg[3] ? ctl.dbg[2] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3], ctl.dbg[3] ? (double)ctl.dbg[4] / ctl.dbg[3] : 0.0);
+    if (getenv("VLA_PRINT_DBG"))
+      fprintf(stderr, "dbg: pick hit %.2f us x %llu  pick miss %.2f us x %llu  complete %.2f us x %llu\n",
+              ctl.dbg[6] ? ctl.dbg[5] / 1e3 / ctl.dbg[6] : 0.0, ctl.dbg[6], ctl.dbg[8] ? ctl.dbg[7] / 1e3 / ctl.dbg[8] : 0.0,
+              ctl.dbg[8], ctl.dbg[10] ? ctl.dbg[9] / 1e3 / ctl.dbg[10] : 0.0, ctl.dbg[10]);
   }
   if (kernel_launches) *kernel_launches = c->n_kernel_launches;
   if (persistent_launches) *persistent_launches = c->n_persistent_launches;

@@ -36,8 +36,8 @@ constexpr int N_FRAME_INPUTS = 4;
 constexpr int GEMM_BM = 128;   // output features per GEMM tile (the MMA M dimension)
 constexpr int GEMM_BK = 64;    // K elements per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int WORKER_THREADS = 128;
-constexpr int GEMM_MAX_BT = 256;     // most tokens per GEMM tile (MMA N)
-constexpr int GEMM_SMEM_BUDGET = 80 * 1024;  // stage memory a GEMM tile aims for (at least two stages are always taken)
+constexpr int GEMM_MAX_BT = 128;     // most tokens per GEMM tile (MMA N)
+constexpr int GEMM_SMEM_BUDGET = 64 * 1024;  // stage memory a GEMM tile aims for (at least two stages are always taken)
 
 struct GemmArgs {
   Ref A, W, W2;        // A bf16 [M,lda]; W (and W2 when dual) bf16 [N,Kp]
@@ -125,12 +125,13 @@ struct NodeDesc {
 // Per-class static description used by the pick.
 struct ClassInfo {
   int32_t tau[3];       // (TC, ALU, MEM) intensity 0..15
-  int32_t smem_units;   // shared-memory need in SMEM_UNIT chunks
-  int32_t tmem_units;   // tensor-memory need in TMEM_UNIT column chunks
-  int32_t pad[3];
+  int32_t smem_units;   // smallest shared-memory need of the class's tiles, in SMEM_UNIT chunks
+  int32_t tmem_units;   // smallest tensor-memory need, in TMEM_UNIT column chunks
+  int32_t group;        // pick group (the phase: tiles of one stream)
+  int32_t pad[2];
 };
 
-constexpr int SMEM_UNIT = 8192;
+constexpr int SMEM_UNIT = 4096;
 constexpr int TMEM_UNIT = 32;
 
 // A multi-producer multi-consumer ring of tile tickets (one per class).
