@@ -106,7 +106,7 @@ typedef struct {
   uint32_t tile;            /* tile index inside the node */
   uint16_t sm;              /* %smid */
   uint8_t worker;           /* worker group on that SM (0 in the ordinary-kernel modes) */
-  uint8_t cls;              /* tile class: phase * 3 + kind */
+  uint8_t cls;              /* tile class: phase * 4 + kind (GEMM, gated GEMM, attention, elementwise) */
   uint64_t frame;           /* frame id the tile belonged to */
   uint64_t t_start, t_end;  /* %globaltimer, ns */
 } vla_trace_rec;

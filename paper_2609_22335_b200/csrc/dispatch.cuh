@@ -7,7 +7,7 @@
 namespace vla {
 
 constexpr unsigned CTRL_EXITING = 0x80000000u;
-constexpr int MAX_WORKERS = 4;
+constexpr int MAX_WORKERS = 3;
 constexpr int SM_STATE_BYTES = 2048;
 
 __device__ __forceinline__ uint64_t gtimer() {
@@ -112,30 +112,43 @@ __device__ inline bool queue_try_pop(const DeviceCtx& ctx, int cls, QueueEntry& 
 
 // ------------------------------------------------------------------ per-SM state of the persistent kernel
 constexpr int MAX_READY = 6;
+constexpr int DISPATCH_THREADS = 64;     // two service warps per SM (claim, retire), after the worker groups
+constexpr int PREFETCH_MIN_AVAIL = 296;  // a busy worker's next tile is fetched early only from queues this deep
+
 struct ReadyItem {
   unsigned long long base;   // reserved queue range
   uint32_t node;
   int n_tiles, cls;
 };
-struct WorkerCmd {
-  int kind;            // 0 run, 1 exit
+
+struct WorkerTile {
   uint32_t inst, node, tile;
   int cls;
   int smem_unit0, smem_units, tmem_unit0, tmem_units;
-  int n_ready;         // successors released by the tile just finished (filled by the leader)
+  uint64_t t0, t1, frame;
+};
+
+// Mailboxes between one worker group and the SM's dispatcher warp (all in shared memory).
+struct WorkerSlot {
+  volatile int mail_state;   // 0 empty, 1 tile ready, 2 leave
+  volatile int done_state;   // 0 empty, 1 finished tile posted
+  volatile int busy;         // a tile is assigned (set at hand-over by the claim warp, cleared by the retire warp)
+  int held_valid;            // claim warp: a claimed tile waits for the worker and for room
+  WorkerTile mail, done, held, fin;
+  int n_ready;
   ReadyItem ready[MAX_READY];
 };
 
 struct SmState {
-  unsigned lock;
   unsigned long long smem_mask;    // bit i set = shared-memory unit i in use
   unsigned tmem_mask;              // bit i set = tensor-memory unit i in use
   int n_smem_units, n_tmem_units;
   PickState pick;
-  int waiter;                      // worker holding a tile while it waits for room (-1: none)
   unsigned tmem_base;
-  unsigned long long tiles;        // tiles this SM ran (added to the global counter at exit)
-  WorkerCmd cur[MAX_WORKERS];
+  int waiter;                      // worker whose claimed tile is waiting for room (-1: none); others then admit only memory-free tiles
+  volatile int quit;               // claim warp -> retire warp: everyone is leaving
+  WorkerTile cur[MAX_WORKERS];     // the tile each worker is running (written by its leader)
+  WorkerSlot slot[MAX_WORKERS];
 };
 static_assert(sizeof(SmState) <= SM_STATE_BYTES, "SM state too large");
 
@@ -147,37 +160,6 @@ __device__ __forceinline__ int find_free(unsigned long long mask, int need, int 
   for (int i = 0; i + need <= total; ++i)
     if (((mask >> i) & want) == 0) return i;
   return -1;
-}
-
-// Tile finished: bump the node's counter; the last tile of a node releases its successors.
-// Released successors get their queue range reserved here and are returned in `cmd->ready`
-// (the whole worker then fills the entries); without `cmd` they are pushed on the spot.
-__device__ inline void complete_tile(const DeviceCtx& ctx, uint32_t inst, uint32_t node_idx, bool persistent, WorkerCmd* cmd) {
-  const NodeDesc& n = ctx.nodes[node_idx];
-  if (cmd) cmd->n_ready = 0;
-  __threadfence();
-  int* cnt = ctx.tiles_done + (size_t)inst * ctx.n_nodes + node_idx;
-  int done = atomicAdd(cnt, 1) + 1;
-  if (done != n.n_tiles) return;
-  __threadfence();
-  *cnt = 0;
-  for (int i = 0; i < n.succ_count; ++i) {
-    int s = ctx.succ[n.succ_begin + i];
-    int* dep = ctx.dep_count + (size_t)inst * ctx.n_nodes + s;
-    int left = atomicSub(dep, 1) - 1;
-    if (left == 0) {
-      const NodeDesc& sn = ctx.nodes[s];
-      *dep = sn.n_pred;
-      if (cmd && cmd->n_ready < MAX_READY) {
-        ReadyItem& it = cmd->ready[cmd->n_ready++];
-        it.base = queue_reserve(ctx, sn.cls, sn.n_tiles);
-        it.node = (uint32_t)s; it.n_tiles = sn.n_tiles; it.cls = sn.cls;
-      } else {
-        queue_push(ctx, sn.cls, inst, (uint32_t)s, sn.n_tiles);
-      }
-    }
-  }
-  if (persistent && n.op == OP_EMIT) atomicSub(&ctx.control->ctrl, 1u);
 }
 
 __device__ inline void write_trace(const DeviceCtx& ctx, uint32_t inst, uint32_t node, uint32_t tile, int worker, int cls,
@@ -220,108 +202,244 @@ __device__ inline void try_admit(const DeviceCtx& ctx) {
   }
 }
 
-// Leader of a worker: find the next tile for this worker under the pick policy.
-// Feasibility is tested with each class's smallest footprint; the tile actually claimed is then
-// given its exact shared-memory and tensor-memory need.  If that does not fit yet, the worker keeps
-// the tile and waits (bounded) for co-resident tiles to finish; meanwhile it is the SM's only
-// "waiter" and the other workers admit nothing that needs shared or tensor memory.
-__device__ inline bool try_pick(const DeviceCtx& ctx, SmState* sm, int worker, uint64_t deadline) {
-  unsigned pending = 0;
-  for (int c = 0; c < N_CLASSES; ++c)
-    if (ld_volatile_s64(&ctx.queues[c].avail) > 0) pending |= 1u << c;
-  if (pending == 0) return false;
-  unsigned spins = 0;
-  while (atomicCAS(&sm->lock, 0u, 1u) != 0u) {
-    __nanosleep(32);
-    if ((++spins & 255u) == 0 && gtimer() > deadline) return false;
+// Global side of a finished tile: bump the node's counter; the last tile of a node releases its
+// successors, whose queue ranges are reserved here and returned in `slot` for the warp to fill.
+__device__ inline void complete_tile(const DeviceCtx& ctx, uint32_t inst, uint32_t node_idx, WorkerSlot* slot) {
+  const NodeDesc& n = ctx.nodes[node_idx];
+  slot->n_ready = 0;
+  __threadfence();
+  int* cnt = ctx.tiles_done + (size_t)inst * ctx.n_nodes + node_idx;
+  int done = atomicAdd(cnt, 1) + 1;
+  if (done != n.n_tiles) return;
+  __threadfence();
+  *cnt = 0;
+  for (int i = 0; i < n.succ_count; ++i) {
+    int s = ctx.succ[n.succ_begin + i];
+    int* dep = ctx.dep_count + (size_t)inst * ctx.n_nodes + s;
+    int left = atomicSub(dep, 1) - 1;
+    if (left == 0) {
+      const NodeDesc& sn = ctx.nodes[s];
+      *dep = sn.n_pred;
+      if (slot->n_ready < MAX_READY) {
+        ReadyItem& it = slot->ready[slot->n_ready++];
+        it.base = queue_reserve(ctx, sn.cls, sn.n_tiles);
+        it.node = (uint32_t)s; it.n_tiles = sn.n_tiles; it.cls = sn.cls;
+      } else {
+        queue_push(ctx, sn.cls, inst, (uint32_t)s, sn.n_tiles);
+      }
+    }
   }
-  bool got = false;
+  if (n.op == OP_EMIT) atomicSub(&ctx.control->ctrl, 1u);
+}
+
+// ------------------------------------------------------------------ the two service warps of an SM
+// Workers never touch global queues or counters.  Two extra warps per SM do it for them, so those
+// round trips overlap tile execution instead of sitting between tiles:
+//   * the CLAIM warp (lane w serves worker w) claims tiles under the pick policy -- for a busy worker one
+//     tile ahead -- and hands a claimed tile over as soon as its worker is free and its exact
+//     shared/tensor-memory need fits;
+//   * the RETIRE warp (lane w serves worker w) takes a finished tile, frees its memory at once, then does
+//     the global bookkeeping (node counter, successors' dependency counters, queue pushes; the whole warp
+//     fills the released successors' entries).
+// Per-SM state is shared-memory words updated with shared-memory atomics by these two warps only.
+__device__ inline void retire_loop(const DeviceCtx& ctx, SmState* sm, int n_workers) {
+  const int lane = threadIdx.x & 31;
+  const bool serving = lane < n_workers;
+  WorkerSlot* slot = sm->slot + (serving ? lane : 0);
+  int tau[N_CLASSES * 3];
+  for (int c = 0; c < N_CLASSES; ++c)
+    for (int x = 0; x < 3; ++x) tau[c * 3 + x] = ctx.classes[c].tau[x];
+  unsigned nap = 40;
+  for (;;) {
+    bool have_fin = false;
+    if (serving && slot->done_state == 1) {
+      slot->fin = slot->done;
+      __threadfence_block();
+      slot->done_state = 0;
+      have_fin = true;
+      const WorkerTile& f = slot->fin;
+      if (f.smem_units) atomicAnd(&sm->smem_mask, ~(unit_bits(f.smem_units) << f.smem_unit0));
+      if (f.tmem_units) atomicAnd(&sm->tmem_mask, ~(unsigned)(unit_bits(f.tmem_units) << f.tmem_unit0));
+      atomicSub(&sm->pick.cta_count[f.cls], 1);
+      for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[f.cls * 3 + x]);
+      __threadfence_block();
+      slot->busy = 0;
+      write_trace(ctx, f.inst, f.node, f.tile, lane, f.cls, f.frame, f.t0, f.t1);
+      complete_tile(ctx, f.inst, f.node, slot);
+    } else if (serving) {
+      slot->n_ready = 0;
+    }
+    __syncwarp();
+    const bool any = __any_sync(0xffffffffu, have_fin);
+    if (any) {
+      for (int w = 0; w < n_workers; ++w) {
+        const int nr = sm->slot[w].n_ready;
+        for (int i = 0; i < nr; ++i) {
+          const ReadyItem it = sm->slot[w].ready[i];
+          queue_fill(ctx, it.cls, it.base, sm->slot[w].fin.inst, it.node, lane, it.n_tiles, 32);
+        }
+      }
+      __syncwarp();
+      if (serving) {
+        for (int i = 0; i < slot->n_ready; ++i) queue_commit(ctx, slot->ready[i].cls, slot->ready[i].n_tiles);
+        slot->n_ready = 0;
+      }
+      __syncwarp();
+      nap = 40;
+    } else {
+      if (sm->quit) break;
+      __nanosleep(nap);
+      if (nap < 400) nap += 40;
+    }
+  }
+}
+
+__device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_workers) {
+  const int lane = threadIdx.x & 31;
+  const bool serving = lane < n_workers;
+  Control* ctl = ctx.control;
+  WorkerSlot* slot = sm->slot + (serving ? lane : 0);
   int tau[N_CLASSES * 3], group[N_CLASSES];
   for (int c = 0; c < N_CLASSES; ++c) {
     for (int x = 0; x < 3; ++x) tau[c * 3 + x] = ctx.classes[c].tau[x];
     group[c] = ctx.classes[c].group;
   }
-  const bool blocked = sm->waiter >= 0 && sm->waiter != worker;
-  WorkerCmd& cmd = sm->cur[worker];
-  for (int attempt = 0; attempt < N_CLASSES && pending; ++attempt) {
-    unsigned feasible = 0;
-    for (int c = 0; c < N_CLASSES; ++c) {
-      const int su = ctx.classes[c].smem_units, tu = ctx.classes[c].tmem_units;
-      if (blocked && (su > 0 || tu > 0)) continue;
-      if (find_free(sm->smem_mask, su, sm->n_smem_units) >= 0 && find_free(sm->tmem_mask, tu, sm->n_tmem_units) >= 0)
-        feasible |= 1u << c;
-    }
-    int phase;
-    int k = pick_choose(N_CLASSES, tau, group, pending, feasible, sm->pick, sm->pick.rr, ctx.policy, &phase);
-    if (k < 0) break;
-    QueueEntry e;
-    if (!queue_try_pop(ctx, k, e, deadline)) {
-      pending &= ~(1u << k);
-      continue;
-    }
-    cmd.kind = 0;
-    cmd.inst = e.inst_node >> 20;
-    cmd.node = e.inst_node & 0xFFFFFu;
-    cmd.tile = e.tile;
-    cmd.cls = k;
-    const NodeDesc& nd = ctx.nodes[cmd.node];
-    cmd.smem_units = (nd.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT;
-    cmd.tmem_units = (nd.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT;
-    pick_commit(sm->pick, k, tau);
-    sm->pick.rr = (k + 1) % N_CLASSES;
-    got = true;
-    break;
-  }
-  if (got) {
-    // exact allocation; hold the tile and wait when the SM is too full right now
-    for (;;) {
-      cmd.smem_unit0 = find_free(sm->smem_mask, cmd.smem_units, sm->n_smem_units);
-      cmd.tmem_unit0 = find_free((unsigned long long)sm->tmem_mask, cmd.tmem_units, sm->n_tmem_units);
-      if (cmd.smem_unit0 >= 0 && cmd.tmem_unit0 >= 0) break;
-      sm->waiter = worker;
-      __threadfence_block();
-      atomicExch(&sm->lock, 0u);
-      __nanosleep(200);
-      if (gtimer() > deadline || ld_volatile_u32(&ctx.control->error) != 0u) {
-        set_error(ctx, DEV_ERR_IDLE_LIMIT, 0x1000u + (unsigned)blockIdx.x);
-        cmd.kind = 1;
-        return true;    // leave: kind = exit
-      }
-      while (atomicCAS(&sm->lock, 0u, 1u) != 0u) __nanosleep(32);
-    }
-    if (sm->waiter == worker) sm->waiter = -1;
-    if (cmd.smem_units) sm->smem_mask |= unit_bits(cmd.smem_units) << cmd.smem_unit0;
-    if (cmd.tmem_units) sm->tmem_mask |= (unsigned)(unit_bits(cmd.tmem_units) << cmd.tmem_unit0);
-  }
-  __threadfence_block();
-  atomicExch(&sm->lock, 0u);
-  return got;
-}
+  uint64_t idle_start = 0, last_progress = gtimer();
+  unsigned iter = 0, nap = 60;
+  bool leaving = false;
 
-__device__ inline void release_resources(const DeviceCtx& ctx, SmState* sm, const WorkerCmd& cmd) {
-  while (atomicCAS(&sm->lock, 0u, 1u) != 0u) __nanosleep(32);
-  if (cmd.smem_units) sm->smem_mask &= ~(unit_bits(cmd.smem_units) << cmd.smem_unit0);
-  if (cmd.tmem_units) sm->tmem_mask &= ~(unsigned)(unit_bits(cmd.tmem_units) << cmd.tmem_unit0);
-  int tau[3] = {ctx.classes[cmd.cls].tau[0], ctx.classes[cmd.cls].tau[1], ctx.classes[cmd.cls].tau[2]};
-  sm->pick.cta_count[cmd.cls] -= 1;
-  for (int x = 0; x < 3; ++x) sm->pick.u[x] -= tau[x];
-  sm->tiles += 1;
-  __threadfence_block();
-  atomicExch(&sm->lock, 0u);
+  for (;;) {
+    ++iter;
+    bool progressed = false;
+    long long av = lane < N_CLASSES ? ld_volatile_s64(&ctx.queues[lane].avail) : 0;
+    const unsigned pending = __ballot_sync(0xffffffffu, av > 0) & ((1u << N_CLASSES) - 1u);
+    const unsigned deep = __ballot_sync(0xffffffffu, av >= PREFETCH_MIN_AVAIL) & ((1u << N_CLASSES) - 1u);
+    // ---- choose, lane by lane, which class each worker claims from
+    int want = -1;
+    for (int w = 0; w < n_workers; ++w) {
+      if (lane == w && !leaving && !slot->held_valid) {
+        const bool busy = slot->busy != 0;
+        const unsigned cand = busy ? (deep & ((1u << N_KINDS) - 1u)) : pending;   // early claims only from deep VLM queues
+        const unsigned long long smask = *reinterpret_cast<volatile unsigned long long*>(&sm->smem_mask);
+        const unsigned tmask = *reinterpret_cast<volatile unsigned*>(&sm->tmem_mask);
+        const bool blocked = sm->waiter >= 0 && sm->waiter != w;
+        unsigned feasible = 0;
+        for (int c = 0; c < N_CLASSES; ++c) {
+          const int su = ctx.classes[c].smem_units, tu = ctx.classes[c].tmem_units;
+          if (busy) { feasible |= 1u << c; continue; }
+          if (blocked && (su > 0 || tu > 0)) continue;
+          if (find_free(smask, su, sm->n_smem_units) >= 0 && find_free((unsigned long long)tmask, tu, sm->n_tmem_units) >= 0)
+            feasible |= 1u << c;
+        }
+        PickState ps;
+        for (int c = 0; c < N_CLASSES; ++c) ps.cta_count[c] = *reinterpret_cast<volatile int*>(&sm->pick.cta_count[c]);
+        for (int x = 0; x < 3; ++x) ps.u[x] = *reinterpret_cast<volatile int*>(&sm->pick.u[x]);
+        int phase;
+        want = pick_choose(N_CLASSES, tau, group, cand, feasible, ps, sm->pick.rr, ctx.policy, &phase);
+        if (want >= 0) {
+          atomicAdd(&sm->pick.cta_count[want], 1);     // counted from the claim on, so the next lane sees it
+          for (int x = 0; x < 3; ++x) atomicAdd(&sm->pick.u[x], tau[want * 3 + x]);
+          sm->pick.rr = (want + 1) % N_CLASSES;
+        }
+      }
+      __syncwarp();
+    }
+    // ---- the claims themselves run in parallel across lanes (global atomics)
+    if (want >= 0) {
+      QueueEntry e;
+      if (queue_try_pop(ctx, want, e, gtimer() + ctx.wait_limit_ns)) {
+        WorkerTile& h = slot->held;
+        h.inst = e.inst_node >> 20; h.node = e.inst_node & 0xFFFFFu; h.tile = e.tile; h.cls = want;
+        const NodeDesc& nd = ctx.nodes[h.node];
+        h.smem_units = (nd.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT;
+        h.tmem_units = (nd.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT;
+        slot->held_valid = 1;
+        progressed = true;
+      } else {                                         // lost the race: undo the count
+        atomicSub(&sm->pick.cta_count[want], 1);
+        for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[want * 3 + x]);
+      }
+    }
+    // ---- hand the held tile over when the worker is free and the tile's exact need fits
+    for (int w = 0; w < n_workers; ++w) {
+      if (lane == w && slot->held_valid && slot->busy == 0 && slot->mail_state == 0) {
+        WorkerTile& h = slot->held;
+        const bool needs_mem = h.smem_units > 0 || h.tmem_units > 0;
+        const bool yield = needs_mem && sm->waiter >= 0 && sm->waiter != w;   // an older claim is waiting for room
+        const unsigned long long smask = *reinterpret_cast<volatile unsigned long long*>(&sm->smem_mask);
+        const unsigned tmask = *reinterpret_cast<volatile unsigned*>(&sm->tmem_mask);
+        int s0 = yield ? -1 : find_free(smask, h.smem_units, sm->n_smem_units);
+        int t0 = yield ? -1 : find_free((unsigned long long)tmask, h.tmem_units, sm->n_tmem_units);
+        if (!yield && (s0 < 0 || t0 < 0)) sm->waiter = w;
+        if (s0 >= 0 && t0 >= 0) {
+          if (sm->waiter == w) sm->waiter = -1;
+          h.smem_unit0 = s0; h.tmem_unit0 = t0;
+          if (h.smem_units) atomicOr(&sm->smem_mask, unit_bits(h.smem_units) << s0);
+          if (h.tmem_units) atomicOr(&sm->tmem_mask, (unsigned)(unit_bits(h.tmem_units) << t0));
+          slot->mail = h;
+          slot->busy = 1;
+          __threadfence_block();
+          slot->mail_state = 1;
+          slot->held_valid = 0;
+          progressed = true;
+        }
+      }
+      __syncwarp();
+    }
+    // ---- admission, exit and watchdog (lane 0 decides, every few rounds)
+    int verdict = 0;   // 1 = leave
+    if (lane == 0 && ((iter & 7u) == 0 || !progressed)) {
+      if (ld_volatile_u32(&ctl->error) != 0u || ld_volatile_u32(&ctl->stop) != 0u) verdict = 1;
+      const unsigned cw = ld_volatile_u32(&ctl->ctrl);
+      if (cw & CTRL_EXITING) verdict = 1;
+      if (!verdict) {
+        try_admit(ctx);
+        const uint64_t now = gtimer();
+        const bool none = cw == 0u && ld_volatile_u64(&ctl->admit_head) >= ld_volatile_u64(&ctl->admit_tail);
+        if (none) {
+          if (idle_start == 0) idle_start = now;
+          else if (now - idle_start > ctx.idle_exit_ns) atomicCAS(&ctl->ctrl, 0u, CTRL_EXITING);
+        } else {
+          idle_start = 0;
+        }
+      }
+    }
+    const bool any_progress = __any_sync(0xffffffffu, progressed || (serving && slot->busy != 0));
+    if (any_progress) last_progress = gtimer();
+    else if (lane == 0 && !verdict && (iter & 63u) == 0 && gtimer() - last_progress > ctx.wait_limit_ns &&
+             ld_volatile_u32(&ctl->ctrl) != 0u) {
+      set_error(ctx, DEV_ERR_IDLE_LIMIT, (unsigned)blockIdx.x);   // frames in flight, nothing moved for too long
+      verdict = 1;
+    }
+    verdict = __shfl_sync(0xffffffffu, verdict, 0);
+    if (verdict) leaving = true;
+    if (leaving) {
+      // stop claiming; once every worker is idle and nothing is posted, send them home
+      const bool quiet = !serving || (slot->busy == 0 && slot->done_state == 0 && slot->mail_state == 0);
+      if (__all_sync(0xffffffffu, quiet)) {
+        if (serving) { __threadfence_block(); slot->mail_state = 2; }
+        __syncwarp();
+        if (lane == 0) { __threadfence_block(); sm->quit = 1; }
+        break;
+      }
+    }
+    if (!__any_sync(0xffffffffu, progressed)) { __nanosleep(nap); if (nap < 600) nap += 60; } else nap = 60;
+  }
 }
 
 // ------------------------------------------------------------------ the persistent co-scheduling kernel
-// One CTA per SM; MAX_WORKERS worker groups of WORKER_THREADS threads.  Each worker's
-// first thread is its leader: it admits ready frames, picks a tile, and after the tile
-// has run resolves dependencies.  Every wait is bounded by ctx.wait_limit_ns.
-__global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_kernel(DeviceCtx ctx, int dyn_smem_bytes) {
+// One CTA per SM: `workers` worker groups of WORKER_THREADS threads run tiles; one more warp is the
+// dispatcher.  Every wait is bounded by ctx.wait_limit_ns.
+__global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS, 1)
+    vla_cosched_kernel(DeviceCtx ctx, int dyn_smem_bytes) {
   extern __shared__ __align__(1024) char smem_raw[];
   SmState* sm = reinterpret_cast<SmState*>(smem_raw);
   char* slab = smem_raw + SM_STATE_BYTES;
+  const int n_workers = (blockDim.x - DISPATCH_THREADS) / WORKER_THREADS;
+  const bool is_dispatcher = threadIdx.x >= n_workers * WORKER_THREADS;
   const int worker = threadIdx.x / WORKER_THREADS;
   const int wt = threadIdx.x % WORKER_THREADS;
   if (threadIdx.x == 0) {
-    sm->lock = 0;
     sm->smem_mask = 0;
     sm->tmem_mask = 0;
     int units = (dyn_smem_bytes - SM_STATE_BYTES) / SMEM_UNIT;
@@ -332,7 +450,11 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_ke
     sm->pick.rr = (int)(blockIdx.x % N_CLASSES);
     sm->tmem_base = 0;
     sm->waiter = -1;
-    sm->tiles = 0;
+    sm->quit = 0;
+    for (int w = 0; w < MAX_WORKERS; ++w) {
+      sm->slot[w].mail_state = 0; sm->slot[w].done_state = 0; sm->slot[w].busy = 0; sm->slot[w].held_valid = 0;
+      sm->slot[w].n_ready = 0;
+    }
   }
   __syncthreads();
   if (threadIdx.x < 32) tmem_alloc(&sm->tmem_base, 512);   // the whole tensor memory of this SM, sub-allocated per tile
@@ -340,103 +462,69 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS, 1) vla_cosched_ke
   __syncthreads();
   tc_fence_after();
   Control* ctl = ctx.control;
-  const int bar_id = worker + 1;
 
-  for (;;) {
-    if (wt == 0) {
-      WorkerCmd& cmd = sm->cur[worker];
-      const uint64_t wait_start = gtimer();
-      uint64_t idle_start = 0;
-      unsigned backoff = 64, polls = 0;
-      unsigned long long bell_seen = ~0ull;
-      cmd.kind = 1;
-      for (;;) {
-        // An idle leader polls one word (the doorbell); the queues are scanned only when it moved.
-        const unsigned long long bell = ld_volatile_u64(&ctl->doorbell);
-        const bool slow = (polls++ & 15u) == 0;
-        if (slow) {
-          if (ld_volatile_u32(&ctl->error) != 0u || ld_volatile_u32(&ctl->stop) != 0u) break;
-          if (ld_volatile_u32(&ctl->ctrl) & CTRL_EXITING) break;
-          try_admit(ctx);
+  if (is_dispatcher) {
+    if (threadIdx.x < n_workers * WORKER_THREADS + 32) claim_loop(ctx, sm, n_workers);
+    else retire_loop(ctx, sm, n_workers);
+  } else {
+    const int bar_id = worker + 1;
+    WorkerSlot* slot = sm->slot + worker;
+    unsigned long long tiles = 0;
+    for (;;) {
+      if (wt == 0) {
+        int st;
+        unsigned naps = 0;
+        while ((st = slot->mail_state) == 0) { __nanosleep(naps < 64 ? 20 : 200); ++naps; }
+        if (st == 1) {
+          sm->cur[worker] = slot->mail;
+          sm->cur[worker].t0 = 1;            // marks "run"
+          __threadfence_block();
+          slot->mail_state = 0;
+        } else {
+          sm->cur[worker].t0 = 0;            // marks "leave"
         }
-        if (bell != bell_seen || slow) {
-          bell_seen = bell;
-#ifdef VLA_TILE_TIMING
-          const uint64_t tp0 = gtimer();
-          const bool hit = try_pick(ctx, sm, worker, wait_start + ctx.wait_limit_ns);
-          atomicAdd(ctl->dbg + (hit ? 5 : 7), gtimer() - tp0); atomicAdd(ctl->dbg + (hit ? 6 : 8), 1ull);
-          if (hit) break;
-#else
-          if (try_pick(ctx, sm, worker, wait_start + ctx.wait_limit_ns)) break;   // cmd.kind = 0 now
-#endif
-        }
-        if (slow) {
-          const uint64_t now = gtimer();
-          const unsigned cw = ld_volatile_u32(&ctl->ctrl);
-          if (cw & CTRL_EXITING) break;
-          const bool none = cw == 0u && ld_volatile_u64(&ctl->admit_head) >= ld_volatile_u64(&ctl->admit_tail);
-          if (none) {
-            if (idle_start == 0) idle_start = now;
-            else if (now - idle_start > ctx.idle_exit_ns) atomicCAS(&ctl->ctrl, 0u, CTRL_EXITING);
-          } else {
-            idle_start = 0;
-            if (now - wait_start > ctx.wait_limit_ns) {   // frames in flight but nothing runnable for too long
-              set_error(ctx, DEV_ERR_IDLE_LIMIT, (unsigned)blockIdx.x);
-              break;
-            }
-          }
-        }
-        __nanosleep(backoff);
-        if (backoff < 2048) backoff <<= 1;
-      }
-    }
-    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
-    const WorkerCmd cmd = sm->cur[worker];
-    if (cmd.kind != 0) break;
-    const NodeDesc& n = ctx.nodes[cmd.node];
-    TileCtx tc;
-    tc.arena = ctx.arena;
-    tc.slot_base = ctx.slot_base[cmd.inst];
-    tc.smem = slab + (size_t)cmd.smem_unit0 * SMEM_UNIT;
-    tc.tmem = sm->tmem_base + (unsigned)cmd.tmem_unit0 * TMEM_UNIT;
-    tc.tid = wt;
-    tc.bar_id = bar_id;
-    tc.error = &ctl->error;
-    tc.tmaps = ctx.tmaps;
-    tc.dbg = ctl->dbg;
-    tc.inputs = ctx.input_ptrs + (size_t)cmd.inst * N_FRAME_INPUTS;
-    tc.amap_base = ctx.n_weight_tmaps + (int)cmd.inst * ctx.n_act_tmaps;
-    const uint64_t t0 = gtimer();
-    tc.deadline = t0 + ctx.wait_limit_ns;
-    const uint64_t frame = *reinterpret_cast<const volatile uint64_t*>(ctx.inst_frame + cmd.inst);
-    run_tile(ctx, tc, n, (int)cmd.tile, (int)cmd.inst, frame);
-    asm volatile("fence.proxy.async;" ::: "memory");   // outputs may be read by TMA on another SM
-    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
-    if (wt == 0) {
-      const uint64_t t1 = gtimer();
-      write_trace(ctx, cmd.inst, cmd.node, cmd.tile, worker, cmd.cls, frame, t0, t1);
-      release_resources(ctx, sm, cmd);
-      complete_tile(ctx, cmd.inst, cmd.node, true, &sm->cur[worker]);
-#ifdef VLA_TILE_TIMING
-      atomicAdd(ctl->dbg + 9, gtimer() - t1); atomicAdd(ctl->dbg + 10, 1ull);
-#endif
-    }
-    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
-    const int n_ready = sm->cur[worker].n_ready;
-    if (n_ready > 0) {
-      for (int i = 0; i < n_ready; ++i) {
-        const ReadyItem it = sm->cur[worker].ready[i];
-        queue_fill(ctx, it.cls, it.base, cmd.inst, it.node, wt, it.n_tiles, WORKER_THREADS);
       }
       asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
-      if (wt == 0)
-        for (int i = 0; i < n_ready; ++i) queue_commit(ctx, sm->cur[worker].ready[i].cls, sm->cur[worker].ready[i].n_tiles);
+      const WorkerTile cmd = sm->cur[worker];
+      if (cmd.t0 == 0) break;
+      const NodeDesc& n = ctx.nodes[cmd.node];
+      TileCtx tc;
+      tc.arena = ctx.arena;
+      tc.slot_base = ctx.slot_base[cmd.inst];
+      tc.smem = slab + (size_t)cmd.smem_unit0 * SMEM_UNIT;
+      tc.tmem = sm->tmem_base + (unsigned)cmd.tmem_unit0 * TMEM_UNIT;
+      tc.tid = wt;
+      tc.bar_id = bar_id;
+      tc.error = &ctl->error;
+      tc.tmaps = ctx.tmaps;
+      tc.dbg = ctl->dbg;
+      tc.inputs = ctx.input_ptrs + (size_t)cmd.inst * N_FRAME_INPUTS;
+      tc.amap_base = ctx.n_weight_tmaps + (int)cmd.inst * ctx.n_act_tmaps;
+      const uint64_t t0 = gtimer();
+      tc.deadline = t0 + ctx.wait_limit_ns;
+      const uint64_t frame = *reinterpret_cast<const volatile uint64_t*>(ctx.inst_frame + cmd.inst);
+      run_tile(ctx, tc, n, (int)cmd.tile, (int)cmd.inst, frame);
+      asm volatile("fence.proxy.async;" ::: "memory");   // outputs may be read by TMA on another SM
+      asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
+      if (wt == 0) {
+        ++tiles;
+        unsigned naps = 0;
+        while (slot->done_state != 0) {
+          __nanosleep(40);
+          if ((++naps & 0xFFFFu) == 0 && gtimer() - t0 > 2 * ctx.wait_limit_ns) break;   // dispatcher gone: give up posting
+        }
+        WorkerTile d = cmd;
+        d.t0 = t0; d.t1 = gtimer(); d.frame = frame;
+        slot->done = d;
+        __threadfence();       // the tile's writes (all threads, ordered by the barrier) before the completion is seen
+        slot->done_state = 1;
+      }
     }
+    if (wt == 0) atomicAdd(&ctl->tiles_done, tiles);
   }
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x < 32) tmem_dealloc(sm->tmem_base, 512);
-  if (threadIdx.x == 0) atomicAdd(&ctl->tiles_done, sm->tiles);
 }
 
 // ------------------------------------------------------------------ one node as an ordinary kernel (CTA = tile)

@@ -171,7 +171,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       ok = mbar_wait(c, full_bar(s), ph);
       if (!ok) break;
 #ifdef VLA_TILE_TIMING
-      if (kb == 0 && g.M > 512) { uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); atomicAdd(c.dbg + 0, t - tt0); }
+      if (kb == 0 && g.M > 512 && c.dbg) { uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); atomicAdd(c.dbg + 0, t - tt0); }
 #endif
       tc_fence_after();
       const uint32_t wsm = stage0 + (uint32_t)(s * stage_bytes);
@@ -221,7 +221,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   tc_fence_before();
   worker_sync(c);
 #ifdef VLA_TILE_TIMING
-  if (c.tid == 64 && g.M > 512) {
+  if (c.tid == 64 && g.M > 512 && c.dbg) {
     uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     atomicAdd(c.dbg + 1, tt1 - tt0); atomicAdd(c.dbg + 2, t - tt1); atomicAdd(c.dbg + 3, 1ull); atomicAdd(c.dbg + 4, (unsigned long long)nkb);
   }

@@ -172,7 +172,7 @@ class Builder {
   int add(NodeDesc n, const std::string& name, int kind) {
     n.phase = phase;
     n.step = step;
-    n.cls = phase * 3 + kind;
+    n.cls = phase * N_KINDS + kind;
     n.n_pred = 0;
     n.succ_begin = n.succ_count = 0;
     if (init_mode) {
@@ -232,7 +232,7 @@ class Builder {
       g.amap = act_map(A, g.Kp, bt);
     }
     n.n_tiles = (int)((g.N + GEMM_BM - 1) / GEMM_BM) * tiles_t;
-    int id = add(n, name, KIND_GEMM);
+    int id = add(n, name, g.dual ? KIND_GEMM2 : KIND_GEMM);
     read(id, A);
     if (o.X.buf >= 0) read(id, o.X);
     if (o.out32.buf >= 0) write(id, o.out32);
@@ -891,23 +891,19 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   // ================================================================== per-class tags and resources
   // (tau_TC, tau_ALU, tau_MEM): hand-assigned intensities per tile class (Section 3.2 of the paper
   // derives them by profiling; the values below follow the per-class roofline of the tile bodies).
-  const int taus[N_CLASSES][3] = {{15, 2, 3}, {8, 8, 2}, {0, 4, 10}, {2, 3, 12}, {1, 8, 4}, {0, 3, 6}};
+  const int taus[N_CLASSES][3] = {{15, 2, 3}, {15, 4, 3}, {8, 8, 2}, {0, 4, 10}, {2, 3, 12}, {2, 4, 12}, {1, 8, 4}, {0, 3, 6}};
   for (int c = 0; c < N_CLASSES; ++c) {
     for (int x_ = 0; x_ < 3; ++x_) p.classes[c].tau[x_] = taus[c][x_];
-    p.classes[c].smem_units = 1 << 20;
-    p.classes[c].tmem_units = 1 << 20;
-    p.classes[c].group = c / 3;
+    p.classes[c].smem_units = 0;
+    p.classes[c].tmem_units = 0;
+    p.classes[c].group = c / N_KINDS;
     p.classes[c].pad[0] = p.classes[c].pad[1] = 0;
   }
   for (const NodeDesc& n : p.nodes) {
     if (n.smem_bytes > 54 * SMEM_UNIT) { set_err(p, "a tile needs more shared memory than one SM offers"); return false; }
     ClassInfo& ci = p.classes[n.cls];
-    ci.smem_units = std::min(ci.smem_units, (n.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT);
-    ci.tmem_units = std::min(ci.tmem_units, (n.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT);
-  }
-  for (int c = 0; c < N_CLASSES; ++c) {
-    if (p.classes[c].smem_units == (1 << 20)) p.classes[c].smem_units = 0;
-    if (p.classes[c].tmem_units == (1 << 20)) p.classes[c].tmem_units = 0;
+    ci.smem_units = std::max(ci.smem_units, (n.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT);
+    ci.tmem_units = std::max(ci.tmem_units, (n.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT);
   }
 
   // ================================================================== arena layout

@@ -172,7 +172,7 @@ uint64_t count_phase_nodes(const Program& p, int phase_sel) {
 int launch_persistent(vla_ctx* c) {
   // reset the control word in stream order, then launch one CTA per SM
   CU(cudaMemcpyAsync(&c->dctx.control->ctrl, c->zero_pinned, sizeof(unsigned), cudaMemcpyHostToDevice, c->sa));
-  vla_cosched_kernel<<<c->sm_count, c->workers * WORKER_THREADS, c->dyn_smem, c->sa>>>(c->dctx, c->dyn_smem);
+  vla_cosched_kernel<<<c->sm_count, c->workers * WORKER_THREADS + DISPATCH_THREADS, c->dyn_smem, c->sa>>>(c->dctx, c->dyn_smem);
   CU(cudaGetLastError());
   CU(cudaEventRecord(c->ev_kernel, c->sa));
   c->kernel_launched = true;

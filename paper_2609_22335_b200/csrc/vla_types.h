@@ -18,9 +18,10 @@ enum Op : int32_t {
   OP_COUNT = 9
 };
 
-enum Kind : int32_t { KIND_GEMM = 0, KIND_ATTN = 1, KIND_ELEM = 2 };
+enum Kind : int32_t { KIND_GEMM = 0, KIND_GEMM2 = 1, KIND_ATTN = 2, KIND_ELEM = 3 };   // GEMM2: two accumulators (gated MLP)
+constexpr int N_KINDS = 4;
 enum Phase : int32_t { PHASE_VLM = 0, PHASE_ACT = 1 };
-constexpr int N_CLASSES = 6;  // phase * 3 + kind
+constexpr int N_CLASSES = 8;  // phase * N_KINDS + kind: one queue per resource shape and stream
 
 enum Act : int32_t { ACT_NONE = 0, ACT_GELU = 1, ACT_SILU = 2 };
 
@@ -125,8 +126,8 @@ struct NodeDesc {
 // Per-class static description used by the pick.
 struct ClassInfo {
   int32_t tau[3];       // (TC, ALU, MEM) intensity 0..15
-  int32_t smem_units;   // smallest shared-memory need of the class's tiles, in SMEM_UNIT chunks
-  int32_t tmem_units;   // smallest tensor-memory need, in TMEM_UNIT column chunks
+  int32_t smem_units;   // largest shared-memory need of the class's tiles, in SMEM_UNIT chunks (a claim must fit this)
+  int32_t tmem_units;   // largest tensor-memory need, in TMEM_UNIT column chunks
   int32_t group;        // pick group (the phase: tiles of one stream)
   int32_t pad[2];
 };
