@@ -113,7 +113,8 @@ __device__ inline bool queue_try_pop(const DeviceCtx& ctx, int cls, QueueEntry& 
 // ------------------------------------------------------------------ per-SM state of the persistent kernel
 constexpr int MAX_READY = 6;
 constexpr int DISPATCH_THREADS = 64;     // two service warps per SM (claim, retire), after the worker groups
-constexpr int PREFETCH_MIN_AVAIL = 296;  // a busy worker's next tile is fetched early only from queues this deep
+constexpr int PREFETCH_MIN_AVAIL = 64;   // tiles are claimed ahead of need only from queues at least this deep
+constexpr int HELD_DEPTH = 2;            // claimed tiles a worker may have waiting
 
 struct ReadyItem {
   unsigned long long base;   // reserved queue range
@@ -130,11 +131,13 @@ struct WorkerTile {
 
 // Mailboxes between one worker group and the SM's dispatcher warp (all in shared memory).
 struct WorkerSlot {
-  volatile int mail_state;   // 0 empty, 1 tile ready, 2 leave
-  volatile int done_state;   // 0 empty, 1 finished tile posted
-  volatile int busy;         // a tile is assigned (set at hand-over by the claim warp, cleared by the retire warp)
-  int held_valid;            // claim warp: a claimed tile waits for the worker and for room
-  WorkerTile mail, done, held, fin;
+  volatile unsigned held_tail;   // claimed tiles pushed by the claim warp (single producer)
+  volatile unsigned held_head;   // claimed tiles taken by the worker (single consumer)
+  volatile int leave;            // claim warp -> worker: go home
+  volatile int done_state;       // 0 empty, 1 finished tile posted for the retire warp
+  volatile int busy;             // the worker is running a tile (set and cleared by the worker)
+  int pad_;
+  WorkerTile done, fin, held[HELD_DEPTH];
   int n_ready;
   ReadyItem ready[MAX_READY];
 };
@@ -258,12 +261,6 @@ __device__ inline void retire_loop(const DeviceCtx& ctx, SmState* sm, int n_work
       slot->done_state = 0;
       have_fin = true;
       const WorkerTile& f = slot->fin;
-      if (f.smem_units) atomicAnd(&sm->smem_mask, ~(unit_bits(f.smem_units) << f.smem_unit0));
-      if (f.tmem_units) atomicAnd(&sm->tmem_mask, ~(unsigned)(unit_bits(f.tmem_units) << f.tmem_unit0));
-      atomicSub(&sm->pick.cta_count[f.cls], 1);
-      for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[f.cls * 3 + x]);
-      __threadfence_block();
-      slot->busy = 0;
       write_trace(ctx, f.inst, f.node, f.tile, lane, f.cls, f.frame, f.t0, f.t1);
       complete_tile(ctx, f.inst, f.node, slot);
     } else if (serving) {
@@ -317,12 +314,15 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     // ---- choose, lane by lane, which class each worker claims from
     int want = -1;
     for (int w = 0; w < n_workers; ++w) {
-      if (lane == w && !leaving && !slot->held_valid) {
-        const bool busy = slot->busy != 0;
-        const unsigned cand = busy ? (deep & ((1u << N_KINDS) - 1u)) : pending;   // early claims only from deep VLM queues
+      const unsigned queued = serving ? slot->held_tail - slot->held_head : 0u;
+      if (lane == w && !leaving && queued < (unsigned)HELD_DEPTH) {
+        const bool busy = slot->busy != 0 || queued > 0;   // anything beyond the first tile is claimed ahead of need
+        // early claims (for a worker that is still running) only from deep VLM queues, and never for worker 0:
+        // one worker per SM always returns to the pool, so a short action-head tile is at most one tile away
+        const unsigned cand = busy ? (w == 0 ? 0u : (deep & ((1u << N_KINDS) - 1u))) : pending;
         const unsigned long long smask = *reinterpret_cast<volatile unsigned long long*>(&sm->smem_mask);
         const unsigned tmask = *reinterpret_cast<volatile unsigned*>(&sm->tmem_mask);
-        const bool blocked = sm->waiter >= 0 && sm->waiter != w;
+        const bool blocked = false;
         unsigned feasible = 0;
         for (int c = 0; c < N_CLASSES; ++c) {
           const int su = ctx.classes[c].smem_units, tu = ctx.classes[c].tmem_units;
@@ -348,43 +348,18 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     if (want >= 0) {
       QueueEntry e;
       if (queue_try_pop(ctx, want, e, gtimer() + ctx.wait_limit_ns)) {
-        WorkerTile& h = slot->held;
+        WorkerTile& h = slot->held[slot->held_tail % HELD_DEPTH];
         h.inst = e.inst_node >> 20; h.node = e.inst_node & 0xFFFFFu; h.tile = e.tile; h.cls = want;
         const NodeDesc& nd = ctx.nodes[h.node];
         h.smem_units = (nd.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT;
         h.tmem_units = (nd.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT;
-        slot->held_valid = 1;
+        __threadfence_block();
+        slot->held_tail = slot->held_tail + 1;      // the worker takes it as soon as it is free
         progressed = true;
       } else {                                         // lost the race: undo the count
         atomicSub(&sm->pick.cta_count[want], 1);
         for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[want * 3 + x]);
       }
-    }
-    // ---- hand the held tile over when the worker is free and the tile's exact need fits
-    for (int w = 0; w < n_workers; ++w) {
-      if (lane == w && slot->held_valid && slot->busy == 0 && slot->mail_state == 0) {
-        WorkerTile& h = slot->held;
-        const bool needs_mem = h.smem_units > 0 || h.tmem_units > 0;
-        const bool yield = needs_mem && sm->waiter >= 0 && sm->waiter != w;   // an older claim is waiting for room
-        const unsigned long long smask = *reinterpret_cast<volatile unsigned long long*>(&sm->smem_mask);
-        const unsigned tmask = *reinterpret_cast<volatile unsigned*>(&sm->tmem_mask);
-        int s0 = yield ? -1 : find_free(smask, h.smem_units, sm->n_smem_units);
-        int t0 = yield ? -1 : find_free((unsigned long long)tmask, h.tmem_units, sm->n_tmem_units);
-        if (!yield && (s0 < 0 || t0 < 0)) sm->waiter = w;
-        if (s0 >= 0 && t0 >= 0) {
-          if (sm->waiter == w) sm->waiter = -1;
-          h.smem_unit0 = s0; h.tmem_unit0 = t0;
-          if (h.smem_units) atomicOr(&sm->smem_mask, unit_bits(h.smem_units) << s0);
-          if (h.tmem_units) atomicOr(&sm->tmem_mask, (unsigned)(unit_bits(h.tmem_units) << t0));
-          slot->mail = h;
-          slot->busy = 1;
-          __threadfence_block();
-          slot->mail_state = 1;
-          slot->held_valid = 0;
-          progressed = true;
-        }
-      }
-      __syncwarp();
     }
     // ---- admission, exit and watchdog (lane 0 decides, every few rounds)
     int verdict = 0;   // 1 = leave
@@ -415,9 +390,9 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     if (verdict) leaving = true;
     if (leaving) {
       // stop claiming; once every worker is idle and nothing is posted, send them home
-      const bool quiet = !serving || (slot->busy == 0 && slot->done_state == 0 && slot->mail_state == 0);
+      const bool quiet = !serving || (slot->busy == 0 && slot->done_state == 0 && slot->held_tail == slot->held_head);
       if (__all_sync(0xffffffffu, quiet)) {
-        if (serving) { __threadfence_block(); slot->mail_state = 2; }
+        if (serving) { __threadfence_block(); slot->leave = 1; }
         __syncwarp();
         if (lane == 0) { __threadfence_block(); sm->quit = 1; }
         break;
@@ -452,7 +427,8 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
     sm->waiter = -1;
     sm->quit = 0;
     for (int w = 0; w < MAX_WORKERS; ++w) {
-      sm->slot[w].mail_state = 0; sm->slot[w].done_state = 0; sm->slot[w].busy = 0; sm->slot[w].held_valid = 0;
+      sm->slot[w].held_tail = 0; sm->slot[w].held_head = 0; sm->slot[w].leave = 0; sm->slot[w].done_state = 0;
+      sm->slot[w].busy = 0;
       sm->slot[w].n_ready = 0;
     }
   }
@@ -470,18 +446,62 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
     const int bar_id = worker + 1;
     WorkerSlot* slot = sm->slot + worker;
     unsigned long long tiles = 0;
+    int tau[N_CLASSES * 3];
+    for (int c = 0; c < N_CLASSES; ++c)
+      for (int x = 0; x < 3; ++x) tau[c * 3 + x] = ctx.classes[c].tau[x];
     for (;;) {
       if (wt == 0) {
+        // take the tile the claim warp holds for this worker, then give it its exact memory need
         int st;
         unsigned naps = 0;
-        while ((st = slot->mail_state) == 0) { __nanosleep(naps < 64 ? 20 : 200); ++naps; }
+#ifdef VLA_TILE_TIMING
+        const uint64_t tw0 = gtimer();
+#endif
+        for (;;) {
+          if (slot->held_tail != slot->held_head) { st = 1; break; }
+          if (slot->leave) { st = 2; break; }
+          __nanosleep(naps < 64 ? 20 : 100);
+          ++naps;
+        }
+#ifdef VLA_TILE_TIMING
+        const uint64_t tw1 = gtimer();
+        atomicAdd(ctl->dbg + 5, tw1 - tw0); atomicAdd(ctl->dbg + 6, 1ull);
+#endif
+        WorkerTile& cur = sm->cur[worker];
         if (st == 1) {
-          sm->cur[worker] = slot->mail;
-          sm->cur[worker].t0 = 1;            // marks "run"
+          cur = slot->held[slot->held_head % HELD_DEPTH];
+          slot->busy = 1;
           __threadfence_block();
-          slot->mail_state = 0;
+          slot->held_head = slot->held_head + 1;   // the claim warp may refill the slot
+          const uint64_t lim = gtimer() + ctx.wait_limit_ns;
+          bool ok = false;
+          for (unsigned spin = 0;; ++spin) {
+            const unsigned long long sm_old = *reinterpret_cast<volatile unsigned long long*>(&sm->smem_mask);
+            const int s0 = find_free(sm_old, cur.smem_units, sm->n_smem_units);
+            if (s0 >= 0) {
+              const unsigned long long sbits = unit_bits(cur.smem_units) << s0;
+              if (cur.smem_units == 0 || atomicCAS(&sm->smem_mask, sm_old, sm_old | sbits) == sm_old) {
+                const unsigned tm_old = *reinterpret_cast<volatile unsigned*>(&sm->tmem_mask);
+                const int t0 = find_free((unsigned long long)tm_old, cur.tmem_units, sm->n_tmem_units);
+                const unsigned tbits = (unsigned)(unit_bits(cur.tmem_units) << (t0 < 0 ? 0 : t0));
+                if (t0 >= 0 && (cur.tmem_units == 0 || atomicCAS(&sm->tmem_mask, tm_old, tm_old | tbits) == tm_old)) {
+                  cur.smem_unit0 = s0; cur.tmem_unit0 = t0;
+                  ok = true;
+                  break;
+                }
+                if (cur.smem_units) atomicAnd(&sm->smem_mask, ~sbits);   // no tensor memory yet: give the shared memory back
+              }
+            }
+            __nanosleep(100);
+            if ((spin & 255u) == 255u && (gtimer() > lim || ld_volatile_u32(&ctl->error) != 0u)) break;
+          }
+#ifdef VLA_TILE_TIMING
+          atomicAdd(ctl->dbg + 7, gtimer() - tw1); atomicAdd(ctl->dbg + 8, 1ull);
+#endif
+          if (!ok) set_error(ctx, DEV_ERR_IDLE_LIMIT, 0x2000u + (unsigned)blockIdx.x);
+          cur.t0 = ok ? 1 : 2;              // 1 run, 2 skip (error), 0 leave
         } else {
-          sm->cur[worker].t0 = 0;            // marks "leave"
+          cur.t0 = 0;
         }
       }
       asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
@@ -503,21 +523,32 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
       const uint64_t t0 = gtimer();
       tc.deadline = t0 + ctx.wait_limit_ns;
       const uint64_t frame = *reinterpret_cast<const volatile uint64_t*>(ctx.inst_frame + cmd.inst);
-      run_tile(ctx, tc, n, (int)cmd.tile, (int)cmd.inst, frame);
+      if (cmd.t0 == 1) run_tile(ctx, tc, n, (int)cmd.tile, (int)cmd.inst, frame);
       asm volatile("fence.proxy.async;" ::: "memory");   // outputs may be read by TMA on another SM
       asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
       if (wt == 0) {
         ++tiles;
+        const uint64_t t1 = gtimer();
+        if (cmd.t0 == 1) {
+          if (cmd.smem_units) atomicAnd(&sm->smem_mask, ~(unit_bits(cmd.smem_units) << cmd.smem_unit0));
+          if (cmd.tmem_units) atomicAnd(&sm->tmem_mask, ~(unsigned)(unit_bits(cmd.tmem_units) << cmd.tmem_unit0));
+        }
+        atomicSub(&sm->pick.cta_count[cmd.cls], 1);
+        for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[cmd.cls * 3 + x]);
         unsigned naps = 0;
         while (slot->done_state != 0) {
           __nanosleep(40);
-          if ((++naps & 0xFFFFu) == 0 && gtimer() - t0 > 2 * ctx.wait_limit_ns) break;   // dispatcher gone: give up posting
+          if ((++naps & 0xFFFFu) == 0 && gtimer() - t0 > 2 * ctx.wait_limit_ns) break;   // retire warp gone: give up posting
         }
+#ifdef VLA_TILE_TIMING
+        atomicAdd(ctl->dbg + 9, gtimer() - t1); atomicAdd(ctl->dbg + 10, 1ull);
+#endif
         WorkerTile d = cmd;
-        d.t0 = t0; d.t1 = gtimer(); d.frame = frame;
+        d.t0 = t0; d.t1 = t1; d.frame = frame;
         slot->done = d;
         __threadfence();       // the tile's writes (all threads, ordered by the barrier) before the completion is seen
         slot->done_state = 1;
+        slot->busy = 0;
       }
     }
     if (wt == 0) atomicAdd(&ctl->tiles_done, tiles);

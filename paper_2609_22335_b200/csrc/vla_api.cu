@@ -607,7 +607,7 @@ int vla_get_counters(vla_ctx* c, uint64_t* tiles, uint64_t* kernel_launches, uin
               ctl.dbg[3] ? ctl.dbg[0] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3] ? ctl.dbg[1] / 1e3 / ctl.dbg[3] : 0.0,
               ctl.dbg[3] ? ctl.dbg[2] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3], ctl.dbg[3] ? (double)ctl.dbg[4] / ctl.dbg[3] : 0.0);
     if (getenv("VLA_PRINT_DBG"))
-      fprintf(stderr, "dbg: pick hit %.2f us x %llu  pick miss %.2f us x %llu  complete %.2f us x %llu\n",
+      fprintf(stderr, "dbg: wait-for-claim %.2f us x %llu  wait-for-room %.2f us x %llu  wait-to-post %.2f us x %llu\n",
               ctl.dbg[6] ? ctl.dbg[5] / 1e3 / ctl.dbg[6] : 0.0, ctl.dbg[6], ctl.dbg[8] ? ctl.dbg[7] / 1e3 / ctl.dbg[8] : 0.0,
               ctl.dbg[8], ctl.dbg[10] ? ctl.dbg[9] / 1e3 / ctl.dbg[10] : 0.0, ctl.dbg[10]);
   }
