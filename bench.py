@@ -35,6 +35,9 @@ from vla_synth.gen import make_weights, frame_inputs  # noqa: E402
 
 METRIC = "action_chunks_per_sec"
 UNIT = "chunks/s"
+# DRAM bytes per action chunk of the persistent kernel, from the ncu capture summarised in
+# profiles/cosched_kernel_cfg2_small_dram.md (small case, scaled by chunks: an upper bound at full size)
+MEASURED_DRAM_BYTES_PER_CHUNK = {"cfg2_smolvla": 2.649e9 + 0.184e9}
 
 
 def measured_peaks():
@@ -125,7 +128,7 @@ def run_mode(m, weights, mode, R, F, steps, warmup, e2e_steps, policy, rank, sam
     eng.load_weights(weights)
     # a small pool of distinct frames per stream, cycled (inputs > L2 in total for the large workloads)
     pool = min(F, 4)
-    host = [[frame_inputs(m, r + 1000 * rank, n, seed=0) for n in range(pool)] for r in range(R)]
+    host = [[frame_inputs(m, gid, n, seed=0) for n in range(pool)] for gid in rank_stream_ids(R, rank)]
     dev = [[{k: (None if v is None else torch.from_numpy(np.ascontiguousarray(v)).to(eng.device)) for k, v in fr.items()}
             for fr in s] for s in host]
     pinned = [[{k: (None if v is None else torch.from_numpy(np.ascontiguousarray(v)).pin_memory()) for k, v in fr.items()}
@@ -149,6 +152,8 @@ def run_mode(m, weights, mode, R, F, steps, warmup, e2e_steps, policy, rank, sam
             torch.distributed.barrier()
 
     def timed(submit, k):
+        eng.wait_idle()
+        time.sleep(0.005)          # the persistent kernel leaves after 200 us idle: the timed region starts with its launch
         dist_barrier()
         torch.cuda.synchronize()
         c0 = eng.counters()
@@ -183,6 +188,26 @@ def run_mode(m, weights, mode, R, F, steps, warmup, e2e_steps, policy, rank, sam
     res["d2h_bytes"] = int(np.prod(eng.chunk_shape)) * 4 * R * F
     eng.close()
     return res
+
+
+def aggregate_over_ranks(step_s, e2e_s, chunks_per_rank, world, device=None):
+    """Whole-job numbers from per-rank step times: the slowest rank sets the time, every rank's chunks count.
+
+    Request streams are independent, so ranks are replicas with no data-path collective; the only
+    communication is this MAX reduction (and the barriers around the timed region)."""
+    import torch
+    if world > 1:
+        t = torch.tensor([step_s, e2e_s or 0.0], dtype=torch.float64, device=device)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        step_s, e2e_s = float(t[0]), (float(t[1]) or None)
+    chunks = chunks_per_rank * world
+    return {"step_s": step_s, "e2e_s": e2e_s, "chunks": chunks, "value": chunks / step_s,
+            "e2e_value": (chunks / e2e_s) if e2e_s else None}
+
+
+def rank_stream_ids(n_streams, rank):
+    """Global request-stream ids served by one rank (weak scaling: every rank serves n_streams of its own)."""
+    return [rank * n_streams + r for r in range(n_streams)]
 
 
 def time_oracle(m, weights, n_frames, dtype=np.float32):
@@ -264,14 +289,8 @@ def main():
     weights = make_weights(m, seed=0)
     sampler = ClockSampler(local) if rank == 0 else None
     res = run_mode(m, weights, args.mode, R, F, args.steps, args.warmup, 0 if args.no_e2e else 1, args.policy, rank, sampler)
-    step_s = res["device_s"] / args.steps
-    e2e_s = res.get("e2e_s")
-    if world > 1:
-        t = torch.tensor([step_s, e2e_s or 0.0], device="cuda", dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        step_s, e2e_s = float(t[0]), (float(t[1]) or None)
-    chunks = R * F * world
-    value = chunks / step_s
+    agg = aggregate_over_ranks(res["device_s"] / args.steps, res.get("e2e_s"), R * F, world, device="cuda")
+    step_s, e2e_s, chunks, value = agg["step_s"], agg["e2e_s"], agg["chunks"], agg["value"]
     peaks = measured_peaks()
     flops_step = work["flops"] * R * F
     t_tensor = flops_step / (peaks["tflops_sustained"] * 1e12)
@@ -285,7 +304,10 @@ def main():
     else:
         achieved = work["weight_bytes"] * F / (res["device_s"] / args.steps) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"]}
-    roof.update({"traffic": None, "peak_source": peaks["source"] + (" (sustained bf16)" if bound == "tensor" else ""),
+    per_chunk = MEASURED_DRAM_BYTES_PER_CHUNK.get(m.name)
+    roof.update({"traffic": (per_chunk * R * F) if per_chunk else None,
+                 "traffic_note": "ncu dram bytes per chunk on a 2x2 case x chunks per step (upper bound)" if per_chunk else None,
+                 "peak_source": peaks["source"] + (" (sustained bf16)" if bound == "tensor" else ""),
                  "kernel": "vla_cosched_kernel (whole step)" if args.mode == "cosched" else "all node kernels of the step",
                  "launches_per_step": launches_per_step, "roof_chunks_per_s": R * F / max(t_tensor, t_hbm)})
     out = {

@@ -113,7 +113,7 @@ typedef struct {
 
 /* Static description of one node of the tile program (for the trace checker). */
 typedef struct {
-  int32_t op, cls, n_tiles, n_pred;
+  int32_t op, cls, n_tiles, n_pred;   /* n_pred: tiles of all predecessor nodes (what the node's counter waits for) */
   int32_t phase;            /* 0 VLM, 1 action head */
   int32_t step;             /* denoising step, -1 outside the loop */
   int32_t succ_begin, succ_count; /* range in the successor array */

@@ -52,34 +52,27 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
 }
 
 // ------------------------------------------------------------------ tile queues
-// Pushing tiles is split in three so a whole worker can fill the entries in parallel:
+// Pushing tiles is split in three so a whole warp can fill the entries in parallel:
 // reserve (one thread), fill (any threads, entry i of the range), commit (one thread, after a barrier).
+// The ring is sized for every tile of every frame slot, so a reservation can never overrun the head.
+__device__ __forceinline__ unsigned long long queue_word(const DeviceCtx& ctx, unsigned long long ticket, uint32_t inst,
+                                                         uint32_t node, uint32_t tile) {
+  const unsigned long long gen = ((ticket >> ctx.q_shift) + 1ull) & 0xFFFFull;
+  return (gen << 48) | ((unsigned long long)(tile & 0xFFFFu) << 32) | (unsigned long long)((inst << 20) | node);
+}
 __device__ inline unsigned long long queue_reserve(const DeviceCtx& ctx, int cls, int n) {
-  TileQueue* q = ctx.queues + cls;
-  const unsigned long long base = atomicAdd(&q->tail, (unsigned long long)n);
-  const unsigned long long head = ld_volatile_u64(&q->head);
-  if (base + n - head > (unsigned long long)ctx.q_capacity) set_error(ctx, DEV_ERR_QUEUE_FULL, cls);
-  return base;
+  return atomicAdd(&ctx.queues[cls].tail, (unsigned long long)n);
 }
 __device__ inline void queue_fill(const DeviceCtx& ctx, int cls, unsigned long long base, uint32_t inst, uint32_t node, int first,
                                   int count, int stride) {
   const unsigned long long mask = (unsigned long long)ctx.q_capacity - 1;
   QueueEntry* ent = ctx.q_entries + (size_t)cls * ctx.q_capacity;
-  unsigned long long* seq = ctx.q_seq + (size_t)cls * ctx.q_capacity;
-  for (int i = first; i < count; i += stride) {
-    QueueEntry e;
-    e.inst_node = (inst << 20) | node;
-    e.tile = (uint32_t)i;
-    ent[(base + i) & mask] = e;
-  }
-  __threadfence();   // entries before their sequence words
   for (int i = first; i < count; i += stride)
-    *reinterpret_cast<volatile unsigned long long*>(seq + ((base + i) & mask)) = base + i + 1;
+    *reinterpret_cast<volatile unsigned long long*>(ent + ((base + i) & mask)) = queue_word(ctx, base + i, inst, node, (uint32_t)i);
 }
 __device__ inline void queue_commit(const DeviceCtx& ctx, int cls, int n) {
   __threadfence();
   atomicAdd(reinterpret_cast<unsigned long long*>(&ctx.queues[cls].avail), (unsigned long long)n);
-  atomicAdd(&ctx.control->doorbell, 1ull);
 }
 // One thread pushes everything (admission of a frame's root tiles).
 __device__ inline void queue_push(const DeviceCtx& ctx, int cls, uint32_t inst, uint32_t node, int n) {
@@ -98,15 +91,17 @@ __device__ inline bool queue_try_pop(const DeviceCtx& ctx, int cls, QueueEntry& 
   }
   const unsigned long long t = atomicAdd(&q->head, 1ull);
   const unsigned long long mask = (unsigned long long)ctx.q_capacity - 1;
-  const unsigned long long* seq = ctx.q_seq + (size_t)cls * ctx.q_capacity + (t & mask);
+  const unsigned long long want = ((t >> ctx.q_shift) + 1ull) & 0xFFFFull;
+  const unsigned long long* slot = ctx.q_entries + (size_t)cls * ctx.q_capacity + (t & mask);
   unsigned spins = 0;
-  while (ld_acquire_u64(seq) != t + 1) {
+  unsigned long long w;
+  while (((w = ld_acquire_u64(slot)) >> 48) != want) {
     if ((++spins & 63u) == 0 && gtimer() > deadline) {
       set_error(ctx, DEV_ERR_WAIT_QUEUE, cls);
       return false;
     }
   }
-  e = ctx.q_entries[(size_t)cls * ctx.q_capacity + (t & mask)];
+  e = w;
   return true;
 }
 
@@ -205,17 +200,13 @@ __device__ inline void try_admit(const DeviceCtx& ctx) {
   }
 }
 
-// Global side of a finished tile: bump the node's counter; the last tile of a node releases its
-// successors, whose queue ranges are reserved here and returned in `slot` for the warp to fill.
+// Global side of a finished tile: every successor node's counter (which counts its predecessors' tiles)
+// goes down by one; a counter reaching zero re-arms itself and releases that node, whose queue range is
+// reserved here and returned in `slot` for the warp to fill.
 __device__ inline void complete_tile(const DeviceCtx& ctx, uint32_t inst, uint32_t node_idx, WorkerSlot* slot) {
   const NodeDesc& n = ctx.nodes[node_idx];
   slot->n_ready = 0;
   __threadfence();
-  int* cnt = ctx.tiles_done + (size_t)inst * ctx.n_nodes + node_idx;
-  int done = atomicAdd(cnt, 1) + 1;
-  if (done != n.n_tiles) return;
-  __threadfence();
-  *cnt = 0;
   for (int i = 0; i < n.succ_count; ++i) {
     int s = ctx.succ[n.succ_begin + i];
     int* dep = ctx.dep_count + (size_t)inst * ctx.n_nodes + s;
@@ -349,7 +340,8 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
       QueueEntry e;
       if (queue_try_pop(ctx, want, e, gtimer() + ctx.wait_limit_ns)) {
         WorkerTile& h = slot->held[slot->held_tail % HELD_DEPTH];
-        h.inst = e.inst_node >> 20; h.node = e.inst_node & 0xFFFFFu; h.tile = e.tile; h.cls = want;
+        h.inst = (uint32_t)(e & 0xFFFFFFFFull) >> 20; h.node = (uint32_t)e & 0xFFFFFu; h.tile = (uint32_t)(e >> 32) & 0xFFFFu;
+        h.cls = want;
         const NodeDesc& nd = ctx.nodes[h.node];
         h.smem_units = (nd.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT;
         h.tmem_units = (nd.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT;

@@ -186,7 +186,7 @@ int vla_op_linear(const void* a, const void* w, float* out32, void* out16, int32
   g.tiles_t = (m + GEMM_MAX_BT - 1) / GEMM_MAX_BT;
   g.bt = (int)op_pad((m + g.tiles_t - 1) / g.tiles_t, 16);
   const int stage = GEMM_BM * GEMM_BK * 2 + g.bt * GEMM_BK * 2;
-  g.stages = std::max(1, std::min(std::max(2, std::min(4, GEMM_SMEM_BUDGET / stage)), g.Kp / GEMM_BK));
+  g.stages = std::max(1, std::min(std::max(2, std::min(4, (g.bt <= 64 ? 100 * 1024 : GEMM_SMEM_BUDGET) / stage)), g.Kp / GEMM_BK));
   g.wmap = 0; g.w2map = 0; g.amap = 1;
   OpMaps maps;
   memset(&maps, 0, sizeof maps);

@@ -220,9 +220,10 @@ class Builder {
     int bt = (int)pad_to((g.M + tiles_t - 1) / tiles_t, 16);
     g.bt = bt; g.tiles_t = tiles_t;
     {
-      // pipeline depth from the stage size; tensor maps for the operands
+      // pipeline depth from the stage size: token-poor tiles (the action head) are bound by TMA latency,
+      // so they get up to 4 stages in flight; tensor maps for the operands
       int stage = GEMM_BM * GEMM_BK * 2 * (g.dual ? 2 : 1) + bt * GEMM_BK * 2;
-      int S = std::max(2, std::min(4, GEMM_SMEM_BUDGET / stage));
+      int S = std::max(2, std::min(4, (bt <= 64 ? 100 * 1024 : GEMM_SMEM_BUDGET) / stage));
       S = std::min(S, std::max(1, g.Kp / GEMM_BK));
       g.stages = S;
       n.smem_bytes = 1024 + S * stage;
@@ -878,7 +879,9 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     auto& pr = b.preds[i];
     std::sort(pr.begin(), pr.end());
     pr.erase(std::unique(pr.begin(), pr.end()), pr.end());
-    p.nodes[i].n_pred = (int)pr.size();
+    int pred_tiles = 0;                     // the counter a node waits on counts its predecessors' tiles
+    for (int q : pr) pred_tiles += p.nodes[q].n_tiles;
+    p.nodes[i].n_pred = pred_tiles;
     for (int q : pr) succ[q].push_back(i);
     if (pr.empty()) p.roots.push_back(i);
   }
@@ -901,6 +904,7 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   }
   for (const NodeDesc& n : p.nodes) {
     if (n.smem_bytes > 54 * SMEM_UNIT) { set_err(p, "a tile needs more shared memory than one SM offers"); return false; }
+    if (n.n_tiles >= 65536) { set_err(p, "a node has too many tiles"); return false; }
     ClassInfo& ci = p.classes[n.cls];
     ci.smem_units = std::max(ci.smem_units, (n.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT);
     ci.tmem_units = std::max(ci.tmem_units, (n.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT);
@@ -932,7 +936,6 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   while ((uint64_t)cap < want && cap < (1 << 24)) cap <<= 1;
   p.q_capacity = cap;
   p.off_q_entries = place(sizeof(QueueEntry) * (uint64_t)cap * N_CLASSES);
-  p.off_q_seq = place(sizeof(unsigned long long) * (uint64_t)cap * N_CLASSES);
   p.admit_capacity = 1;
   while (p.admit_capacity < 2 * p.n_inst) p.admit_capacity <<= 1;
   p.off_admit = place(sizeof(AdmitRec) * p.admit_capacity);

@@ -71,7 +71,7 @@ struct Program {
 
   // arena layout (byte offsets)
   uint64_t off_weights = 0, off_consts = 0, off_nodes = 0, off_succ = 0, off_roots = 0, off_classes = 0,
-           off_control = 0, off_queues = 0, off_q_entries = 0, off_q_seq = 0, off_admit = 0, off_dep = 0,
+           off_control = 0, off_queues = 0, off_q_entries = 0, off_admit = 0, off_dep = 0,
            off_tiles_done = 0, off_inst_frame = 0, off_slot_base = 0, off_input_ptrs = 0, off_trace = 0, off_tmaps = 0,
            off_init_nodes = 0, off_slots = 0;
   uint64_t slot_bytes = 0, arena_bytes = 0, zero_bytes_begin = 0;

@@ -8,40 +8,34 @@
 namespace vla {
 
 // ------------------------------------------------------------------ RMSNorm tile (one warp per row, float4 lanes)
-// Rows up to 2048 wide are read once and held in registers; wider rows take a second pass through L2.
-__device__ void tile_rmsnorm(const TileCtx& c, const NormArgs& a, int tile) {
-  constexpr int MAXV = 16;
-  const int warp = c.tid >> 5, lane = c.tid & 31;
-  const float4* g4 = reinterpret_cast<const float4*>(resolve<const float>(c, a.g));
-  const float* mod = resolve<const float>(c, a.mod);
-  unsigned short* out = resolve<unsigned short>(c, a.out);
-  const float* xbase = resolve<const float>(c, a.x);
-  const int d4 = a.d >> 2;                      // widths are multiples of 4
-  const bool in_regs = d4 <= 32 * MAXV;
-  for (int rr = warp; rr < a.rows_per_tile; rr += WORKER_THREADS / 32) {
-    const int r = tile * a.rows_per_tile + rr;
-    if (r >= a.M) break;
-    const float4* x4 = reinterpret_cast<const float4*>(xbase + (size_t)r * a.ldx);
-    float4 v[MAXV];
+// A warp keeps RIF rows in flight (their loads are issued before any arithmetic), each held in registers:
+// RIF x NV float4 per lane covers widths up to 128 * NV.
+template <int RIF, int NV>
+__device__ __forceinline__ void rmsnorm_rows(const NormArgs& a, const float* xbase, const float4* g4, const float* mod,
+                                             unsigned short* out, int r0, int nrows, int lane) {
+  const int d4 = a.d >> 2;
+  float4 v[RIF][NV];
+#pragma unroll
+  for (int q = 0; q < RIF; ++q) {
+    const float4* x4 = reinterpret_cast<const float4*>(xbase + (size_t)(r0 + q) * a.ldx);
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+      const int i = lane + 32 * k;
+      v[q][k] = (q < nrows && i < d4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < RIF; ++q) {
+    if (q >= nrows) break;
     float ss = 0.f;
-    if (in_regs) {
 #pragma unroll
-      for (int k = 0; k < MAXV; ++k) {
-        const int i = lane + 32 * k;
-        v[k] = i < d4 ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-#pragma unroll
-      for (int k = 0; k < MAXV; ++k) {
-        ss = fmaf(v[k].x, v[k].x, ss); ss = fmaf(v[k].y, v[k].y, ss); ss = fmaf(v[k].z, v[k].z, ss); ss = fmaf(v[k].w, v[k].w, ss);
-      }
-    } else {
-      for (int i = lane; i < d4; i += 32) {
-        float4 t = __ldcg(x4 + i);
-        ss = fmaf(t.x, t.x, ss); ss = fmaf(t.y, t.y, ss); ss = fmaf(t.z, t.z, ss); ss = fmaf(t.w, t.w, ss);
-      }
+    for (int k = 0; k < NV; ++k) {
+      ss = fmaf(v[q][k].x, v[q][k].x, ss); ss = fmaf(v[q][k].y, v[q][k].y, ss);
+      ss = fmaf(v[q][k].z, v[q][k].z, ss); ss = fmaf(v[q][k].w, v[q][k].w, ss);
     }
     ss = warp_sum(ss);
     const float inv = 1.0f / sqrtf(ss / (float)a.d + 1e-6f);
+    const int r = r0 + q;
     size_t orow = r, ocol0 = 0;
     if (a.shuffle > 1) {
       int y = r / a.grid, xx = r % a.grid, s = a.shuffle;
@@ -49,8 +43,11 @@ __device__ void tile_rmsnorm(const TileCtx& c, const NormArgs& a, int tile) {
       ocol0 = (size_t)((y % s) * s + (xx % s)) * a.d;
     }
     uint2* o2 = reinterpret_cast<uint2*>(out + orow * a.ldo + ocol0);
-    auto emit = [&](int i, float4 t) {
-      float4 gg = g4[i];
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+      const int i = lane + 32 * k;
+      if (i >= d4) continue;
+      const float4 t = v[q][k], gg = g4[i];
       float y0 = t.x * inv * gg.x, y1 = t.y * inv * gg.y, y2 = t.z * inv * gg.z, y3 = t.w * inv * gg.w;
       if (mod) {
         float4 ga = reinterpret_cast<const float4*>(mod)[i], be = reinterpret_cast<const float4*>(mod + a.d)[i];
@@ -59,15 +56,50 @@ __device__ void tile_rmsnorm(const TileCtx& c, const NormArgs& a, int tile) {
       }
       __nv_bfloat162 lo = __floats2bfloat162_rn(y0, y1), hi = __floats2bfloat162_rn(y2, y3);
       o2[i] = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
-    };
-    if (in_regs) {
-#pragma unroll
-      for (int k = 0; k < MAXV; ++k) {
-        const int i = lane + 32 * k;
-        if (i < d4) emit(i, v[k]);
+    }
+  }
+}
+
+__device__ void tile_rmsnorm(const TileCtx& c, const NormArgs& a, int tile) {
+  const int warp = c.tid >> 5, lane = c.tid & 31;
+  const float4* g4 = reinterpret_cast<const float4*>(resolve<const float>(c, a.g));
+  const float* mod = resolve<const float>(c, a.mod);
+  unsigned short* out = resolve<unsigned short>(c, a.out);
+  const float* xbase = resolve<const float>(c, a.x);
+  const int d4 = a.d >> 2;                      // widths are multiples of 4
+  // this warp's rows: a contiguous share of the tile's rows
+  const int per_warp = (a.rows_per_tile + 3) / 4;
+  const int row_lo = tile * a.rows_per_tile + warp * per_warp;
+  const int row_hi = min(min(row_lo + per_warp, (tile + 1) * a.rows_per_tile), a.M);
+  if (d4 <= 128) {
+    for (int r = row_lo; r < row_hi; r += 4) rmsnorm_rows<4, 4>(a, xbase, g4, mod, out, r, min(4, row_hi - r), lane);
+  } else if (d4 <= 256) {
+    for (int r = row_lo; r < row_hi; r += 2) rmsnorm_rows<2, 8>(a, xbase, g4, mod, out, r, min(2, row_hi - r), lane);
+  } else if (d4 <= 512) {
+    for (int r = row_lo; r < row_hi; ++r) rmsnorm_rows<1, 16>(a, xbase, g4, mod, out, r, 1, lane);
+  } else {
+    // very wide rows: two passes through L2
+    for (int r = row_lo; r < row_hi; ++r) {
+      const float4* x4 = reinterpret_cast<const float4*>(xbase + (size_t)r * a.ldx);
+      float ss = 0.f;
+      for (int i = lane; i < d4; i += 32) {
+        float4 t = __ldcg(x4 + i);
+        ss = fmaf(t.x, t.x, ss); ss = fmaf(t.y, t.y, ss); ss = fmaf(t.z, t.z, ss); ss = fmaf(t.w, t.w, ss);
       }
-    } else {
-      for (int i = lane; i < d4; i += 32) emit(i, __ldcg(x4 + i));
+      ss = warp_sum(ss);
+      const float inv = 1.0f / sqrtf(ss / (float)a.d + 1e-6f);
+      uint2* o2 = reinterpret_cast<uint2*>(out + (size_t)r * a.ldo);
+      for (int i = lane; i < d4; i += 32) {
+        const float4 t = __ldcg(x4 + i), gg = g4[i];
+        float y0 = t.x * inv * gg.x, y1 = t.y * inv * gg.y, y2 = t.z * inv * gg.z, y3 = t.w * inv * gg.w;
+        if (mod) {
+          float4 ga = reinterpret_cast<const float4*>(mod)[i], be = reinterpret_cast<const float4*>(mod + a.d)[i];
+          y0 = y0 * (1.0f + ga.x) + be.x; y1 = y1 * (1.0f + ga.y) + be.y;
+          y2 = y2 * (1.0f + ga.z) + be.z; y3 = y3 * (1.0f + ga.w) + be.w;
+        }
+        __nv_bfloat162 lo = __floats2bfloat162_rn(y0, y1), hi = __floats2bfloat162_rn(y2, y3);
+        o2[i] = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+      }
     }
   }
 }

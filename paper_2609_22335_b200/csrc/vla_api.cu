@@ -362,7 +362,6 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
   x.control = at<Control>(c, p.off_control);
   x.queues = at<TileQueue>(c, p.off_queues);
   x.q_entries = at<QueueEntry>(c, p.off_q_entries);
-  x.q_seq = at<unsigned long long>(c, p.off_q_seq);
   x.admit_ring = at<AdmitRec>(c, p.off_admit);
   x.dep_count = at<int32_t>(c, p.off_dep);
   x.tiles_done = at<int32_t>(c, p.off_tiles_done);
@@ -386,6 +385,8 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
   x.n_inst = p.n_inst;
   x.n_roots = (int)p.roots.size();
   x.q_capacity = p.q_capacity;
+  x.q_shift = 0;
+  while ((1 << x.q_shift) < p.q_capacity) ++x.q_shift;
   x.admit_capacity = p.admit_capacity;
   x.trace_capacity = p.trace_capacity;
   x.policy = opts->policy;

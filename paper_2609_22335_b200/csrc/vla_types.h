@@ -143,10 +143,10 @@ struct TileQueue {             // one 128-byte line per queue
   unsigned long long pad[13];
 };
 
-struct QueueEntry {            // 8 bytes: one tile
-  uint32_t inst_node;          // inst << 20 | node
-  uint32_t tile;
-};
+// One queued tile is one 64-bit word, written and read atomically:
+//   bits 63..48 generation tag ((ticket / capacity + 1) & 0xFFFF; 0 = never written),
+//   bits 47..32 tile index inside the node, bits 31..0 inst << 20 | node.
+typedef unsigned long long QueueEntry;
 
 struct AdmitRec {              // written by the host (copy stream), read by the dispatcher
   uint32_t inst;
@@ -198,7 +198,6 @@ struct DeviceCtx {
   Control* control;
   TileQueue* queues;             // [N_CLASSES]
   QueueEntry* q_entries;         // [N_CLASSES][q_capacity]
-  unsigned long long* q_seq;     // [N_CLASSES][q_capacity] ticket+1 when the entry is valid
   AdmitRec* admit_ring;
   int32_t* dep_count;            // [n_inst][n_nodes]
   int32_t* tiles_done;           // [n_inst][n_nodes]
@@ -213,7 +212,7 @@ struct DeviceCtx {
   const void* tmaps;             // CUtensorMap table (128 B each): weight maps, then n_act_tmaps per frame slot
   int32_t n_weight_tmaps, n_act_tmaps;
   int32_t n_nodes, n_inst, n_roots;
-  int32_t q_capacity, admit_capacity;
+  int32_t q_capacity, q_shift, admit_capacity;   // q_capacity = 1 << q_shift
   uint32_t trace_capacity;
   int32_t policy, workers_per_sm;
   uint64_t wait_limit_ns, idle_exit_ns;
