@@ -117,6 +117,7 @@ typedef struct {
   int32_t phase;            /* 0 VLM, 1 action head */
   int32_t step;             /* denoising step, -1 outside the loop */
   int32_t succ_begin, succ_count; /* range in the successor array */
+  int32_t smem_bytes, tmem_cols;  /* shared memory and tensor-memory columns one tile of the node occupies */
   char name[48];
 } vla_node_info;
 

@@ -56,7 +56,8 @@ class vla_trace_rec(C.Structure):
 
 class vla_node_info(C.Structure):
     _fields_ = [("op", C.c_int32), ("cls", C.c_int32), ("n_tiles", C.c_int32), ("n_pred", C.c_int32), ("phase", C.c_int32),
-                ("step", C.c_int32), ("succ_begin", C.c_int32), ("succ_count", C.c_int32), ("name", C.c_char * 48)]
+                ("step", C.c_int32), ("succ_begin", C.c_int32), ("succ_count", C.c_int32), ("smem_bytes", C.c_int32), ("tmem_cols", C.c_int32),
+                ("name", C.c_char * 48)]
 
 
 TRACE_DTYPE = np.dtype([("inst", "<u4"), ("node", "<u4"), ("tile", "<u4"), ("sm", "<u2"), ("worker", "u1"), ("cls", "u1"),
@@ -305,6 +306,7 @@ class Engine:
         succ = (C.c_int32 * max(ns.value, 1))()
         self._check(self.lib.vla_program_info(self.ctx, nodes, nn.value, C.byref(nn), succ, ns.value, C.byref(ns)))
         out = [dict(op=n.op, cls=n.cls, n_tiles=n.n_tiles, n_pred=n.n_pred, phase=n.phase, step=n.step,
+                    smem_bytes=n.smem_bytes, tmem_cols=n.tmem_cols,
                     succ=[succ[n.succ_begin + i] for i in range(n.succ_count)], name=n.name.decode()) for n in nodes]
         return out
 

@@ -28,7 +28,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
            "-shared", "-Xcompiler", "-fPIC", "-x", "cu",
-           "-DVLA_EXPORTS", "-o", LIB]
+           "-DVLA_EXPORTS", "-o", LIB,
+           # no implicit multiply-add contraction: the same tile body is compiled into several kernels (the
+           # persistent one, the per-node ones, the single-op ones) and must round identically in all of them;
+           # the fused multiply-adds the bodies want are written as fmaf()
+           "-fmad=false"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     if os.environ.get("VLA_TILE_TIMING"):

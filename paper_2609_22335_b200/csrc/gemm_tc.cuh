@@ -94,6 +94,12 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// 16-byte asynchronous copy global -> shared through L2 (the source was written by other SMs)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   uint32_t r[16];
   asm volatile(
@@ -105,6 +111,58 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Epilogue phase 1 (thread = output feature, the TMEM lane it owns): read the accumulators 16 token columns at a
+// time, apply the row scale and the activation, and park the values in shared memory as [token][feature]; a
+// feature of the V^T part of a q|k|v projection is written from here, 16 consecutive tokens per store pair.
+struct Phase1Args {
+  float* St; const float* rs; unsigned short* outT_row;
+  float c_acc, c_x; uint32_t lane_base; int bt, nt, tid, t0;
+  bool x_staged;            // the residual rows already sit in St: accumulate on top of them
+};
+template <int ACT, bool DUAL>
+__device__ __forceinline__ void gemm_phase1(const Phase1Args& p) {
+  for (int c0 = 0; c0 < p.nt; c0 += 16) {
+    float a[16], b[16], v[16];
+    tmem_ld16(p.lane_base + (uint32_t)c0, a);
+    if (DUAL) tmem_ld16(p.lane_base + (uint32_t)(p.bt + c0), b);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float sc = p.rs ? p.rs[c0 + j] : 1.0f;
+      float t = apply_act_t<ACT>(a[j] * sc);
+      if (DUAL) t *= b[j] * sc;
+      v[j] = t * p.c_acc;
+    }
+    if (p.outT_row) {
+      unsigned short* op = p.outT_row + p.t0 + c0;
+      uint32_t pk[8];
+#pragma unroll
+      for (int j = 0; j < 16; j += 2) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[j], v[j + 1]);
+        pk[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      if (p.nt - c0 >= 16) {
+        *reinterpret_cast<uint4*>(op) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        *reinterpret_cast<uint4*>(op + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (j < p.nt - c0) op[j] = (unsigned short)((j & 1) ? (pk[j >> 1] >> 16) : (pk[j >> 1] & 0xFFFFu));
+      }
+    }
+    float* sp = p.St + (size_t)c0 * GEMM_BM + p.tid;
+    if (p.x_staged) {
+      float x[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) x[j] = sp[j * GEMM_BM];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) sp[j * GEMM_BM] = fmaf(p.c_x, x[j], v[j]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) sp[j * GEMM_BM] = v[j];
+    }
+  }
 }
 
 constexpr int GEMM_BAR_BYTES = 1024;   // barrier block at the head of the slab (keeps the stages 1024-byte aligned)
@@ -135,6 +193,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   worker_sync(c);
 
   const uint32_t tmem_d = c.tmem;                 // accumulator columns [0, bt) (and [bt, 2 bt) when dual)
+  float* rs_smem = reinterpret_cast<float*>(c.smem + 256);       // [bt] row scales, inside the barrier block
 #ifdef VLA_TILE_TIMING
   uint64_t tt0; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt0));
 #endif
@@ -189,33 +248,150 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
     if (ok) umma_commit(accum_bar);     // accumulators complete
     }
     __syncwarp();
+  } else if (g.rs_d > 0) {
+    // ---------------- folded RMSNorm: row scales from the stream's per-row partial sums of squares, summed in a
+    // fixed order while the main loop runs (thread j: tokens j and j + 64)
+    const float* ssp = resolve<const float>(c, g.ss_in);
+    for (int tkn = c.tid - 64; tkn < g.bt; tkn += 64) {
+      float ssq = 0.f;
+      if (tkn < nt)
+        for (int q = 0; q < g.ss_nft; ++q) ssq += ld_act(ssp + (size_t)(t0 + tkn) * g.ss_nft + q);
+      rs_smem[tkn] = 1.0f / sqrtf(ssq / (float)g.rs_d + 1e-6f);
+    }
   }
 
-  // ---------------- epilogue: warp w owns TMEM lanes 32w..32w+31 = features f0+32w..
+  // ---------------- epilogue in two phases.
+  // Phase 1 (thread = output feature, the TMEM lane it owns): read the accumulators, apply the row scale and the
+  // activation, and park the values in shared memory (the pipeline stages are free now) as [token][feature];
+  // the V^T part of a q|k|v projection is written from here, 16 consecutive tokens per thread.
+  // Phase 2 (warp = token row, lane = 4 consecutive features): add the residual / vectors / tables and store
+  // whole 512-byte rows; the row's sum of squares over this tile's features goes to the stream's partials.
   const bool ready = mbar_wait(c, accum_bar, 0u);
   __syncwarp();
   tc_fence_after();
 #ifdef VLA_TILE_TIMING
   uint64_t tt1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt1));
 #endif
+  GemmPtrs ptrs = gemm_ptrs(c, g);
+  float* St = reinterpret_cast<float*>(c.smem + GEMM_BAR_BYTES);   // [bt][128] fp32
+  const bool vec4 = (g.N % 4 == 0) && (!ptrs.X || g.ldx % 4 == 0) && (!ptrs.tab || g.ldtab % 4 == 0) &&
+                    (!ptrs.tab2 || g.ldtab2 % 4 == 0) && (!ptrs.out32 || g.ldo32 % 4 == 0) && (!ptrs.out16 || g.ldo16 % 4 == 0);
+  const int gf = f0 + 4 * lane;            // phase 2: this lane's four consecutive features
+  const bool fok = gf < g.N;
+  // The residual rows of this tile start their way into the staging area now (asynchronous 16-byte copies
+  // through L2, no registers held), so their latency overlaps the accumulator read-out.
+  const bool x_staged = vec4 && ptrs.X != nullptr;
+  if (x_staged) {
+    if (ready && fok)
+      for (int tok = warp; tok < nt; tok += 4)
+        cp_async16(smem_u32(St + (size_t)tok * GEMM_BM + 4 * lane), ptrs.X + (size_t)(t0 + tok) * g.ldx + gf);
+    cp_async_wait_all();
+  }
+  if (g.rs_d > 0 || x_staged) worker_sync(c);     // row scales written by warps 2 and 3; residual rows landed
   if (ready) {
-    GemmPtrs ptrs = gemm_ptrs(c, g);
-    const int f = f0 + warp * 32 + lane;
-    const bool fok = f < g.N;
-    const float vecf = (ptrs.vec && fok) ? ptrs.vec[f] : 0.f;
-    const uint32_t lane_base = tmem_d + ((uint32_t)(warp * 32) << 16);
-    for (int c0 = 0; c0 < nt; c0 += 16) {
-      float a[16], b[16];
-      tmem_ld16(lane_base + (uint32_t)c0, a);
-      if (g.dual) tmem_ld16(lane_base + (uint32_t)(g.bt + c0), b);
-      if (!fok) continue;
-      const int n = min(16, nt - c0), r0 = t0 + c0;
-      if (g.dual) {
-        if (g.act == ACT_SILU) gemm_store16<ACT_SILU, true>(g, ptrs, r0, n, f, vecf, a, b);
-        else gemm_store16<ACT_GELU, true>(g, ptrs, r0, n, f, vecf, a, b);
-      } else if (g.act == ACT_GELU) gemm_store16<ACT_GELU, false>(g, ptrs, r0, n, f, vecf, a, b);
-      else if (g.act == ACT_SILU) gemm_store16<ACT_SILU, false>(g, ptrs, r0, n, f, vecf, a, b);
-      else gemm_store16<ACT_NONE, false>(g, ptrs, r0, n, f, vecf, a, b);
+    Phase1Args p1;
+    p1.St = St; p1.rs = g.rs_d > 0 ? rs_smem : nullptr; p1.c_acc = g.c_acc; p1.c_x = g.c_x; p1.x_staged = x_staged;
+    p1.lane_base = tmem_d + ((uint32_t)(warp * 32) << 16);
+    p1.bt = g.bt; p1.nt = nt; p1.tid = c.tid; p1.t0 = t0;
+    const int f = f0 + c.tid;
+    p1.outT_row = (ptrs.outT != nullptr && f >= g.t_col0 && f < g.N) ? ptrs.outT + (size_t)(f - g.t_col0) * g.ldoT : nullptr;
+    if (g.dual) {
+      if (g.act == ACT_SILU) gemm_phase1<ACT_SILU, true>(p1);
+      else if (g.act == ACT_GELU) gemm_phase1<ACT_GELU, true>(p1);
+      else gemm_phase1<ACT_NONE, true>(p1);
+    } else {
+      if (g.act == ACT_GELU) gemm_phase1<ACT_GELU, false>(p1);
+      else if (g.act == ACT_SILU) gemm_phase1<ACT_SILU, false>(p1);
+      else gemm_phase1<ACT_NONE, false>(p1);
+    }
+  }
+  worker_sync(c);
+#ifdef VLA_TILE_TIMING
+  if (c.tid == 64 && g.M > 512 && c.dbg) {
+    uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    atomicAdd(c.dbg + 11, t - tt1);
+    if (ptrs.X) { atomicAdd(c.dbg + 12, 1ull); }
+  }
+#endif
+  if (ready) {
+    float* ssq_out = resolve<float>(c, g.ss_out);
+    if (vec4) {
+      const bool skip16 = ptrs.outT != nullptr && gf >= g.t_col0;      // these columns went to V^T in phase 1
+      float4 vecv = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (ptrs.vec && fok) vecv = *reinterpret_cast<const float4*>(ptrs.vec + gf);
+      // four token rows per pass; the lane's share of each row's sum of squares is left in the row's first 32
+      // words (rotated by the row's slot so the final per-row additions run without bank conflicts)
+      constexpr int RP = 4;
+      for (int tok0 = warp; tok0 < nt; tok0 += 4 * RP) {
+        float4 v[RP];
+#pragma unroll
+        for (int q = 0; q < RP; ++q) {
+          const int tok = tok0 + 4 * q;
+          v[q] = tok < nt ? *reinterpret_cast<const float4*>(St + (size_t)tok * GEMM_BM + 4 * lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < RP; ++q) {
+          const int tok = tok0 + 4 * q;
+          if (tok < nt) {
+            const int r = t0 + tok;
+            float4 w = v[q];
+            w.x += vecv.x; w.y += vecv.y; w.z += vecv.z; w.w += vecv.w;
+            if (fok && ptrs.tab) {
+              const float4 t = *reinterpret_cast<const float4*>(ptrs.tab + (size_t)r * g.ldtab + gf);
+              w.x += t.x; w.y += t.y; w.z += t.z; w.w += t.w;
+            }
+            if (fok && ptrs.tab2) {
+              const float4 t = *reinterpret_cast<const float4*>(ptrs.tab2 + (size_t)r * g.ldtab2 + gf);
+              w.x += t.x; w.y += t.y; w.z += t.z; w.w += t.w;
+            }
+            if (fok) {
+              if (ptrs.out32) *reinterpret_cast<float4*>(ptrs.out32 + (size_t)r * g.ldo32 + gf) = w;
+              if (ptrs.out16 && !skip16) {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+                *reinterpret_cast<uint2*>(ptrs.out16 + (size_t)r * g.ldo16 + gf) =
+                    make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+              }
+            }
+            if (ssq_out) {
+              const float sq = fok ? (w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w) : 0.f;
+              St[(size_t)tok * GEMM_BM + ((lane + (tok >> 2)) & 31)] = sq;
+            }
+          }
+        }
+      }
+      if (ssq_out) {
+        __syncwarp();
+        const int tok = warp + 4 * lane;                 // this lane's row: slot `lane` of this warp
+        if (tok < nt) {
+          float sq = 0.f;
+#pragma unroll 8
+          for (int i = 0; i < 32; ++i) sq += St[(size_t)tok * GEMM_BM + ((i + lane) & 31)];   // lane order 0..31
+          ssq_out[(size_t)(t0 + tok) * g.ss_out_ld + ft] = sq;
+        }
+      }
+    } else {
+      // odd widths (e.g. a 7-wide action output): one feature per lane and pass
+      for (int tok = warp; tok < nt; tok += 4) {
+        const int r = t0 + tok;
+        float sq = 0.f;
+        for (int q = lane; q < GEMM_BM; q += 32) {
+          const int of = f0 + q;
+          if (of >= g.N) continue;
+          float v = St[(size_t)tok * GEMM_BM + q];
+          if (ptrs.X) v = fmaf(g.c_x, ld_act(ptrs.X + (size_t)r * g.ldx + of), v);
+          if (ptrs.vec) v += ptrs.vec[of];
+          if (ptrs.tab) v += ptrs.tab[(size_t)r * g.ldtab + of];
+          if (ptrs.tab2) v += ptrs.tab2[(size_t)r * g.ldtab2 + of];
+          if (ptrs.out32) ptrs.out32[(size_t)r * g.ldo32 + of] = v;
+          if (ptrs.out16 && !(ptrs.outT && of >= g.t_col0)) ptrs.out16[(size_t)r * g.ldo16 + of] = f32_to_bf16_bits(v);
+          sq = fmaf(v, v, sq);
+        }
+        if (ssq_out) {
+          sq = warp_sum(sq);
+          if (lane == 0) ssq_out[(size_t)r * g.ss_out_ld + ft] = sq;
+        }
+      }
     }
   }
   tc_fence_before();

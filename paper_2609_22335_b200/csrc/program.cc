@@ -57,6 +57,19 @@ class Builder {
     acc.emplace_back();
     return (int)p.bufs.size() - 1;
   }
+  std::map<int, int> ss_of;     // bf16 stream mirror -> its per-row partial sums of squares
+  // bf16 mirror of a residual stream of width d plus, per row, one sum of squares per 128 columns
+  int stream_mirror(const std::string& name, int64_t nrows, int64_t d) {
+    int bf = buf(name, nrows, pad_to(d, GEMM_BK), 2);
+    int ss = buf(name + ".ss", nrows, (d + GEMM_BM - 1) / GEMM_BM, 4);
+    ss_of[bf] = ss;
+    return bf;
+  }
+  View ss_view(const View& v) const {
+    auto it = ss_of.find(v.buf);
+    if (it == ss_of.end()) return View();
+    return View{it->second, v.row0, v.rows, 0};
+  }
   static Ref in_ref(int idx, uint64_t byte_off = 0) { return REF_INPUT | ((uint64_t)idx << 56) | byte_off; }
   View all(int b) const { return View{b, 0, p.bufs[b].rows, 0}; }
   View rows(int b, int64_t r0, int64_t n, int64_t c0 = 0) const { return View{b, r0, n, c0}; }
@@ -197,6 +210,8 @@ class Builder {
     int act = ACT_NONE;
     int W2 = -1;
     int64_t w_row0 = 0;
+    int norm_gain = -1;      // >= 0: A is the raw residual stream; RMSNorm with this gain is folded into the GEMM
+    int norm_d = 0;
   };
   int gemm(const std::string& name, const View& A, int W, int64_t N, const GemmOpt& o) {
     const DevTensor& wt = p.dev_tensors[W];
@@ -216,17 +231,25 @@ class Builder {
     g.out16 = ref(o.out16); g.ldo16 = o.out16.buf >= 0 ? (int)ld(o.out16) : 0;
     g.outT = ref(o.outT); g.ldoT = o.outT.buf >= 0 ? (int)ld(o.outT) : 0; g.t_col0 = o.t_col0;
     g.act = o.act;
+    g.rs_d = 0; g.ss_nft = 0; g.ss_out_ld = 0; g.ss_in = 0; g.ss_out = 0;
+    const View ss_in = o.norm_gain >= 0 ? ss_view(A) : View();
+    const View ss_out = ss_view(o.out16);
+    if (ss_in.buf >= 0) { g.ss_in = ref(ss_in); g.ss_nft = (int)ld(ss_in); }
+    if (ss_out.buf >= 0) { g.ss_out = ref(ss_out); g.ss_out_ld = (int)ld(ss_out); }
+    if (o.norm_gain >= 0) {
+      if (ss_in.buf < 0) p.error = "internal: folded norm needs a stream mirror as operand (" + name + ")";
+      g.rs_d = o.norm_d;
+      p.folds.push_back({W, o.norm_gain});
+      if (o.W2 >= 0) p.folds.push_back({o.W2, o.norm_gain});
+    }
     int tiles_t = (int)((g.M + GEMM_MAX_BT - 1) / GEMM_MAX_BT);
     int bt = (int)pad_to((g.M + tiles_t - 1) / tiles_t, 16);
     g.bt = bt; g.tiles_t = tiles_t;
     {
-      // pipeline depth from the stage size: token-poor tiles (the action head) are bound by TMA latency,
-      // so they get up to 4 stages in flight; tensor maps for the operands
-      int stage = GEMM_BM * GEMM_BK * 2 * (g.dual ? 2 : 1) + bt * GEMM_BK * 2;
-      int S = std::max(2, std::min(4, (bt <= 64 ? 100 * 1024 : GEMM_SMEM_BUDGET) / stage));
-      S = std::min(S, std::max(1, g.Kp / GEMM_BK));
+      // pipeline depth from the stage size; tensor maps for the operands
+      const int S = gemm_stages(bt, g.dual != 0, g.Kp);
       g.stages = S;
-      n.smem_bytes = 1024 + S * stage;
+      n.smem_bytes = gemm_smem_bytes(bt, g.dual != 0, S);
       n.tmem_cols = (int)pad_to((int64_t)bt * (g.dual ? 2 : 1), TMEM_UNIT);
       g.wmap = weight_map(W, N);
       g.w2map = o.W2 >= 0 ? weight_map(o.W2, N) : 0;
@@ -239,6 +262,8 @@ class Builder {
     if (o.out32.buf >= 0) write(id, o.out32);
     if (o.out16.buf >= 0) write(id, o.out16);
     if (o.outT.buf >= 0) write(id, o.outT);
+    if (ss_in.buf >= 0) read(id, ss_in);
+    if (ss_out.buf >= 0) write(id, ss_out);
     if (A.rows * 1 > 0 && p.bufs[A.buf].ld < wt.ld && !init_mode) {
       p.error = "internal: activation row pitch shorter than padded K in " + name;
     }
@@ -337,10 +362,11 @@ class Builder {
 
   // q|k|v projection of `A` into `dst`: one GEMM whose V columns are written transposed; with RoPE the
   // GEMM writes fp32 and a rotary tile produces the bf16 q|k and V^T.
-  void qkv_project(const std::string& name, const View& A, int W, const QKV& dst, int hd, int scratch32, int pos0) {
+  void qkv_project(const std::string& name, const View& A, int W, const QKV& dst, int hd, int scratch32, int pos0,
+                   int norm_gain = -1, int norm_d = 0) {
     const int64_t nqk = (int64_t)(dst.hq + dst.hkv) * dst.hs, nall = nqk + (int64_t)dst.hkv * dst.hs;
     if (scratch32 >= 0) {
-      GemmOpt gq; gq.out32 = all(scratch32);
+      GemmOpt gq; gq.out32 = all(scratch32); gq.norm_gain = norm_gain; gq.norm_d = norm_d;
       gemm(name + "qkv", A, W, nall, gq);
       NodeDesc n;
       std::memset(&n, 0, sizeof n);
@@ -357,6 +383,7 @@ class Builder {
       write(id, all(dst.vt));
     } else {
       GemmOpt gq; gq.out16 = all(dst.qk); gq.outT = all(dst.vt); gq.t_col0 = (int)nqk;
+      gq.norm_gain = norm_gain; gq.norm_d = norm_d;
       gemm(name + "qkv", A, W, nall, gq);
     }
   }
@@ -374,12 +401,15 @@ class Builder {
     a.vec = vec; a.tab = tab; a.ldt = ldt;
     a.out = ref(out); a.ldo = out.buf >= 0 ? (int)ld(out) : 0;
     a.out16 = ref(out16); a.ldo16 = out16.buf >= 0 ? (int)ld(out16) : 0;
+    const View ssv = ss_view(out16);
+    a.ss_out = ref(ssv); a.ss_ld = ssv.buf >= 0 ? (int)ld(ssv) : 0;
     a.M = M; a.N = N;
     n.n_tiles = 1;
     int id = add(n, name, KIND_ELEM);
     if (in.buf >= 0) read(id, in);
     if (out.buf >= 0) write(id, out);
     if (out16.buf >= 0) write(id, out16);
+    if (ssv.buf >= 0) write(id, ssv);
     return id;
   }
 };
@@ -624,7 +654,7 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
 
   // LLM
   int x = b.buf("llm.x", S, D, 4);
-  int h = b.buf("llm.h", S, P64(D), 2);
+  int xb = b.stream_mirror("llm.xb", S, D);                // bf16 mirror of the residual stream (GEMM operand)
   int qkv32 = d.rope ? b.buf("llm.qkv32", S, nqkv, 4) : -1;
   std::vector<Builder::QKV> lq(d.llm_layers);
   {
@@ -666,11 +696,12 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
       g.tab = b.wref(w_vpos); g.ldtab = dv;
       if (w_lpos >= 0) { g.tab2 = b.wref(w_lpos, (int64_t)c * tpc); g.ldtab2 = D; }
       g.out32 = b.rows(x, (int64_t)c * tpc, tpc);
+      g.out16 = b.rows(xb, (int64_t)c * tpc, tpc);
       b.gemm(N_("vis%d.patch", c), b.all(patches), w_patch, dv, g);
       continue;
     }
     int xv = b.buf(N_("vis%d.x", c), T, dv, 4);
-    int hv = b.buf(N_("vis%d.h", c), T, P64(dv), 2);
+    int xvb = b.stream_mirror(N_("vis%d.xb", c), T, dv);   // bf16 mirror of the residual stream (GEMM operand)
     Builder::QKV vq;
     if (d.vis_layers > 0) vq = b.make_qkv(N_("vis%d.qkv", c), T, d.vis_heads, d.vis_heads, vhs);
     int vatt = d.vis_layers > 0 ? b.buf(N_("vis%d.att", c), T, P64(hvd), 2) : -1;
@@ -679,20 +710,19 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     {
       Builder::GemmOpt g;
       g.tab = b.wref(w_vpos); g.ldtab = dv;
-      if (d.vis_layers > 0) g.out32 = b.all(xv); else g.out16 = b.all(shuf);
+      if (d.vis_layers > 0) { g.out32 = b.all(xv); g.out16 = b.all(xvb); } else g.out16 = b.all(shuf);
       b.gemm(N_("vis%d.patch", c), b.all(patches), w_patch, dv, g);
     }
     for (int i = 0; i < d.vis_layers; ++i) {
-      b.rmsnorm(N_("vis%d.L%d.n1", c, i), b.all(xv), venc[i].n1, b.all(hv));
-      b.qkv_project(N_("vis%d.L%d.", c, i), b.all(hv), venc[i].wqkv, vq, d.vis_hd, -1, 0);
+      // the two RMSNorms of a layer are folded into the GEMMs that consume them (A = bf16 mirror of the stream)
+      b.qkv_project(N_("vis%d.L%d.", c, i), b.all(xvb), venc[i].wqkv, vq, d.vis_hd, -1, 0, venc[i].n1, dv);
       b.attention(N_("vis%d.L%d.attn", c, i), b.rows(vq.qk, 0, T, 0), T, vq, nullptr, b.all(vatt), d.vis_heads, d.vis_heads,
                   d.vis_hd, vhs, false);
-      Builder::GemmOpt go; go.X = b.all(xv); go.out32 = b.all(xv);
+      Builder::GemmOpt go; go.X = b.all(xv); go.out32 = b.all(xv); go.out16 = b.all(xvb);
       b.gemm(N_("vis%d.L%d.wo", c, i), b.all(vatt), venc[i].wo, dv, go);
-      b.rmsnorm(N_("vis%d.L%d.n2", c, i), b.all(xv), venc[i].n2, b.all(hv));
-      Builder::GemmOpt g1; g1.act = ACT_GELU; g1.out16 = b.all(vmid);
-      b.gemm(N_("vis%d.L%d.w1", c, i), b.all(hv), venc[i].w1, d.vis_mlp, g1);
-      Builder::GemmOpt g2; g2.X = b.all(xv); g2.out32 = b.all(xv);
+      Builder::GemmOpt g1; g1.act = ACT_GELU; g1.out16 = b.all(vmid); g1.norm_gain = venc[i].n2; g1.norm_d = dv;
+      b.gemm(N_("vis%d.L%d.w1", c, i), b.all(xvb), venc[i].w1, d.vis_mlp, g1);
+      Builder::GemmOpt g2; g2.X = b.all(xv); g2.out32 = b.all(xv); g2.out16 = b.all(xvb);
       b.gemm(N_("vis%d.L%d.w2", c, i), b.all(vmid), venc[i].w2, dv, g2);
     }
     if (d.vis_layers > 0)
@@ -701,6 +731,7 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
       Builder::GemmOpt g;
       if (w_lpos >= 0) { g.tab = b.wref(w_lpos, (int64_t)c * tpc); g.ldtab = D; }
       g.out32 = b.rows(x, (int64_t)c * tpc, tpc);
+      g.out16 = b.rows(xb, (int64_t)c * tpc, tpc);
       b.gemm(N_("vis%d.conn", c), b.all(shuf), w_conn, D, g);
     }
   }
@@ -714,28 +745,33 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     a.pos = w_lpos >= 0 ? b.wref(w_lpos, n_img) : 0;
     a.out = b.ref(b.rows(x, n_img, d.n_text));
     a.n = d.n_text; a.d = D; a.ldo = D; a.vocab = d.vocab; a.rows_per_tile = 16; a.ldt = (int)P64(D);
+    a.out16 = b.ref(b.rows(xb, n_img, d.n_text)); a.ldo16 = (int)P64(D);
+    {
+      View sv = b.ss_view(b.rows(xb, n_img, d.n_text));
+      a.ss_out = b.ref(sv); a.ss_ld = (int)b.ld(sv);
+    }
     n.n_tiles = (d.n_text + 15) / 16;
     int id = b.add(n, "llm.embed", KIND_ELEM);
     b.write(id, b.rows(x, n_img, d.n_text));
+    b.write(id, b.rows(xb, n_img, d.n_text));
+    b.write(id, b.ss_view(b.rows(xb, n_img, d.n_text)));
   }
   for (int i = 0; i < d.llm_layers; ++i) {
-    b.rmsnorm(N_("llm.L%d.n1", i), b.all(x), lw[i].n1, b.all(h));
-    b.qkv_project(N_("llm.L%d.", i), b.all(h), lw[i].wqkv, lq[i], d.hd, qkv32, 0);
+    b.qkv_project(N_("llm.L%d.", i), b.all(xb), lw[i].wqkv, lq[i], d.hd, qkv32, 0, lw[i].n1, D);
     b.attention(N_("llm.L%d.attn", i), b.rows(lq[i].qk, 0, S, 0), S, lq[i], nullptr, b.all(att), d.hq, d.hkv, d.hd, lhs,
                 d.causal != 0);
-    Builder::GemmOpt go; go.X = b.all(x); go.out32 = b.all(x);
+    Builder::GemmOpt go; go.X = b.all(x); go.out32 = b.all(x); go.out16 = b.all(xb);
     b.gemm(N_("llm.L%d.wo", i), b.all(att), lw[i].wo, D, go);
-    b.rmsnorm(N_("llm.L%d.n2", i), b.all(x), lw[i].n2, b.all(h));
-    Builder::GemmOpt g1; g1.out16 = b.all(mid);
+    Builder::GemmOpt g1; g1.out16 = b.all(mid); g1.norm_gain = lw[i].n2; g1.norm_d = D;
     if (gated) {
       g1.W2 = lw[i].wu;
       g1.act = d.mlp_kind == VLA_MLP_SWIGLU ? ACT_SILU : ACT_GELU;
-      b.gemm(N_("llm.L%d.gu", i), b.all(h), lw[i].wg, d.mlp, g1);
+      b.gemm(N_("llm.L%d.gu", i), b.all(xb), lw[i].wg, d.mlp, g1);
     } else {
       g1.act = ACT_GELU;
-      b.gemm(N_("llm.L%d.w1", i), b.all(h), lw[i].w1, d.mlp, g1);
+      b.gemm(N_("llm.L%d.w1", i), b.all(xb), lw[i].w1, d.mlp, g1);
     }
-    Builder::GemmOpt g2; g2.X = b.all(x); g2.out32 = b.all(x);
+    Builder::GemmOpt g2; g2.X = b.all(x); g2.out32 = b.all(x); g2.out16 = b.all(xb);
     b.gemm(N_("llm.L%d.w2", i), b.all(mid), gated ? lw[i].wd : lw[i].w2, D, g2);
   }
   b.rmsnorm("llm.norm", b.all(x), w_lnorm, b.all(hidden));
@@ -757,7 +793,8 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   int xs = b.buf("act.x", d.horizon, d.act_dim, 4);
   int xbf = b.buf("act.xbf", d.horizon, P64(d.act_dim), 2);
   int z = b.buf("act.z", Ta, da, 4);
-  int hz = b.buf("act.h", Ta, P64(da), 2);
+  int zb = b.stream_mirror("act.zb", Ta, da);              // bf16 mirror of the head's residual stream (GEMM operand)
+  int hz = d.head == VLA_HEAD_C ? b.buf("act.h", Ta, P64(da), 2) : -1;   // adaLN-modulated norms are separate tiles
   Builder::QKV aq = b.make_qkv("act.qkv", Ta, a_hq, a_hkv, ahs);
   int aqkv32 = (d.head == VLA_HEAD_B && d.rope) ? b.buf("act.qkv32", Ta, a_nqkv, 4) : -1;
   int aatt = b.buf("act.att", Ta, P64(std::max(a_nq, nq)), 2);
@@ -785,13 +822,14 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     Ref ct_k = b.ref(b.rows(c_ct, k, 1));
     if (first) {
       b.addrows(N_("act.s%d.tok0", k), b.all(tok0), 0, 0, 1, da, d.head == VLA_HEAD_D ? ct_k : 0, 0, 0, b.rows(z, 0, 1),
-                View());
+                b.rows(zb, 0, 1));
     }
     {
       Builder::GemmOpt g;
       if (d.head == VLA_HEAD_A || d.head == VLA_HEAD_B) g.vec = ct_k;
       if (head_pos) { g.tab = b.wref(w_apos, first); g.ldtab = da; }
       g.out32 = b.rows(z, first, d.horizon);
+      g.out16 = b.rows(zb, first, d.horizon);
       b.gemm(N_("act.s%d.in", k), b.all(xbf), w_ain, da, g);
     }
     for (int i = 0; i < d.act_layers; ++i) {
@@ -799,54 +837,57 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
       auto NN = [&](const char* leaf) { std::snprintf(nm, sizeof nm, "act.s%d.L%d.%s", k, i, leaf); return std::string(nm); };
       Ref mod1 = d.head == VLA_HEAD_C ? b.ref(b.rows(c_mod1[i], k, 1)) : 0;
       Ref mod2 = d.head == VLA_HEAD_C ? b.ref(b.rows(c_mod2[i], k, 1)) : 0;
-      b.rmsnorm(NN("n1"), b.all(z), a.n1, b.all(hz), mod1);
+      // Without adaLN the RMSNorms are folded into the GEMMs that consume them (A = bf16 mirror zb);
+      // with adaLN (head C) the modulated norm stays a tile of its own writing hz.
+      const bool fold = d.head != VLA_HEAD_C;
+      View nin = fold ? b.all(zb) : b.all(hz);
+      if (!fold) b.rmsnorm(NN("n1"), b.all(z), a.n1, b.all(hz), mod1);
       bool cross_only = d.head == VLA_HEAD_C && (i % 2 == 1);
+      auto resid = [&]() { Builder::GemmOpt go; go.X = b.all(z); go.out32 = b.all(z); go.out16 = b.all(zb); return go; };
       if (!cross_only) {
-        b.qkv_project(NN(""), b.all(hz), a.wqkv, aq, ahd, aqkv32, S);
+        b.qkv_project(NN(""), nin, a.wqkv, aq, ahd, aqkv32, S, fold ? a.n1 : -1, da);
         View att_out = b.rows(aatt, 0, Ta);
         if (d.head == VLA_HEAD_B)
           b.attention(NN("attn"), b.rows(aq.qk, 0, Ta, 0), Ta, lq[i], &aq, att_out, d.hq, d.hkv, d.hd, lhs, false);
         else
           b.attention(NN("attn"), b.rows(aq.qk, 0, Ta, 0), Ta, aq, nullptr, att_out, d.act_heads, d.act_heads, ahd, ahs, false);
-        Builder::GemmOpt go; go.X = b.all(z); go.out32 = b.all(z);
-        b.gemm(NN("wo"), b.all(aatt), a.wo, da, go);
+        b.gemm(NN("wo"), b.all(aatt), a.wo, da, resid());
       }
+      int mlp_gain = a.n2;
       if (d.head == VLA_HEAD_A) {
-        b.rmsnorm(NN("n2"), b.all(z), a.n2, b.all(hz));
-        Builder::GemmOpt gq; gq.out16 = b.all(aqc);
-        b.gemm(NN("cq"), b.all(hz), a.cq, nq, gq);
+        Builder::GemmOpt gq; gq.out16 = b.all(aqc); gq.norm_gain = a.n2; gq.norm_d = da;
+        b.gemm(NN("cq"), b.all(zb), a.cq, nq, gq);
         b.attention(NN("xattn"), b.all(aqc), Ta, lq[d.llm_layers - 1], nullptr, b.all(aatt), d.hq, d.hkv, d.hd, lhs, false);
-        Builder::GemmOpt go; go.X = b.all(z); go.out32 = b.all(z);
-        b.gemm(NN("co"), b.all(aatt), a.co, da, go);
-        b.rmsnorm(NN("n3"), b.all(z), a.n3, b.all(hz));
+        b.gemm(NN("co"), b.all(aatt), a.co, da, resid());
+        mlp_gain = a.n3;
       } else if (cross_only) {
         Builder::GemmOpt gq; gq.out16 = b.all(aqc);
         b.gemm(NN("cq"), b.all(hz), a.cq, da, gq);
         b.attention(NN("xattn"), b.all(aqc), Ta, ckv[i], nullptr, b.all(aatt), d.act_heads, d.act_heads, ahd, ahs, false);
-        Builder::GemmOpt go; go.X = b.all(z); go.out32 = b.all(z);
-        b.gemm(NN("co"), b.all(aatt), a.co, da, go);
+        b.gemm(NN("co"), b.all(aatt), a.co, da, resid());
         b.rmsnorm(NN("n2"), b.all(z), a.n2, b.all(hz), mod2);
-      } else {
+      } else if (!fold) {
         b.rmsnorm(NN("n2"), b.all(z), a.n2, b.all(hz), mod2);
       }
       Builder::GemmOpt g1; g1.out16 = b.all(amid);
+      if (fold) { g1.norm_gain = mlp_gain; g1.norm_d = da; }
       if (agated) {
         g1.W2 = a.wu;
         g1.act = d.act_mlp_kind == VLA_MLP_SWIGLU ? ACT_SILU : ACT_GELU;
-        b.gemm(NN("gu"), b.all(hz), a.wg, d.act_mlp, g1);
+        b.gemm(NN("gu"), nin, a.wg, d.act_mlp, g1);
       } else {
         g1.act = ACT_GELU;
-        b.gemm(NN("w1"), b.all(hz), a.w1, d.act_mlp, g1);
+        b.gemm(NN("w1"), nin, a.w1, d.act_mlp, g1);
       }
-      Builder::GemmOpt g2; g2.X = b.all(z); g2.out32 = b.all(z);
-      b.gemm(NN("w2"), b.all(amid), agated ? a.wd : a.w2, da, g2);
+      b.gemm(NN("w2"), b.all(amid), agated ? a.wd : a.w2, da, resid());
     }
-    b.rmsnorm(N_("act.s%d.norm", k), b.all(z), w_anorm, b.all(hz));
     {
+      // final RMSNorm folded into the output projection; the solver update is its epilogue
       Builder::GemmOpt g;
       g.X = b.all(xs); g.c_x = p.step_c_x[k]; g.c_acc = p.step_c_acc[k];
       g.out32 = b.all(xs); g.out16 = b.all(xbf);
-      b.gemm(N_("act.s%d.out", k), b.rows(hz, first, d.horizon), w_aout, d.act_dim, g);
+      g.norm_gain = w_anorm; g.norm_d = da;
+      b.gemm(N_("act.s%d.out", k), b.rows(zb, first, d.horizon), w_aout, d.act_dim, g);
     }
   }
   b.step = -1;

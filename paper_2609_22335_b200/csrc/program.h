@@ -63,6 +63,7 @@ struct Program {
   std::map<std::string, int> dev_index;
   std::vector<BufInfo> bufs;
   std::map<std::string, int> buf_index;
+  std::vector<std::pair<int, int>> folds;  // (weight matrix, gain vector): columns of the matrix get multiplied by the gain at load
   std::vector<TmapSpec> wmaps;          // weight maps (shared by all frame slots)
   std::vector<TmapSpec> amaps;          // activation maps, instantiated once per frame slot
 

@@ -129,6 +129,8 @@ __device__ void tile_embed(const TileCtx& c, const EmbedArgs& a, int tile) {
   const unsigned short* table = resolve<const unsigned short>(c, a.table);
   const float* pos = resolve<const float>(c, a.pos);
   float* obase = resolve<float>(c, a.out);
+  unsigned short* o16 = resolve<unsigned short>(c, a.out16);
+  float* ss = resolve<float>(c, a.ss_out);
   for (int rr = warp; rr < a.rows_per_tile; rr += WORKER_THREADS / 32) {
     const int r = tile * a.rows_per_tile + rr;
     if (r >= a.n) break;
@@ -136,10 +138,17 @@ __device__ void tile_embed(const TileCtx& c, const EmbedArgs& a, int tile) {
     id = min(max(id, 0), a.vocab - 1);
     const unsigned short* row = table + (size_t)id * a.ldt;
     float* out = obase + (size_t)r * a.ldo;
-    for (int i = lane; i < a.d; i += 32) {
-      float v = bf16_bits_to_f32(row[i]);
-      if (pos) v += pos[(size_t)r * a.d + i];
-      out[i] = v;
+    for (int b0 = 0; b0 < a.d; b0 += 128) {            // one 128-column block at a time (4 columns per lane)
+      float sq = 0.f;
+      for (int i = b0 + lane; i < min(b0 + 128, a.d); i += 32) {
+        float v = bf16_bits_to_f32(row[i]);
+        if (pos) v += pos[(size_t)r * a.d + i];
+        out[i] = v;
+        if (o16) o16[(size_t)r * a.ldo16 + i] = f32_to_bf16_bits(v);
+        sq = fmaf(v, v, sq);
+      }
+      sq = warp_sum(sq);
+      if (ss && lane == 0) ss[(size_t)r * a.ss_ld + (b0 >> 7)] = sq;
     }
   }
 }
@@ -185,6 +194,22 @@ __device__ void tile_addrows(const TileCtx& c, const AddRowsArgs& a, int) {
     if (tab) v += tab[(size_t)r * a.ldt + col];
     if (out) out[(size_t)r * a.ldo + col] = v;
     if (out16) out16[(size_t)r * a.ldo16 + col] = f32_to_bf16_bits(v);
+  }
+  float* ss = resolve<float>(c, a.ss_out);
+  if (ss) {
+    // per-row sums of squares of what was just written, one partial per 128 columns (one thread per partial)
+    const int nb = (a.N + 127) / 128;
+    for (int e = c.tid; e < a.M * nb; e += WORKER_THREADS) {
+      const int r = e / nb, b0 = (e % nb) * 128;
+      float sq = 0.f;
+      for (int col = b0; col < min(b0 + 128, a.N); ++col) {
+        float v = ld_act(in + (size_t)r * a.ldi + col);
+        if (vec) v += vec[col];
+        if (tab) v += tab[(size_t)r * a.ldt + col];
+        sq = fmaf(v, v, sq);
+      }
+      ss[(size_t)r * a.ss_ld + (b0 >> 7)] = sq;
+    }
   }
 }
 

@@ -102,71 +102,4 @@ __device__ __forceinline__ GemmPtrs gemm_ptrs(const TileCtx& c, const GemmArgs& 
   p.outT = resolve<unsigned short>(c, g.outT);
   return p;
 }
-// Epilogue of one thread's 16 consecutive tokens of one output feature f:
-//   out[r][f] = c_x X[r][f] + c_acc * (act(acc) [* acc2]) + vec[f] + tab[r][f] + tab2[r][f]
-// Loads are issued for all 16 tokens before any arithmetic or store so that they overlap
-// (X and the fp32 output may be the same buffer, which would otherwise serialise them).
-template <int ACT, bool DUAL>
-__device__ __forceinline__ void gemm_store16(const GemmArgs& g, const GemmPtrs& p, int r0, int n, int f, float vecf,
-                                             const float* a, const float* b) {
-  float v[16];
-#pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    float t = apply_act_t<ACT>(a[j]);
-    if (DUAL) t *= b[j];
-    v[j] = t * g.c_acc + vecf;
-  }
-  if (p.X) {
-    const float* xp = p.X + (size_t)r0 * g.ldx + f;
-    float x[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) x[j] = j < n ? __ldcg(xp + (size_t)j * g.ldx) : 0.f;
-#pragma unroll
-    for (int j = 0; j < 16; ++j) v[j] = fmaf(g.c_x, x[j], v[j]);
-  }
-  if (p.tab) {
-    const float* tp = p.tab + (size_t)r0 * g.ldtab + f;
-    float x[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) x[j] = j < n ? tp[(size_t)j * g.ldtab] : 0.f;
-#pragma unroll
-    for (int j = 0; j < 16; ++j) v[j] += x[j];
-  }
-  if (p.tab2) {
-    const float* tp = p.tab2 + (size_t)r0 * g.ldtab2 + f;
-    float x[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) x[j] = j < n ? tp[(size_t)j * g.ldtab2] : 0.f;
-#pragma unroll
-    for (int j = 0; j < 16; ++j) v[j] += x[j];
-  }
-  if (p.out32) {
-    float* op = p.out32 + (size_t)r0 * g.ldo32 + f;
-#pragma unroll
-    for (int j = 0; j < 16; ++j)
-      if (j < n) op[(size_t)j * g.ldo32] = v[j];
-  }
-  if (p.outT && f >= g.t_col0) {
-    // transposed output: this thread's 16 tokens are contiguous in row f - t_col0
-    unsigned short* op = p.outT + (size_t)(f - g.t_col0) * g.ldoT + r0;
-    uint32_t pk[8];
-#pragma unroll
-    for (int j = 0; j < 16; j += 2) {
-      __nv_bfloat162 h = __floats2bfloat162_rn(v[j], v[j + 1]);
-      pk[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
-    }
-    if (n == 16) {
-      *reinterpret_cast<uint4*>(op) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-      *reinterpret_cast<uint4*>(op + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-    } else {
-      for (int j = 0; j < n; ++j) op[j] = (unsigned short)((j & 1) ? (pk[j >> 1] >> 16) : (pk[j >> 1] & 0xFFFFu));
-    }
-  } else if (p.out16) {
-    unsigned short* op = p.out16 + (size_t)r0 * g.ldo16 + f;
-#pragma unroll
-    for (int j = 0; j < 16; ++j)
-      if (j < n) op[(size_t)j * g.ldo16] = f32_to_bf16_bits(v[j]);
-  }
-}
-
 }  // namespace vla

@@ -181,6 +181,17 @@ int launch_persistent(vla_ctx* c) {
   return VLA_OK;
 }
 
+// RMSNorm gains are folded into the matrices that consume the normalised rows: W[n][k] *= g[k] (bf16, nearest even).
+__global__ void vla_fold_gain_kernel(unsigned short* w, int64_t rows, int cols, int64_t ld, const float* g) {
+  const int64_t total = rows * cols;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = e / cols;
+    const int k = (int)(e % cols);
+    unsigned short* p = w + r * ld + k;
+    *p = f32_to_bf16_bits(bf16_bits_to_f32(*p) * g[k]);
+  }
+}
+
 // (Re)launch the persistent kernel if it is not running and frames are waiting.
 int ensure_persistent(vla_ctx* c) {
   if (c->pending_frames == 0) return VLA_OK;
@@ -460,6 +471,20 @@ int vla_load_weights(vla_ctx* c, const vla_tensor* tensors, size_t n, int32_t fi
   if (!final_call) return VLA_OK;
   for (auto& s : p.sources)
     if (!s.loaded) return fail(c, VLA_ERR_INVALID, "tensor '%s' was not supplied", s.name.c_str());
+  // fold the RMSNorm gains into the weights of the GEMMs that apply those norms (each pair once)
+  {
+    std::vector<std::pair<int, int>> done;
+    for (auto& f : p.folds) {
+      if (std::find(done.begin(), done.end(), f) != done.end()) continue;
+      done.push_back(f);
+      const DevTensor& wt = p.dev_tensors[f.first];
+      const DevTensor& gt = p.dev_tensors[f.second];
+      vla_fold_gain_kernel<<<592, 256, 0, c->sa>>>(reinterpret_cast<unsigned short*>(c->arena + p.off_weights + wt.offset), wt.rows,
+                                                   (int)wt.cols, wt.ld,
+                                                   reinterpret_cast<const float*>(c->arena + p.off_weights + gt.offset));
+      CU(cudaGetLastError());
+    }
+  }
   // one-off constants (time-embedding MLP, adaLN modulation) on the GPU, serially
   const NodeDesc* init_dev = at<NodeDesc>(c, p.off_init_nodes);
   for (size_t i = 0; i < p.init_program.size(); ++i) {
@@ -563,6 +588,7 @@ int vla_program_info(vla_ctx* c, vla_node_info* nodes, size_t node_cap, size_t* 
       vla_node_info& o = nodes[i];
       o.op = n.op; o.cls = n.cls; o.n_tiles = n.n_tiles; o.n_pred = n.n_pred; o.phase = n.phase; o.step = n.step;
       o.succ_begin = n.succ_begin; o.succ_count = n.succ_count;
+      o.smem_bytes = n.smem_bytes; o.tmem_cols = n.tmem_cols;
       std::memset(o.name, 0, sizeof o.name);
       std::strncpy(o.name, p.node_names[i].c_str(), sizeof(o.name) - 1);
     }
@@ -607,6 +633,8 @@ int vla_get_counters(vla_ctx* c, uint64_t* tiles, uint64_t* kernel_launches, uin
       fprintf(stderr, "dbg: first_full %.2f us  mainloop %.2f us  epilogue %.2f us  tiles %llu  kb/tile %.1f\n",
               ctl.dbg[3] ? ctl.dbg[0] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3] ? ctl.dbg[1] / 1e3 / ctl.dbg[3] : 0.0,
               ctl.dbg[3] ? ctl.dbg[2] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3], ctl.dbg[3] ? (double)ctl.dbg[4] / ctl.dbg[3] : 0.0);
+    if (getenv("VLA_PRINT_DBG"))
+      fprintf(stderr, "dbg: epilogue phase 1 %.2f us (sync+ptrs %.2f us), tiles with residual %llu\n", ctl.dbg[3] ? ctl.dbg[11] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3] ? ctl.dbg[13] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[12]);
     if (getenv("VLA_PRINT_DBG"))
       fprintf(stderr, "dbg: wait-for-claim %.2f us x %llu  wait-for-room %.2f us x %llu  wait-to-post %.2f us x %llu\n",
               ctl.dbg[6] ? ctl.dbg[5] / 1e3 / ctl.dbg[6] : 0.0, ctl.dbg[6], ctl.dbg[8] ? ctl.dbg[7] / 1e3 / ctl.dbg[8] : 0.0,

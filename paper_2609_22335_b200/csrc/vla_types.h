@@ -38,7 +38,23 @@ constexpr int GEMM_BM = 128;   // output features per GEMM tile (the MMA M dimen
 constexpr int GEMM_BK = 64;    // K elements per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int WORKER_THREADS = 128;
 constexpr int GEMM_MAX_BT = 128;     // most tokens per GEMM tile (MMA N)
-constexpr int GEMM_SMEM_BUDGET = 64 * 1024;  // stage memory a GEMM tile aims for (at least two stages are always taken)
+constexpr int GEMM_SMEM_BUDGET = 64 * 1024;  // stage memory a token-rich GEMM tile aims for (at least two stages are always taken)
+constexpr int GEMM_SMEM_BUDGET_SMALL = 84 * 1024;  // token-poor tiles (<= 64 tokens) are bound by TMA latency and get deeper
+                                                   // pipelines, but must fit the room one finished token-rich tile leaves
+                                                   // on an SM that runs three of them (3 x 17 of 56 four-KB units)
+// TMA pipeline depth of a GEMM tile with `bt` tokens per tile.
+inline int gemm_stage_bytes(int bt, bool dual) { return GEMM_BM * GEMM_BK * 2 * (dual ? 2 : 1) + bt * GEMM_BK * 2; }
+inline int gemm_stages(int bt, bool dual, int Kp) {
+  const int stage = gemm_stage_bytes(bt, dual);
+  int S = (bt <= 64 ? GEMM_SMEM_BUDGET_SMALL : GEMM_SMEM_BUDGET) / stage;
+  S = S < 2 ? 2 : (S > 4 ? 4 : S);
+  const int nkb = Kp / GEMM_BK;
+  return S < nkb ? S : (nkb < 1 ? 1 : nkb);
+}
+inline int gemm_smem_bytes(int bt, bool dual, int S) {      // the epilogue parks the tile in the stage memory as fp32
+  const int a = S * gemm_stage_bytes(bt, dual), b = bt * GEMM_BM * 4;
+  return 1024 + (a > b ? a : b);
+}
 
 struct GemmArgs {
   Ref A, W, W2;        // A bf16 [M,lda]; W (and W2 when dual) bf16 [N,Kp]
@@ -54,6 +70,11 @@ struct GemmArgs {
   float c_acc, c_x;    // out = c_x * X + c_acc * acc + vec + tab + tab2
   int32_t wmap, w2map, amap;  // tensor-map indices: shared weight maps, activation map relative to the slot's first
   int32_t stages;             // TMA pipeline depth
+  int32_t rs_d;               // > 0: A holds the raw residual stream (bf16) and RMSNorm is folded into the GEMM: every
+                              // output row is scaled by 1/sqrt(sum_j ss_in[row][j] / rs_d + 1e-6)
+  int32_t ss_nft, ss_out_ld, pad_;
+  Ref ss_in;                  // fp32 [M, ss_nft]: per-row sums of squares of the stream, one partial per 128 columns
+  Ref ss_out;                 // optional fp32 [M, ss_out_ld]: this tile writes the partial of its 128 output features
 };
 
 struct NormArgs {
@@ -80,6 +101,9 @@ struct PatchArgs {
 };
 
 struct EmbedArgs {
+  Ref out16;                  // optional bf16 mirror of the output rows
+  Ref ss_out;                 // optional fp32 [n, ss_ld] per-row sums of squares, one partial per 128 columns
+  int32_t ldo16, ss_ld;
   Ref ids, table, pos, out;   // ids int32 [n]; table bf16 [vocab,d]; pos fp32 [n,d] or null; out fp32 rows
   int32_t n, d, ldo, vocab, rows_per_tile, ldt;
 };
@@ -91,7 +115,8 @@ struct RopeArgs {
 
 struct AddRowsArgs {
   Ref in, vec, tab, out, out16;  // fp32; out16 optional bf16 copy
-  int32_t M, N, ldi, ldt, ldo, ldo16;
+  Ref ss_out;                    // optional fp32 [M, ss_ld] per-row sums of squares, one partial per 128 columns
+  int32_t M, N, ldi, ldt, ldo, ldo16, ss_ld, pad_;
 };
 
 struct TimeEmbArgs {

@@ -32,7 +32,8 @@ def test_full_size_sampled_parity(m, frames, check_two_stream):
         ref = O.action_chunk(m, w, fr[r][n], np.float32)
         rel = float(np.linalg.norm(got[r][n] - ref) / np.linalg.norm(ref))
         mx = float(np.max(np.abs(got[r][n] - ref)))
-        scale = max(1.0, float(np.sqrt(np.mean(ref * ref))))     # DDIM with untrained weights amplifies the sample ~5-7x
+        # DDIM with untrained weights amplifies the sample ~5-7x: its absolute bound is taken relative to the rms
+        scale = max(1.0, float(np.sqrt(np.mean(ref * ref)))) if m.solver == "ddim" else 1.0
         assert rel <= REL_L2_TOL, (m.name, r, n, rel)
         assert mx <= MAX_ABS_TOL * scale, (m.name, r, n, mx, scale)
     # every chunk of every stream is finite and distinct streams differ

@@ -54,7 +54,10 @@ def _check_vs_oracle(m, w, frames, got, dtype=np.float32):
             rel = float(np.linalg.norm(got[r][n] - ref) / np.linalg.norm(ref))
             mx = float(np.max(np.abs(got[r][n] - ref)))
             worst = (max(worst[0], rel), max(worst[1], mx))
-            assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL, (m.name, r, n, rel, mx)
+            # DDIM with untrained weights multiplies the sample by ~1/sqrt(alpha_bar_90) = 7, so for that solver the
+            # absolute bound is taken relative to the chunk's rms (it then is the same relative requirement)
+            scale = max(1.0, float(np.sqrt(np.mean(ref * ref)))) if m.solver == "ddim" else 1.0
+            assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL * scale, (m.name, r, n, rel, mx)
     return worst
 
 
@@ -206,3 +209,19 @@ def test_policy_probe_matches_algorithm_1():
         k, ph = admission_decision(st, taus, pending, feas, rr_start=rr)
         assert got[0] == (-1 if k is None else k) and got[1] == ph
         assert got[2] == st.cta_count and got[3] == st.u
+
+
+@pytest.mark.parametrize("key", ["cfg1", "cfg3s", "cfg5s"])
+def test_non_unit_norm_gains(key):
+    """RMSNorm gains other than one (the library folds them into the consuming matrices at load)."""
+    m = SMALL[key]
+    w = make_weights(m, seed=0)
+    rng = np.random.default_rng(9)
+    from vla_synth.configs import is_gain
+    from vla_synth.gen import round_to_bf16
+    for name in w.names():
+        if is_gain(name):
+            w.override(name, round_to_bf16(rng.uniform(0.5, 1.5, size=w.shapes[name]).astype(np.float32)))
+    frames = [[frame_inputs(m, r, n, seed=0) for n in range(2)] for r in range(2)]
+    got, _ = _run(m, w, frames, "cosched")
+    _check_vs_oracle(m, w, frames, got)
