@@ -89,6 +89,9 @@ typedef struct {
   uint64_t wait_limit_ns;   /* bound of every device-side wait; 0 = default (2 s) */
   uint32_t trace_capacity;  /* tile records kept by the device trace; 0 = tracing off */
   int32_t workers_per_sm;   /* COSCHED worker groups per SM; 0 = default */
+  int32_t u_max;            /* saturation value of the per-SM utilisation counters in the pick's Phase-2 score
+                             * (Section 3.3); 0 = default: 15 x worker groups per SM (the hardware proposal's
+                             * 8-bit registers would be 255) */
 } vla_runtime_opts;
 
 typedef struct {
@@ -173,9 +176,11 @@ int vla_get_counters(vla_ctx* ctx, uint64_t* tiles, uint64_t* kernel_launches, u
 
 /* Runs the device pick function (the COSCHED policy) once on the GPU for a given per-SM
  * state, so tests can compare it with Algorithm 1.  All arrays HOST, n_cls <= 8.
- * cta_count/u are updated as the admission would; *picked = class or -1; *phase = 1, 2 or 0. */
+ * cta_count/u are updated as the admission would; *picked = class or -1; *phase = 1, 2 or 0.
+ * u_max: saturation value used by the Phase-2 score (<= 0: the paper's 255). */
 int vla_policy_probe(int32_t n_cls, const int32_t* taus /*[n_cls*3]*/, const int32_t* pending, const int32_t* feasible,
-                     int32_t* cta_count, int32_t* u /*[3]*/, int32_t rr_start, int32_t* picked, int32_t* phase);
+                     int32_t* cta_count, int32_t* u /*[3]*/, int32_t rr_start, int32_t u_max, int32_t* picked,
+                     int32_t* phase);
 
 /* ---- stand-alone operators: the engine's tile bodies on caller-owned DEVICE tensors ------------------------
  * Both run asynchronously on `stream` (a cudaStream_t; NULL = default stream). */

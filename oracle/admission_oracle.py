@@ -41,15 +41,15 @@ class SMState:
         return s
 
 
-def score(state: SMState, tau) -> int:
-    """s = sum over pipelines of headroom times intensity."""
-    return sum((U_MAX - state.u[x]) * tau[x] for x in range(3))
+def score(state: SMState, tau, u_max: int = U_MAX) -> int:
+    """s = sum over pipelines of headroom times intensity (headroom never negative)."""
+    return sum((u_max - min(u_max, state.u[x])) * tau[x] for x in range(3))
 
 
-def admit(state: SMState, k: int, tau) -> None:
+def admit(state: SMState, k: int, tau, u_max: int = U_MAX) -> None:
     state.cta_count[k] += 1
     for x in range(3):
-        state.u[x] = min(U_MAX, state.u[x] + tau[x])
+        state.u[x] = min(u_max, state.u[x] + tau[x])
 
 
 def complete(state: SMState, k: int, tau) -> None:
@@ -58,10 +58,12 @@ def complete(state: SMState, k: int, tau) -> None:
         state.u[x] = max(0, state.u[x] - tau[x])
 
 
-def admission_decision(state: SMState, taus, pending, feasible, rr_start: int = 0):
+def admission_decision(state: SMState, taus, pending, feasible, rr_start: int = 0, u_max: int = U_MAX):
     """One invocation: returns (kernel admitted or None, phase 1|2|0) and updates ``state``.
 
-    taus[k] = (tau_TC, tau_ALU, tau_MEM); pending[k], feasible[k] booleans.
+    taus[k] = (tau_TC, tau_ALU, tau_MEM); pending[k], feasible[k] booleans.  ``u_max`` is the
+    saturation value of the utilisation registers (Section 3.3: 8-bit, 255); a caller whose SM
+    holds fewer, larger units of work passes the value its counters reach on a full SM.
     """
     n = len(taus)
     # Phase 1
@@ -70,7 +72,7 @@ def admission_decision(state: SMState, taus, pending, feasible, rr_start: int = 
         if not pending[k]:
             continue
         if state.cta_count[k] == 0 and feasible[k]:
-            admit(state, k, taus[k])
+            admit(state, k, taus[k], u_max)
             return k, 1
     # Phase 2
     best_score, best_kernel = -1, None
@@ -79,12 +81,12 @@ def admission_decision(state: SMState, taus, pending, feasible, rr_start: int = 
             continue
         if not feasible[k]:
             continue
-        s = score(state, taus[k])
+        s = score(state, taus[k], u_max)
         if s > best_score:
             best_score, best_kernel = s, k
     if best_kernel is None:
         return None, 0
-    admit(state, best_kernel, taus[best_kernel])
+    admit(state, best_kernel, taus[best_kernel], u_max)
     return best_kernel, 2
 
 

@@ -41,7 +41,8 @@ class vla_model_desc(C.Structure):
 class vla_runtime_opts(C.Structure):
     _fields_ = [("arena", C.c_void_p), ("arena_bytes", C.c_size_t), ("stream_a", C.c_void_p), ("stream_b", C.c_void_p),
                 ("mode", C.c_int32), ("n_streams", C.c_int32), ("ring_depth", C.c_int32), ("policy", C.c_int32),
-                ("wait_limit_ns", C.c_uint64), ("trace_capacity", C.c_uint32), ("workers_per_sm", C.c_int32)]
+                ("wait_limit_ns", C.c_uint64), ("trace_capacity", C.c_uint32), ("workers_per_sm", C.c_int32),
+                ("u_max", C.c_int32)]
 
 
 class vla_tensor(C.Structure):
@@ -89,7 +90,7 @@ def load_library() -> C.CDLL:
     lib.vla_debug_fetch.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_char_p, C.c_void_p, C.c_size_t, P(C.c_size_t)]
     lib.vla_get_counters.argtypes = [C.c_void_p, P(C.c_uint64), P(C.c_uint64), P(C.c_uint64)]
     lib.vla_policy_probe.argtypes = [C.c_int32, P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32),
-                                     C.c_int32, P(C.c_int32), P(C.c_int32)]
+                                     C.c_int32, C.c_int32, P(C.c_int32), P(C.c_int32)]
     lib.vla_op_attention_scratch_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, P(C.c_size_t)]
     lib.vla_op_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 6 + [C.c_void_p, C.c_size_t, C.c_void_p]
     lib.vla_op_linear.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 4 + [C.c_void_p]
@@ -140,7 +141,7 @@ class Engine:
     """One library context plus the torch-owned arena and streams it runs on."""
 
     def __init__(self, model, mode="cosched", n_streams=None, ring_depth=2, policy=0, trace_capacity=0,
-                 wait_limit_ns=0, workers_per_sm=0, device="cuda:0"):
+                 wait_limit_ns=0, workers_per_sm=0, u_max=0, device="cuda:0"):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU fallback)")
@@ -161,6 +162,7 @@ class Engine:
         self.opts.wait_limit_ns = wait_limit_ns
         self.opts.trace_capacity = trace_capacity
         self.opts.workers_per_sm = workers_per_sm
+        self.opts.u_max = u_max
         self.arena_bytes = vla_required_arena_bytes(self.desc, self.opts)
         self.arena = torch.empty(self.arena_bytes + 256, dtype=torch.uint8, device=self.device)
         base = self.arena.data_ptr()
@@ -335,7 +337,7 @@ class Engine:
             pass
 
 
-def policy_probe(taus, pending, feasible, cta_count, u, rr_start=0):
+def policy_probe(taus, pending, feasible, cta_count, u, rr_start=0, u_max=0):
     """Runs the device pick once on the GPU; returns (picked, phase, cta_count, u)."""
     lib = load_library()
     n = len(taus)
@@ -345,7 +347,7 @@ def policy_probe(taus, pending, feasible, cta_count, u, rr_start=0):
     cc = (C.c_int32 * n)(*[int(x) for x in cta_count])
     uu = (C.c_int32 * 3)(*[int(x) for x in u])
     picked, phase = C.c_int32(-1), C.c_int32(0)
-    rc = lib.vla_policy_probe(n, flat, pend, feas, cc, uu, rr_start, C.byref(picked), C.byref(phase))
+    rc = lib.vla_policy_probe(n, flat, pend, feas, cc, uu, rr_start, u_max, C.byref(picked), C.byref(phase))
     if rc != VLA_OK:
         raise VlaError(rc, "policy probe failed")
     return picked.value, phase.value, list(cc), list(uu)

@@ -207,23 +207,30 @@ __device__ inline void complete_tile(const DeviceCtx& ctx, uint32_t inst, uint32
   const NodeDesc& n = ctx.nodes[node_idx];
   slot->n_ready = 0;
   __threadfence();
-  for (int i = 0; i < n.succ_count; ++i) {
-    int s = ctx.succ[n.succ_begin + i];
-    int* dep = ctx.dep_count + (size_t)inst * ctx.n_nodes + s;
-    int left = atomicSub(dep, 1) - 1;
-    if (left == 0) {
-      const NodeDesc& sn = ctx.nodes[s];
-      *dep = sn.n_pred;
+  const int n_succ = __ldg(&n.succ_count), succ0 = __ldg(&n.succ_begin);
+  for (int i0 = 0; i0 < n_succ; i0 += 4) {
+    // up to four successors per pass: their counters are decremented by independent atomics in flight together
+    int s[4], left[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) s[j] = i0 + j < n_succ ? __ldg(ctx.succ + succ0 + i0 + j) : -1;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) left[j] = s[j] >= 0 ? atomicSub(ctx.dep_count + (size_t)inst * ctx.n_nodes + s[j], 1) - 1 : 1;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (left[j] != 0) continue;
+      const NodeDesc& sn = ctx.nodes[s[j]];
+      const int sn_tiles = __ldg(&sn.n_tiles), sn_cls = __ldg(&sn.cls);
+      ctx.dep_count[(size_t)inst * ctx.n_nodes + s[j]] = __ldg(&sn.n_pred);
       if (slot->n_ready < MAX_READY) {
         ReadyItem& it = slot->ready[slot->n_ready++];
-        it.base = queue_reserve(ctx, sn.cls, sn.n_tiles);
-        it.node = (uint32_t)s; it.n_tiles = sn.n_tiles; it.cls = sn.cls;
+        it.base = queue_reserve(ctx, sn_cls, sn_tiles);
+        it.node = (uint32_t)s[j]; it.n_tiles = sn_tiles; it.cls = sn_cls;
       } else {
-        queue_push(ctx, sn.cls, inst, (uint32_t)s, sn.n_tiles);
+        queue_push(ctx, sn_cls, inst, (uint32_t)s[j], sn_tiles);
       }
     }
   }
-  if (n.op == OP_EMIT) atomicSub(&ctx.control->ctrl, 1u);
+  if (__ldg(&n.op) == OP_EMIT) atomicSub(&ctx.control->ctrl, 1u);
 }
 
 // ------------------------------------------------------------------ the two service warps of an SM
@@ -326,7 +333,7 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         for (int c = 0; c < N_CLASSES; ++c) ps.cta_count[c] = *reinterpret_cast<volatile int*>(&sm->pick.cta_count[c]);
         for (int x = 0; x < 3; ++x) ps.u[x] = *reinterpret_cast<volatile int*>(&sm->pick.u[x]);
         int phase;
-        want = pick_choose(N_CLASSES, tau, group, cand, feasible, ps, sm->pick.rr, ctx.policy, &phase);
+        want = pick_choose(N_CLASSES, tau, group, cand, feasible, ps, sm->pick.rr, ctx.policy, ctx.u_max, &phase);
         if (want >= 0) {
           atomicAdd(&sm->pick.cta_count[want], 1);     // counted from the claim on, so the next lane sees it
           for (int x = 0; x < 3; ++x) atomicAdd(&sm->pick.u[x], tau[want * 3 + x]);
@@ -342,9 +349,9 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         WorkerTile& h = slot->held[slot->held_tail % HELD_DEPTH];
         h.inst = (uint32_t)(e & 0xFFFFFFFFull) >> 20; h.node = (uint32_t)e & 0xFFFFFu; h.tile = (uint32_t)(e >> 32) & 0xFFFFu;
         h.cls = want;
-        const NodeDesc& nd = ctx.nodes[h.node];
-        h.smem_units = (nd.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT;
-        h.tmem_units = (nd.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT;
+        const NodeDesc& nd = ctx.nodes[h.node];                 // the program is immutable: read-only cached loads
+        h.smem_units = (__ldg(&nd.smem_bytes) + SMEM_UNIT - 1) / SMEM_UNIT;
+        h.tmem_units = (__ldg(&nd.tmem_cols) + TMEM_UNIT - 1) / TMEM_UNIT;
         __threadfence_block();
         slot->held_tail = slot->held_tail + 1;      // the worker takes it as soon as it is free
         progressed = true;
@@ -593,11 +600,11 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_node_kernel(DeviceCtx ctx,
 
 // ------------------------------------------------------------------ pick probe (tests)
 __global__ void vla_pick_probe_kernel(int n_cls, const int* tau, unsigned pending, unsigned feasible, PickState* st,
-                                      int rr_start, int policy, int* out) {
+                                      int rr_start, int policy, int u_max, int* out) {
   int phase;
   int group[PICK_MAX_CLASSES];
   for (int i = 0; i < PICK_MAX_CLASSES; ++i) group[i] = i;   // one class per group: the paper's listing
-  int k = pick_choose(n_cls, tau, group, pending, feasible, *st, rr_start, policy, &phase);
+  int k = pick_choose(n_cls, tau, group, pending, feasible, *st, rr_start, policy, u_max, &phase);
   if (k >= 0) pick_commit(*st, k, tau);
   out[0] = k;
   out[1] = phase;

@@ -16,7 +16,10 @@
 //   Phase 2  otherwise the pending feasible class with the largest
 //            s = sum_x (U_max - U_x[j]) * tau_x(k); strict '>' keeps the first seen.
 //
-// Counters are 32-bit and exact; headroom is clamped at U_max = 255 when scoring.
+// Counters are 32-bit and exact; headroom is clamped at U_max when scoring.  U_max is the value a
+// utilisation counter reaches on a full SM: 255 for the paper's 8-bit registers with up to 32 resident
+// CTAs, 15 x (worker groups per SM) here, where an SM holds that many tiles.  With the hardware's 255
+// and three tiles the headroom would never move and Phase 2 would degenerate to a fixed class order.
 #pragma once
 #include <stdint.h>
 
@@ -41,7 +44,7 @@ enum PickPolicy : int { POLICY_TWO_PHASE = 0, POLICY_CLASS_ORDER = 1, POLICY_ROU
 
 // Returns the chosen class or -1; *phase = 1 or 2 (0 when nothing was chosen).
 VLA_HD inline int pick_choose(int n_cls, const int* tau /*[n_cls][3]*/, const int* group /*[n_cls]*/, unsigned pending,
-                              unsigned feasible, const PickState& st, int rr_start, int policy, int* phase) {
+                              unsigned feasible, const PickState& st, int rr_start, int policy, int u_max, int* phase) {
   *phase = 0;
   unsigned ok = pending & feasible;
   if (ok == 0) return -1;
@@ -69,8 +72,8 @@ VLA_HD inline int pick_choose(int n_cls, const int* tau /*[n_cls][3]*/, const in
     if (!(ok & (1u << k))) continue;
     int s = 0;
     for (int x = 0; x < 3; ++x) {
-      int used = st.u[x] > PICK_U_MAX ? PICK_U_MAX : st.u[x];
-      s += (PICK_U_MAX - used) * tau[k * 3 + x];
+      int used = st.u[x] > u_max ? u_max : st.u[x];
+      s += (u_max - used) * tau[k * 3 + x];
     }
     if (s > best_score) { best_score = s; best = k; }
   }

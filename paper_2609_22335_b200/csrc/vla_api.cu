@@ -402,6 +402,7 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
   x.trace_capacity = p.trace_capacity;
   x.policy = opts->policy;
   x.workers_per_sm = c->workers;
+  x.u_max = opts->u_max > 0 ? opts->u_max : 15 * c->workers;
   x.wait_limit_ns = opts->wait_limit_ns ? opts->wait_limit_ns : 5000000000ull;
   x.idle_exit_ns = 200000ull;
   x.chunk_elems = (int)chunk_elems;
@@ -646,7 +647,7 @@ int vla_get_counters(vla_ctx* c, uint64_t* tiles, uint64_t* kernel_launches, uin
 }
 
 int vla_policy_probe(int32_t n_cls, const int32_t* taus, const int32_t* pending, const int32_t* feasible, int32_t* cta_count,
-                     int32_t* u, int32_t rr_start, int32_t* picked, int32_t* phase) {
+                     int32_t* u, int32_t rr_start, int32_t u_max, int32_t* picked, int32_t* phase) {
   if (n_cls < 1 || n_cls > PICK_MAX_CLASSES || !taus || !pending || !feasible || !cta_count || !u || !picked || !phase)
     return VLA_ERR_INVALID;
   PickState st;
@@ -665,7 +666,7 @@ int vla_policy_probe(int32_t n_cls, const int32_t* taus, const int32_t* pending,
   int out[2] = {-1, 0};
   cudaMemcpy(d_tau, taus, sizeof(int) * n_cls * 3, cudaMemcpyHostToDevice);
   cudaMemcpy(d_st, &st, sizeof st, cudaMemcpyHostToDevice);
-  vla_pick_probe_kernel<<<1, 1>>>(n_cls, d_tau, pm, fm, d_st, rr_start, POLICY_TWO_PHASE, d_out);
+  vla_pick_probe_kernel<<<1, 1>>>(n_cls, d_tau, pm, fm, d_st, rr_start, POLICY_TWO_PHASE, u_max > 0 ? u_max : PICK_U_MAX, d_out);
   cudaError_t e = cudaDeviceSynchronize();
   cudaMemcpy(out, d_out, 8, cudaMemcpyDeviceToHost);
   cudaMemcpy(&st, d_st, sizeof st, cudaMemcpyDeviceToHost);

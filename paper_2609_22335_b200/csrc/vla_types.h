@@ -240,6 +240,7 @@ struct DeviceCtx {
   int32_t q_capacity, q_shift, admit_capacity;   // q_capacity = 1 << q_shift
   uint32_t trace_capacity;
   int32_t policy, workers_per_sm;
+  int32_t u_max, pad_u;     // saturation value of the utilisation counters in the pick's score
   uint64_t wait_limit_ns, idle_exit_ns;
   int32_t chunk_elems;
 };
