@@ -146,7 +146,9 @@ int vla_submit_frame(vla_ctx* ctx, int32_t stream, const float* image, const int
                      const float* state, const float* noise, uint64_t* frame_id);
 
 /* Same as vla_submit_frame but the four inputs are DEVICE pointers (already resident
- * in HBM); they are copied device-to-device into the frame slot. */
+ * in HBM).  Nothing is copied: the tiles read the arrays in place through the frame
+ * slot's pointer table, so the caller must keep them valid and unmodified until this
+ * frame's chunk has been returned by vla_poll_actions (or the context is idle). */
 int vla_submit_frame_device(vla_ctx* ctx, int32_t stream, const float* image, const int32_t* text_ids,
                             const float* state, const float* noise, uint64_t* frame_id);
 

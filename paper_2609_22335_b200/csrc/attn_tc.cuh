@@ -181,13 +181,23 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a, int tile) {
     tmem_ld16_nowait(tmem_s + lane_off + 32u, sr + 32);
     tmem_ld16_nowait(tmem_s + lane_off + 48u, sr + 48);
     tmem_ld_wait();
-    float mx = m_run;
+    // full blocks (the common case) run without per-key predicates; four independent max / sum chains keep
+    // the single warp a scheduler sees from waiting on its own results
+    const bool full = __all_sync(0xffffffffu, lim >= ATTN_BN);
+    float m4[4] = {m_run, -INFINITY, -INFINITY, -INFINITY};
+    if (full) {
 #pragma unroll
-    for (int j = 0; j < ATTN_BN; ++j)
-      if (j < lim) mx = fmaxf(mx, __uint_as_float(sr[j]));
+      for (int j = 0; j < ATTN_BN; ++j) m4[j & 3] = fmaxf(m4[j & 3], __uint_as_float(sr[j]));
+    } else {
+#pragma unroll
+      for (int j = 0; j < ATTN_BN; ++j)
+        if (j < lim) m4[j & 3] = fmaxf(m4[j & 3], __uint_as_float(sr[j]));
+    }
+    const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
     const float alpha = (m_run == -INFINITY) ? 0.f : exp2_fast((m_run - mx) * a.scale_log2e);
-    const float mb = mx * a.scale_log2e;
-    float sum = 0.f;
+    const float sl2 = a.scale_log2e;
+    const float mb = mx * sl2;
+    float s4[4] = {0.f, 0.f, 0.f, 0.f};
     char* prow = Ps_gen + (size_t)r_in * 128;
 #pragma unroll
     for (int ch = 0; ch < ATTN_BN / 8; ++ch) {
@@ -195,14 +205,16 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a, int tile) {
 #pragma unroll
       for (int j = 0; j < 8; j += 2) {
         const int jj = ch * 8 + j;
-        float p0 = (jj < lim) ? exp2_fast(fmaf(__uint_as_float(sr[jj]), a.scale_log2e, -mb)) : 0.f;
-        float p1 = (jj + 1 < lim) ? exp2_fast(fmaf(__uint_as_float(sr[jj + 1]), a.scale_log2e, -mb)) : 0.f;
-        __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);     // the row sum uses the rounded probabilities the MMA sees
-        sum += __low2float(h2) + __high2float(h2);
+        float p0 = exp2_fast(fmaf(__uint_as_float(sr[jj]), sl2, -mb));
+        float p1 = exp2_fast(fmaf(__uint_as_float(sr[jj + 1]), sl2, -mb));
+        if (!full) { p0 = (jj < lim) ? p0 : 0.f; p1 = (jj + 1 < lim) ? p1 : 0.f; }
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+        s4[(j >> 1) & 3] += p0 + p1;
         pk[j >> 1] = *reinterpret_cast<uint32_t*>(&h2);
       }
       *reinterpret_cast<uint4*>(prow + ((ch ^ (r_in & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
     }
+    const float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
     l_run = l_run * alpha + sum;
     m_run = mx;
     // rescale O where a row maximum moved (warp-uniform decision: the TMEM accesses are warp-wide)

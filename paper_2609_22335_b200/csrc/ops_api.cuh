@@ -145,7 +145,7 @@ inline int op_attention_run(const void* q, const void* k, const void* v, void* o
       !op_encode(&maps.m[2], vt, (int64_t)hkv * hd, tkv, tpad, hd))
     return VLA_ERR_CUDA;
   const int nbox = (hd + 63) / 64;
-  const int smem = 1024 + nbox * 128 * 128 + nbox * a.bn * 128 + hd * 128 + 128 * 128;
+  const int smem = attn_smem_bytes(hd);
   int tmem_cols = 32;
   while (tmem_cols < a.bn + hd) tmem_cols <<= 1;
   if (cudaFuncSetAttribute(vla_op_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)

@@ -338,8 +338,7 @@ class Builder {
     a.bn = 64;
     a.q_blocks = (tq + 127) / 128;
     a.scale_log2e = 1.4426950408889634f / std::sqrt((float)hd);
-    const int nbox = (hs + 63) / 64;
-    n.smem_bytes = 1024 + nbox * 128 * 128 + nbox * a.bn * 128 + hs * 128 + 128 * 128;
+    n.smem_bytes = attn_smem_bytes(hs);
     n.tmem_cols = (int)pad_to(a.bn + hs, TMEM_UNIT);
     n.n_tiles = hq * a.q_blocks;
     // tensor maps: Q rows in 128-row boxes, K rows in bn-row boxes, V^T in hs-row boxes of 64 tokens

@@ -56,6 +56,13 @@ inline int gemm_smem_bytes(int bt, bool dual, int S) {      // the epilogue park
   return 1024 + (a > b ? a : b);
 }
 
+// Shared memory of one attention tile: barrier block, Q (128 rows), one K block and one V^T block of 64 keys,
+// and the probability tile.  hs = head stride (head dim padded to a multiple of 16).
+inline int attn_smem_bytes(int hs) {
+  const int nbox = (hs + 63) / 64;
+  return 1024 + nbox * 128 * 128 + nbox * 64 * 128 + hs * 128 + 128 * 128;
+}
+
 struct GemmArgs {
   Ref A, W, W2;        // A bf16 [M,lda]; W (and W2 when dual) bf16 [N,Kp]
   Ref X;               // optional fp32 addend [M,ldx], scaled by c_x
@@ -206,7 +213,7 @@ struct Control {                 // polled words and hot counters live on separa
   unsigned long long pad2[15];
   unsigned long long tiles_done;
   unsigned long long trace_count;
-  unsigned long long dbg[14];    // scratch counters for kernel bring-up (see VLA_TILE_TIMING)
+  unsigned long long dbg[24];    // scratch counters for kernel bring-up (see VLA_TILE_TIMING)
 };
 
 enum DevError : uint32_t {
