@@ -68,14 +68,16 @@ struct KvBlock {
   int seg, kv0;
   bool valid;
 };
-__device__ __forceinline__ KvBlock kv_first(const AttnArgs& a) {
+template <typename A>
+__device__ __forceinline__ KvBlock kv_first(const A& a) {
   KvBlock b;
   b.seg = a.t0 > 0 ? 0 : 1;
   b.kv0 = 0;
   b.valid = (a.t0 > 0 || a.t1 > 0);
   return b;
 }
-__device__ __forceinline__ KvBlock kv_next(const AttnArgs& a, KvBlock b, int q_last) {
+template <typename A>
+__device__ __forceinline__ KvBlock kv_next(const A& a, KvBlock b, int q_last) {
   b.kv0 += ATTN_BN;
   const int L = b.seg == 0 ? a.t0 : a.t1;
   if (b.kv0 >= L) {
@@ -86,7 +88,13 @@ __device__ __forceinline__ KvBlock kv_next(const AttnArgs& a, KvBlock b, int q_l
   return b;
 }
 
-__device__ void tile_attention(const TileCtx& c, const AttnArgs& a, int tile) {
+__device__ void tile_attention(const TileCtx& c, const AttnArgs& a_in, int tile) {
+  // The node's arguments live in global memory; the shared-memory stores and the asm statements of the block loop
+  // would make the compiler fetch them again and again, so the ones the loop uses are copied into registers.
+  struct { int32_t k0map, v0map, k1map, v1map, t0, t1, causal, hq, hkv, hs, hd, q_blocks, qmap, tq, ldo; float scale_log2e; Ref out; } a;
+  a.k0map = a_in.k0map; a.v0map = a_in.v0map; a.k1map = a_in.k1map; a.v1map = a_in.v1map; a.t0 = a_in.t0; a.t1 = a_in.t1;
+  a.causal = a_in.causal; a.hq = a_in.hq; a.hkv = a_in.hkv; a.hs = a_in.hs; a.hd = a_in.hd; a.q_blocks = a_in.q_blocks;
+  a.qmap = a_in.qmap; a.tq = a_in.tq; a.ldo = a_in.ldo; a.scale_log2e = a_in.scale_log2e; a.out = a_in.out;
   const int warp = c.tid >> 5, lane = c.tid & 31;
   const int head = tile / a.q_blocks, qb = tile % a.q_blocks;
   const int g = (head * a.hkv) / a.hq;

@@ -317,7 +317,10 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         const bool busy = slot->busy != 0 || queued > 0;   // anything beyond the first tile is claimed ahead of need
         // early claims (for a worker that is still running) only from deep VLM queues, and never for worker 0:
         // one worker per SM always returns to the pool, so a short action-head tile is at most one tile away
-        const unsigned cand = busy ? (w == 0 ? 0u : (deep & ((1u << N_KINDS) - 1u))) : pending;
+        // worker 0 is also the SM's reserve for the action head: it takes VLM tiles only while no action-head tile is pending
+        const unsigned act_mask = ((1u << N_KINDS) - 1u) << N_KINDS;
+        const unsigned cand = busy ? (w == 0 ? 0u : (deep & ((1u << N_KINDS) - 1u)))
+                                   : ((w == 0 && ctx.policy == POLICY_TWO_PHASE && (pending & act_mask)) ? (pending & act_mask) : pending);
         const unsigned long long smask = *reinterpret_cast<volatile unsigned long long*>(&sm->smem_mask);
         const unsigned tmask = *reinterpret_cast<volatile unsigned*>(&sm->tmem_mask);
         const bool blocked = false;

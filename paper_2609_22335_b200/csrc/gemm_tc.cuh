@@ -176,7 +176,9 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   const int nkb = g.Kp / GEMM_BK;
   const int S = g.stages;
   const int a_bytes = g.bt * GEMM_BK * 2;
-  const int stage_bytes = GEMM_W_STAGE_BYTES * (g.dual ? 2 : 1) + a_bytes;
+  const bool dual = g.dual != 0;            // arguments used inside the loops, out of global memory once
+  const int bt = g.bt;
+  const int stage_bytes = GEMM_W_STAGE_BYTES * (dual ? 2 : 1) + a_bytes;
 
   uint64_t* bars = reinterpret_cast<uint64_t*>(c.smem);          // full[S], empty[S], accum
   const uint32_t bar0 = smem_u32(bars);
@@ -214,15 +216,15 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
       const uint32_t dst = stage0 + (uint32_t)(s * stage_bytes);
       tma_load_2d(dst, wmap, full_bar(s), kb * GEMM_BK, f0);
-      if (g.dual) tma_load_2d(dst + GEMM_W_STAGE_BYTES, w2map, full_bar(s), kb * GEMM_BK, f0);
-      tma_load_2d(dst + GEMM_W_STAGE_BYTES * (g.dual ? 2 : 1), amap, full_bar(s), kb * GEMM_BK, t0);
+      if (dual) tma_load_2d(dst + GEMM_W_STAGE_BYTES, w2map, full_bar(s), kb * GEMM_BK, f0);
+      tma_load_2d(dst + GEMM_W_STAGE_BYTES * (dual ? 2 : 1), amap, full_bar(s), kb * GEMM_BK, t0);
     }
     }
     __syncwarp();
   } else if (warp == 1) {
     if (lane == 0) {
     // ---------------- MMA issuer
-    const uint32_t idesc = umma_idesc_bf16(g.bt);
+    const uint32_t idesc = umma_idesc_bf16(bt);
     bool ok = true;
     for (int kb = 0; kb < nkb && ok; ++kb) {
       const int s = kb % S;
@@ -234,14 +236,14 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
 #endif
       tc_fence_after();
       const uint32_t wsm = stage0 + (uint32_t)(s * stage_bytes);
-      const uint32_t asm_ = wsm + GEMM_W_STAGE_BYTES * (g.dual ? 2 : 1);
+      const uint32_t asm_ = wsm + GEMM_W_STAGE_BYTES * (dual ? 2 : 1);
       const uint64_t wd = umma_desc_sw128(wsm), ad = umma_desc_sw128(asm_);
       const uint64_t w2d = umma_desc_sw128(wsm + GEMM_W_STAGE_BYTES);
 #pragma unroll
       for (int k = 0; k < GEMM_BK / 16; ++k) {
         const uint32_t accumulate = (kb | k) != 0 ? 1u : 0u;
         umma_bf16(tmem_d, wd + 2u * k, ad + 2u * k, idesc, accumulate);          // 16 bf16 = 32 bytes per K step
-        if (g.dual) umma_bf16(tmem_d + (uint32_t)g.bt, w2d + 2u * k, ad + 2u * k, idesc, accumulate);
+        if (dual) umma_bf16(tmem_d + (uint32_t)bt, w2d + 2u * k, ad + 2u * k, idesc, accumulate);
       }
       umma_commit(empty_bar(s));        // stage reusable once these MMAs have read it
     }
@@ -252,11 +254,13 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
     // ---------------- folded RMSNorm: row scales from the stream's per-row partial sums of squares, summed in a
     // fixed order while the main loop runs (thread j: tokens j and j + 64)
     const float* ssp = resolve<const float>(c, g.ss_in);
-    for (int tkn = c.tid - 64; tkn < g.bt; tkn += 64) {
+    const int ss_nft = g.ss_nft;
+    const float inv_d = (float)g.rs_d;
+    for (int tkn = c.tid - 64; tkn < bt; tkn += 64) {
       float ssq = 0.f;
       if (tkn < nt)
-        for (int q = 0; q < g.ss_nft; ++q) ssq += ld_act(ssp + (size_t)(t0 + tkn) * g.ss_nft + q);
-      rs_smem[tkn] = 1.0f / sqrtf(ssq / (float)g.rs_d + 1e-6f);
+        for (int q = 0; q < ss_nft; ++q) ssq += ld_act(ssp + (size_t)(t0 + tkn) * ss_nft + q);
+      rs_smem[tkn] = 1.0f / sqrtf(ssq / inv_d + 1e-6f);
     }
   }
 
@@ -316,7 +320,15 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   if (ready) {
     float* ssq_out = resolve<float>(c, g.ss_out);
     if (vec4) {
+      // the node's arguments live in global memory, which the stores below might alias as far as the compiler
+      // knows: everything the row loop needs is taken into registers first
+      const size_t ldo32 = (size_t)g.ldo32, ldo16 = (size_t)g.ldo16, ldtab = (size_t)g.ldtab, ldtab2 = (size_t)g.ldtab2;
+      const size_t ss_ld = (size_t)g.ss_out_ld;
+      const float* const tab = fok ? ptrs.tab : nullptr;
+      const float* const tab2 = fok ? ptrs.tab2 : nullptr;
+      float* const o32 = fok ? ptrs.out32 : nullptr;
       const bool skip16 = ptrs.outT != nullptr && gf >= g.t_col0;      // these columns went to V^T in phase 1
+      unsigned short* const o16 = (fok && !skip16) ? ptrs.out16 : nullptr;
       float4 vecv = make_float4(0.f, 0.f, 0.f, 0.f);
       if (ptrs.vec && fok) vecv = *reinterpret_cast<const float4*>(ptrs.vec + gf);
       // four token rows per pass; the lane's share of each row's sum of squares is left in the row's first 32
@@ -337,21 +349,19 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
             const int r = t0 + tok;
             float4 w = v[q];
             w.x += vecv.x; w.y += vecv.y; w.z += vecv.z; w.w += vecv.w;
-            if (fok && ptrs.tab) {
-              const float4 t = *reinterpret_cast<const float4*>(ptrs.tab + (size_t)r * g.ldtab + gf);
+            if (tab) {
+              const float4 t = *reinterpret_cast<const float4*>(tab + (size_t)r * ldtab + gf);
               w.x += t.x; w.y += t.y; w.z += t.z; w.w += t.w;
             }
-            if (fok && ptrs.tab2) {
-              const float4 t = *reinterpret_cast<const float4*>(ptrs.tab2 + (size_t)r * g.ldtab2 + gf);
+            if (tab2) {
+              const float4 t = *reinterpret_cast<const float4*>(tab2 + (size_t)r * ldtab2 + gf);
               w.x += t.x; w.y += t.y; w.z += t.z; w.w += t.w;
             }
-            if (fok) {
-              if (ptrs.out32) *reinterpret_cast<float4*>(ptrs.out32 + (size_t)r * g.ldo32 + gf) = w;
-              if (ptrs.out16 && !skip16) {
-                __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
-                *reinterpret_cast<uint2*>(ptrs.out16 + (size_t)r * g.ldo16 + gf) =
-                    make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
-              }
+            if (o32) *reinterpret_cast<float4*>(o32 + (size_t)r * ldo32 + gf) = w;
+            if (o16) {
+              __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+              *reinterpret_cast<uint2*>(o16 + (size_t)r * ldo16 + gf) =
+                  make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
             }
             if (ssq_out) {
               const float sq = fok ? (w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w) : 0.f;
@@ -367,7 +377,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
           float sq = 0.f;
 #pragma unroll 8
           for (int i = 0; i < 32; ++i) sq += St[(size_t)tok * GEMM_BM + ((i + lane) & 31)];   // lane order 0..31
-          ssq_out[(size_t)(t0 + tok) * g.ss_out_ld + ft] = sq;
+          ssq_out[(size_t)(t0 + tok) * ss_ld + ft] = sq;
         }
       }
     } else {
@@ -394,6 +404,13 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       }
     }
   }
+#ifdef VLA_TILE_TIMING
+  if (c.tid == 64 && g.M > 512 && c.dbg) {
+    uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    const int kind = ptrs.X ? 0 : (g.act != ACT_NONE ? 1 : (ptrs.outT ? 2 : 3));     // residual, w1, qkv, other
+    atomicAdd(c.dbg + 14 + 2 * kind, t - tt1); atomicAdd(c.dbg + 15 + 2 * kind, 1ull);
+  }
+#endif
   tc_fence_before();
   worker_sync(c);
 #ifdef VLA_TILE_TIMING

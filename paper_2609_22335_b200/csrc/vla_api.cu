@@ -637,6 +637,10 @@ int vla_get_counters(vla_ctx* c, uint64_t* tiles, uint64_t* kernel_launches, uin
     if (getenv("VLA_PRINT_DBG"))
       fprintf(stderr, "dbg: epilogue phase 1 %.2f us (sync+ptrs %.2f us), tiles with residual %llu\n", ctl.dbg[3] ? ctl.dbg[11] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3] ? ctl.dbg[13] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[12]);
     if (getenv("VLA_PRINT_DBG"))
+      fprintf(stderr, "dbg: epilogue (own warp, before the last barrier) by kind: residual %.2f us x %llu  gelu %.2f us x %llu  qkv %.2f us x %llu  other %.2f us x %llu\n",
+              ctl.dbg[15] ? ctl.dbg[14] / 1e3 / ctl.dbg[15] : 0.0, ctl.dbg[15], ctl.dbg[17] ? ctl.dbg[16] / 1e3 / ctl.dbg[17] : 0.0, ctl.dbg[17],
+              ctl.dbg[19] ? ctl.dbg[18] / 1e3 / ctl.dbg[19] : 0.0, ctl.dbg[19], ctl.dbg[21] ? ctl.dbg[20] / 1e3 / ctl.dbg[21] : 0.0, ctl.dbg[21]);
+    if (getenv("VLA_PRINT_DBG"))
       fprintf(stderr, "dbg: wait-for-claim %.2f us x %llu  wait-for-room %.2f us x %llu  wait-to-post %.2f us x %llu\n",
               ctl.dbg[6] ? ctl.dbg[5] / 1e3 / ctl.dbg[6] : 0.0, ctl.dbg[6], ctl.dbg[8] ? ctl.dbg[7] / 1e3 / ctl.dbg[8] : 0.0,
               ctl.dbg[8], ctl.dbg[10] ? ctl.dbg[9] / 1e3 / ctl.dbg[10] : 0.0, ctl.dbg[10]);
