@@ -55,29 +55,42 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
 // Pushing tiles is split in three so a whole warp can fill the entries in parallel:
 // reserve (one thread), fill (any threads, entry i of the range), commit (one thread, after a barrier).
 // The ring is sized for every tile of every frame slot, so a reservation can never overrun the head.
+// One entry = one 64-bit word: generation (12 bits, never 0 for a written entry of the current lap... the lap count + 1)
+// | node (20) | frame slot (9) | tile (12) | and the node's per-tile resource need in units so that a claim needs no
+// second load: shared memory (6) and tensor memory (5).
+constexpr int QW_NODE_BITS = 20, QW_INST_BITS = 9, QW_TILE_BITS = 12, QW_SMEM_BITS = 6, QW_TMEM_BITS = 5, QW_GEN_BITS = 12;
+static_assert(QW_NODE_BITS + QW_INST_BITS + QW_TILE_BITS + QW_SMEM_BITS + QW_TMEM_BITS + QW_GEN_BITS == 64, "queue word layout");
+__device__ __forceinline__ unsigned long long queue_gen(const DeviceCtx& ctx, unsigned long long ticket) {
+  return ((ticket >> ctx.q_shift) + 1ull) & ((1ull << QW_GEN_BITS) - 1ull);
+}
 __device__ __forceinline__ unsigned long long queue_word(const DeviceCtx& ctx, unsigned long long ticket, uint32_t inst,
-                                                         uint32_t node, uint32_t tile) {
-  const unsigned long long gen = ((ticket >> ctx.q_shift) + 1ull) & 0xFFFFull;
-  return (gen << 48) | ((unsigned long long)(tile & 0xFFFFu) << 32) | (unsigned long long)((inst << 20) | node);
+                                                         uint32_t node, uint32_t tile, uint32_t res_units) {
+  // res_units = smem units | tmem units << QW_SMEM_BITS
+  return (queue_gen(ctx, ticket) << (64 - QW_GEN_BITS)) | ((unsigned long long)res_units << (QW_NODE_BITS + QW_INST_BITS + QW_TILE_BITS)) |
+         ((unsigned long long)tile << (QW_NODE_BITS + QW_INST_BITS)) | ((unsigned long long)inst << QW_NODE_BITS) | (unsigned long long)node;
 }
 __device__ inline unsigned long long queue_reserve(const DeviceCtx& ctx, int cls, int n) {
   return atomicAdd(&ctx.queues[cls].tail, (unsigned long long)n);
 }
-__device__ inline void queue_fill(const DeviceCtx& ctx, int cls, unsigned long long base, uint32_t inst, uint32_t node, int first,
-                                  int count, int stride) {
+__device__ inline void queue_fill(const DeviceCtx& ctx, int cls, unsigned long long base, uint32_t inst, uint32_t node,
+                                  uint32_t res_units, int first, int count, int stride) {
   const unsigned long long mask = (unsigned long long)ctx.q_capacity - 1;
   QueueEntry* ent = ctx.q_entries + (size_t)cls * ctx.q_capacity;
   for (int i = first; i < count; i += stride)
-    *reinterpret_cast<volatile unsigned long long*>(ent + ((base + i) & mask)) = queue_word(ctx, base + i, inst, node, (uint32_t)i);
+    *reinterpret_cast<volatile unsigned long long*>(ent + ((base + i) & mask)) = queue_word(ctx, base + i, inst, node, (uint32_t)i, res_units);
 }
 __device__ inline void queue_commit(const DeviceCtx& ctx, int cls, int n) {
   __threadfence();
   atomicAdd(reinterpret_cast<unsigned long long*>(&ctx.queues[cls].avail), (unsigned long long)n);
 }
 // One thread pushes everything (admission of a frame's root tiles).
+__device__ __forceinline__ uint32_t node_res_units(const NodeDesc& nd) {
+  return (uint32_t)((__ldg(&nd.smem_bytes) + SMEM_UNIT - 1) / SMEM_UNIT) |
+         ((uint32_t)((__ldg(&nd.tmem_cols) + TMEM_UNIT - 1) / TMEM_UNIT) << QW_SMEM_BITS);
+}
 __device__ inline void queue_push(const DeviceCtx& ctx, int cls, uint32_t inst, uint32_t node, int n) {
   const unsigned long long base = queue_reserve(ctx, cls, n);
-  queue_fill(ctx, cls, base, inst, node, 0, n, 1);
+  queue_fill(ctx, cls, base, inst, node, node_res_units(ctx.nodes[node]), 0, n, 1);
   queue_commit(ctx, cls, n);
 }
 
@@ -91,11 +104,11 @@ __device__ inline bool queue_try_pop(const DeviceCtx& ctx, int cls, QueueEntry& 
   }
   const unsigned long long t = atomicAdd(&q->head, 1ull);
   const unsigned long long mask = (unsigned long long)ctx.q_capacity - 1;
-  const unsigned long long want = ((t >> ctx.q_shift) + 1ull) & 0xFFFFull;
+  const unsigned long long want = queue_gen(ctx, t);
   const unsigned long long* slot = ctx.q_entries + (size_t)cls * ctx.q_capacity + (t & mask);
   unsigned spins = 0;
   unsigned long long w;
-  while (((w = ld_acquire_u64(slot)) >> 48) != want) {
+  while (((w = ld_acquire_u64(slot)) >> (64 - QW_GEN_BITS)) != want) {
     if ((++spins & 63u) == 0 && gtimer() > deadline) {
       set_error(ctx, DEV_ERR_WAIT_QUEUE, cls);
       return false;
@@ -113,7 +126,7 @@ constexpr int HELD_DEPTH = 2;            // claimed tiles a worker may have wait
 
 struct ReadyItem {
   unsigned long long base;   // reserved queue range
-  uint32_t node;
+  uint32_t node, res_units;
   int n_tiles, cls;
 };
 
@@ -121,6 +134,7 @@ struct WorkerTile {
   uint32_t inst, node, tile;
   int cls;
   int smem_unit0, smem_units, tmem_unit0, tmem_units;
+  int succ_begin, succ_count, op, pad_;     // of the tile's node, filled in by the worker for the retire warp
   uint64_t t0, t1, frame;
 };
 
@@ -151,13 +165,18 @@ struct SmState {
 static_assert(sizeof(SmState) <= SM_STATE_BYTES, "SM state too large");
 
 __device__ __forceinline__ unsigned long long unit_bits(int n) { return n >= 64 ? ~0ull : ((1ull << n) - 1ull); }
+// Lowest position of `need` consecutive free units among the first `total` (bit set = in use), or -1.
+// run keeps the positions where k consecutive free units start; k doubles until it reaches `need`.
 __device__ __forceinline__ int find_free(unsigned long long mask, int need, int total) {
   if (need == 0) return 0;
   if (need > total) return -1;
-  const unsigned long long want = unit_bits(need);
-  for (int i = 0; i + need <= total; ++i)
-    if (((mask >> i) & want) == 0) return i;
-  return -1;
+  unsigned long long run = ~mask & unit_bits(total);
+  for (int k = 1; k < need;) {
+    const int step = min(k, need - k);
+    run &= run >> step;
+    k += step;
+  }
+  return run ? __ffsll((long long)run) - 1 : -1;
 }
 
 __device__ inline void write_trace(const DeviceCtx& ctx, uint32_t inst, uint32_t node, uint32_t tile, int worker, int cls,
@@ -203,34 +222,41 @@ __device__ inline void try_admit(const DeviceCtx& ctx) {
 // Global side of a finished tile: every successor node's counter (which counts its predecessors' tiles)
 // goes down by one; a counter reaching zero re-arms itself and releases that node, whose queue range is
 // reserved here and returned in `slot` for the warp to fill.
-__device__ inline void complete_tile(const DeviceCtx& ctx, uint32_t inst, uint32_t node_idx, WorkerSlot* slot) {
-  const NodeDesc& n = ctx.nodes[node_idx];
+__device__ inline void complete_tile(const DeviceCtx& ctx, const WorkerTile& f, WorkerSlot* slot) {
+  const uint32_t inst = f.inst;
   slot->n_ready = 0;
   __threadfence();
-  const int n_succ = __ldg(&n.succ_count), succ0 = __ldg(&n.succ_begin);
+  const int n_succ = f.succ_count, succ0 = f.succ_begin;      // carried by the tile's record: no load of its node here
   for (int i0 = 0; i0 < n_succ; i0 += 4) {
-    // up to four successors per pass: their counters are decremented by independent atomics in flight together
-    int s[4], left[4];
+    // up to four successors per pass: one 16-byte load each, then their counters are decremented by independent
+    // atomics in flight together
+    SuccInfo si[4];
+    int left[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) s[j] = i0 + j < n_succ ? __ldg(ctx.succ + succ0 + i0 + j) : -1;
+    for (int j = 0; j < 4; ++j) {
+      si[j].node = -1;
+      if (i0 + j < n_succ) {
+        const int4 v = __ldg(reinterpret_cast<const int4*>(ctx.succ + succ0 + i0 + j));
+        si[j].node = v.x; si[j].n_tiles = v.y; si[j].cls = v.z; si[j].n_pred = v.w;
+      }
+    }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) left[j] = s[j] >= 0 ? atomicSub(ctx.dep_count + (size_t)inst * ctx.n_nodes + s[j], 1) - 1 : 1;
+    for (int j = 0; j < 4; ++j) left[j] = si[j].node >= 0 ? atomicSub(ctx.dep_count + (size_t)inst * ctx.n_nodes + si[j].node, 1) - 1 : 1;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       if (left[j] != 0) continue;
-      const NodeDesc& sn = ctx.nodes[s[j]];
-      const int sn_tiles = __ldg(&sn.n_tiles), sn_cls = __ldg(&sn.cls);
-      ctx.dep_count[(size_t)inst * ctx.n_nodes + s[j]] = __ldg(&sn.n_pred);
+      ctx.dep_count[(size_t)inst * ctx.n_nodes + si[j].node] = si[j].n_pred;
       if (slot->n_ready < MAX_READY) {
         ReadyItem& it = slot->ready[slot->n_ready++];
-        it.base = queue_reserve(ctx, sn_cls, sn_tiles);
-        it.node = (uint32_t)s[j]; it.n_tiles = sn_tiles; it.cls = sn_cls;
+        it.base = queue_reserve(ctx, si[j].cls, si[j].n_tiles);
+        it.node = (uint32_t)si[j].node; it.n_tiles = si[j].n_tiles; it.cls = si[j].cls;
+        it.res_units = node_res_units(ctx.nodes[si[j].node]);
       } else {
-        queue_push(ctx, sn_cls, inst, (uint32_t)s[j], sn_tiles);
+        queue_push(ctx, si[j].cls, inst, (uint32_t)si[j].node, si[j].n_tiles);
       }
     }
   }
-  if (__ldg(&n.op) == OP_EMIT) atomicSub(&ctx.control->ctrl, 1u);
+  if (f.op == OP_EMIT) atomicSub(&ctx.control->ctrl, 1u);
 }
 
 // ------------------------------------------------------------------ the two service warps of an SM
@@ -260,7 +286,7 @@ __device__ inline void retire_loop(const DeviceCtx& ctx, SmState* sm, int n_work
       have_fin = true;
       const WorkerTile& f = slot->fin;
       write_trace(ctx, f.inst, f.node, f.tile, lane, f.cls, f.frame, f.t0, f.t1);
-      complete_tile(ctx, f.inst, f.node, slot);
+      complete_tile(ctx, f, slot);
     } else if (serving) {
       slot->n_ready = 0;
     }
@@ -271,7 +297,7 @@ __device__ inline void retire_loop(const DeviceCtx& ctx, SmState* sm, int n_work
         const int nr = sm->slot[w].n_ready;
         for (int i = 0; i < nr; ++i) {
           const ReadyItem it = sm->slot[w].ready[i];
-          queue_fill(ctx, it.cls, it.base, sm->slot[w].fin.inst, it.node, lane, it.n_tiles, 32);
+          queue_fill(ctx, it.cls, it.base, sm->slot[w].fin.inst, it.node, it.res_units, lane, it.n_tiles, 32);
         }
       }
       __syncwarp();
@@ -350,11 +376,12 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
       QueueEntry e;
       if (queue_try_pop(ctx, want, e, gtimer() + ctx.wait_limit_ns)) {
         WorkerTile& h = slot->held[slot->held_tail % HELD_DEPTH];
-        h.inst = (uint32_t)(e & 0xFFFFFFFFull) >> 20; h.node = (uint32_t)e & 0xFFFFFu; h.tile = (uint32_t)(e >> 32) & 0xFFFFu;
+        h.node = (uint32_t)e & ((1u << QW_NODE_BITS) - 1u);
+        h.inst = (uint32_t)(e >> QW_NODE_BITS) & ((1u << QW_INST_BITS) - 1u);
+        h.tile = (uint32_t)(e >> (QW_NODE_BITS + QW_INST_BITS)) & ((1u << QW_TILE_BITS) - 1u);
+        h.smem_units = (int)((e >> (QW_NODE_BITS + QW_INST_BITS + QW_TILE_BITS)) & ((1u << QW_SMEM_BITS) - 1u));
+        h.tmem_units = (int)((e >> (QW_NODE_BITS + QW_INST_BITS + QW_TILE_BITS + QW_SMEM_BITS)) & ((1u << QW_TMEM_BITS) - 1u));
         h.cls = want;
-        const NodeDesc& nd = ctx.nodes[h.node];                 // the program is immutable: read-only cached loads
-        h.smem_units = (__ldg(&nd.smem_bytes) + SMEM_UNIT - 1) / SMEM_UNIT;
-        h.tmem_units = (__ldg(&nd.tmem_cols) + TMEM_UNIT - 1) / TMEM_UNIT;
         __threadfence_block();
         slot->held_tail = slot->held_tail + 1;      // the worker takes it as soon as it is free
         progressed = true;
@@ -365,7 +392,7 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     }
     // ---- admission, exit and watchdog (lane 0 decides, every few rounds)
     int verdict = 0;   // 1 = leave
-    if (lane == 0 && ((iter & 7u) == 0 || !progressed)) {
+    if (lane == 0 && (iter & 3u) == 0) {              // several dependent round trips: not on every poll
       if (ld_volatile_u32(&ctl->error) != 0u || ld_volatile_u32(&ctl->stop) != 0u) verdict = 1;
       const unsigned cw = ld_volatile_u32(&ctl->ctrl);
       if (cw & CTRL_EXITING) verdict = 1;
@@ -400,7 +427,7 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         break;
       }
     }
-    if (!__any_sync(0xffffffffu, progressed)) { __nanosleep(nap); if (nap < 600) nap += 60; } else nap = 60;
+    if (!__any_sync(0xffffffffu, progressed)) { __nanosleep(nap); if (nap < 240) nap += 60; } else nap = 60;
   }
 }
 
@@ -524,7 +551,10 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
       tc.amap_base = ctx.n_weight_tmaps + (int)cmd.inst * ctx.n_act_tmaps;
       const uint64_t t0 = gtimer();
       tc.deadline = t0 + ctx.wait_limit_ns;
-      const uint64_t frame = *reinterpret_cast<const volatile uint64_t*>(ctx.inst_frame + cmd.inst);
+      // the frame id is only needed by the emit tile and by the trace
+      const int n_op = __ldg(&n.op);
+      const uint64_t frame = (ctx.trace_capacity != 0 || n_op == OP_EMIT)
+                                 ? *reinterpret_cast<const volatile uint64_t*>(ctx.inst_frame + cmd.inst) : 0ull;
       if (cmd.t0 == 1) run_tile(ctx, tc, n, (int)cmd.tile, (int)cmd.inst, frame);
       asm volatile("fence.proxy.async;" ::: "memory");   // outputs may be read by TMA on another SM
       asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
@@ -535,8 +565,9 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
           if (cmd.smem_units) atomicAnd(&sm->smem_mask, ~(unit_bits(cmd.smem_units) << cmd.smem_unit0));
           if (cmd.tmem_units) atomicAnd(&sm->tmem_mask, ~(unsigned)(unit_bits(cmd.tmem_units) << cmd.tmem_unit0));
         }
-        atomicSub(&sm->pick.cta_count[cmd.cls], 1);
-        for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[cmd.cls * 3 + x]);
+        WorkerTile d = cmd;
+        d.t0 = t0; d.t1 = t1; d.frame = frame;
+        d.succ_begin = __ldg(&n.succ_begin); d.succ_count = __ldg(&n.succ_count); d.op = n_op;
         unsigned naps = 0;
         while (slot->done_state != 0) {
           __nanosleep(40);
@@ -545,12 +576,12 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
 #ifdef VLA_TILE_TIMING
         atomicAdd(ctl->dbg + 9, gtimer() - t1); atomicAdd(ctl->dbg + 10, 1ull);
 #endif
-        WorkerTile d = cmd;
-        d.t0 = t0; d.t1 = t1; d.frame = frame;
         slot->done = d;
         __threadfence();       // the tile's writes (all threads, ordered by the barrier) before the completion is seen
         slot->done_state = 1;
         slot->busy = 0;
+        atomicSub(&sm->pick.cta_count[cmd.cls], 1);    // the pick's view of this SM, after the completion is on its way
+        for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[cmd.cls * 3 + x]);
       }
     }
     if (wt == 0) atomicAdd(&ctl->tiles_done, tiles);

@@ -276,6 +276,9 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
 #ifdef VLA_TILE_TIMING
   uint64_t tt1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt1));
 #endif
+#ifdef VLA_TILE_TIMING
+  long long ck[6]; ck[0] = clock64();
+#endif
   GemmPtrs ptrs = gemm_ptrs(c, g);
   float* St = reinterpret_cast<float*>(c.smem + GEMM_BAR_BYTES);   // [bt][128] fp32
   const bool vec4 = (g.N % 4 == 0) && (!ptrs.X || g.ldx % 4 == 0) && (!ptrs.tab || g.ldtab % 4 == 0) &&
@@ -292,6 +295,9 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
     cp_async_wait_all();
   }
   if (g.rs_d > 0 || x_staged) worker_sync(c);     // row scales written by warps 2 and 3; residual rows landed
+#ifdef VLA_TILE_TIMING
+  ck[1] = clock64();
+#endif
   if (ready) {
     Phase1Args p1;
     p1.St = St; p1.rs = g.rs_d > 0 ? rs_smem : nullptr; p1.c_acc = g.c_acc; p1.c_x = g.c_x; p1.x_staged = x_staged;
@@ -309,13 +315,13 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       else gemm_phase1<ACT_NONE, false>(p1);
     }
   }
+#ifdef VLA_TILE_TIMING
+  ck[2] = clock64();
+#endif
   worker_sync(c);
 #ifdef VLA_TILE_TIMING
-  if (c.tid == 64 && g.M > 512 && c.dbg) {
-    uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    atomicAdd(c.dbg + 11, t - tt1);
-    if (ptrs.X) { atomicAdd(c.dbg + 12, 1ull); }
-  }
+  ck[3] = clock64();
+  uint64_t tt2; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt2));
 #endif
   if (ready) {
     float* ssq_out = resolve<float>(c, g.ss_out);
@@ -370,6 +376,9 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
           }
         }
       }
+#ifdef VLA_TILE_TIMING
+      ck[4] = clock64();
+#endif
       if (ssq_out) {
         __syncwarp();
         const int tok = warp + 4 * lane;                 // this lane's row: slot `lane` of this warp
@@ -409,6 +418,14 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
     uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     const int kind = ptrs.X ? 0 : (g.act != ACT_NONE ? 1 : (ptrs.outT ? 2 : 3));     // residual, w1, qkv, other
     atomicAdd(c.dbg + 14 + 2 * kind, t - tt1); atomicAdd(c.dbg + 15 + 2 * kind, 1ull);
+    atomicAdd(c.dbg + 11, tt2 - tt1);
+    if (ptrs.X) { atomicAdd(c.dbg + 12, 1ull); }
+    ck[5] = clock64();
+    if (kind == 0 || kind == 2) {
+      const int b = kind == 0 ? 24 : 30;
+      for (int i = 0; i < 5; ++i) atomicAdd(c.dbg + b + i, (unsigned long long)(ck[i + 1] - ck[i]));
+      atomicAdd(c.dbg + b + 5, 1ull);
+    }
   }
 #endif
   tc_fence_before();

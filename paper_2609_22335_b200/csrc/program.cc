@@ -963,7 +963,7 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   p.zero_bytes_begin = 0;   // the whole arena starts zeroed: weight padding rows and columns rely on it
   p.off_nodes = place(sizeof(NodeDesc) * p.nodes.size());
   p.off_init_nodes = place(sizeof(NodeDesc) * p.init_program.size());
-  p.off_succ = place(sizeof(int32_t) * std::max<size_t>(p.succ.size(), 1));
+  p.off_succ = place(sizeof(SuccInfo) * std::max<size_t>(p.succ.size(), 1));
   p.off_roots = place(sizeof(int32_t) * std::max<size_t>(p.roots.size(), 1));
   p.off_classes = place(sizeof(ClassInfo) * N_CLASSES);
   p.off_control = place(sizeof(Control));

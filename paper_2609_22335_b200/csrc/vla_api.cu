@@ -322,6 +322,13 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
   for (auto& n : p.nodes) c->max_node_smem = std::max(c->max_node_smem, n.smem_bytes);
   for (auto& n : p.init_program) c->max_node_smem = std::max(c->max_node_smem, n.smem_bytes);
   if (c->max_node_smem > c->dyn_smem - SM_STATE_BYTES) return fail(c, VLA_ERR_INVALID, "a tile needs more shared memory than an SM has");
+  // field widths of a queue entry (one 64-bit word)
+  if (p.nodes.size() >= (1u << QW_NODE_BITS) || p.n_inst > (1 << QW_INST_BITS))
+    return fail(c, VLA_ERR_INVALID, "tile program too large for the queue entry layout (nodes < 2^20, streams x ring depth <= 512)");
+  for (auto& n : p.nodes)
+    if (n.n_tiles > (1 << QW_TILE_BITS) || (n.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT >= (1 << QW_SMEM_BITS) ||
+        (n.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT >= (1 << QW_TMEM_BITS))
+      return fail(c, VLA_ERR_INVALID, "a node has more tiles or needs more memory than a queue entry can describe");
   CU(cudaFuncSetAttribute(vla_node_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, std::max(c->max_node_smem, 1024)));
   CU(cudaStreamCreateWithFlags(&c->scopy, cudaStreamNonBlocking));
   CU(cudaEventCreateWithFlags(&c->ev_kernel, cudaEventDisableTiming));
@@ -332,7 +339,14 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
   CU(cudaMemcpy(at<char>(c, p.off_nodes), p.nodes.data(), sizeof(NodeDesc) * p.nodes.size(), cudaMemcpyHostToDevice));
   if (!p.init_program.empty())
     CU(cudaMemcpy(at<char>(c, p.off_init_nodes), p.init_program.data(), sizeof(NodeDesc) * p.init_program.size(), cudaMemcpyHostToDevice));
-  if (!p.succ.empty()) CU(cudaMemcpy(at<char>(c, p.off_succ), p.succ.data(), 4 * p.succ.size(), cudaMemcpyHostToDevice));
+  if (!p.succ.empty()) {
+    std::vector<SuccInfo> si(p.succ.size());
+    for (size_t i = 0; i < si.size(); ++i) {
+      const NodeDesc& sn = p.nodes[p.succ[i]];
+      si[i] = SuccInfo{p.succ[i], sn.n_tiles, sn.cls, sn.n_pred};
+    }
+    CU(cudaMemcpy(at<char>(c, p.off_succ), si.data(), sizeof(SuccInfo) * si.size(), cudaMemcpyHostToDevice));
+  }
   CU(cudaMemcpy(at<char>(c, p.off_roots), p.roots.data(), 4 * p.roots.size(), cudaMemcpyHostToDevice));
   CU(cudaMemcpy(at<char>(c, p.off_classes), p.classes, sizeof(ClassInfo) * N_CLASSES, cudaMemcpyHostToDevice));
   {
@@ -368,7 +382,7 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
   std::memset(&x, 0, sizeof x);
   x.arena = c->arena;
   x.nodes = at<NodeDesc>(c, p.off_nodes);
-  x.succ = at<int32_t>(c, p.off_succ);
+  x.succ = at<SuccInfo>(c, p.off_succ);
   x.classes = at<ClassInfo>(c, p.off_classes);
   x.control = at<Control>(c, p.off_control);
   x.queues = at<TileQueue>(c, p.off_queues);
@@ -640,6 +654,12 @@ int vla_get_counters(vla_ctx* c, uint64_t* tiles, uint64_t* kernel_launches, uin
       fprintf(stderr, "dbg: epilogue (own warp, before the last barrier) by kind: residual %.2f us x %llu  gelu %.2f us x %llu  qkv %.2f us x %llu  other %.2f us x %llu\n",
               ctl.dbg[15] ? ctl.dbg[14] / 1e3 / ctl.dbg[15] : 0.0, ctl.dbg[15], ctl.dbg[17] ? ctl.dbg[16] / 1e3 / ctl.dbg[17] : 0.0, ctl.dbg[17],
               ctl.dbg[19] ? ctl.dbg[18] / 1e3 / ctl.dbg[19] : 0.0, ctl.dbg[19], ctl.dbg[21] ? ctl.dbg[20] / 1e3 / ctl.dbg[21] : 0.0, ctl.dbg[21]);
+    if (getenv("VLA_PRINT_DBG"))
+      for (int b = 24; b <= 30; b += 6)
+        if (ctl.dbg[b + 5])
+          fprintf(stderr, "dbg: epilogue clocks (%s): ptrs+stage+sync %.0f  phase1 %.0f  sync %.0f  phase2 rows %.0f  row sums+rest %.0f (x %llu)\n",
+                  b == 24 ? "residual" : "qkv", (double)ctl.dbg[b] / ctl.dbg[b + 5], (double)ctl.dbg[b + 1] / ctl.dbg[b + 5],
+                  (double)ctl.dbg[b + 2] / ctl.dbg[b + 5], (double)ctl.dbg[b + 3] / ctl.dbg[b + 5], (double)ctl.dbg[b + 4] / ctl.dbg[b + 5], ctl.dbg[b + 5]);
     if (getenv("VLA_PRINT_DBG"))
       fprintf(stderr, "dbg: wait-for-claim %.2f us x %llu  wait-for-room %.2f us x %llu  wait-to-post %.2f us x %llu\n",
               ctl.dbg[6] ? ctl.dbg[5] / 1e3 / ctl.dbg[6] : 0.0, ctl.dbg[6], ctl.dbg[8] ? ctl.dbg[7] / 1e3 / ctl.dbg[8] : 0.0,

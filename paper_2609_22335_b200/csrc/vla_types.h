@@ -213,7 +213,7 @@ struct Control {                 // polled words and hot counters live on separa
   unsigned long long pad2[15];
   unsigned long long tiles_done;
   unsigned long long trace_count;
-  unsigned long long dbg[24];    // scratch counters for kernel bring-up (see VLA_TILE_TIMING)
+  unsigned long long dbg[40];    // scratch counters for kernel bring-up (see VLA_TILE_TIMING)
 };
 
 enum DevError : uint32_t {
@@ -222,10 +222,13 @@ enum DevError : uint32_t {
 };
 
 // Everything a kernel needs, passed by value.
+// One successor edge as the retire path reads it: everything needed to release the node in one 16-byte load.
+struct SuccInfo { int32_t node, n_tiles, cls, n_pred; };
+
 struct DeviceCtx {
   char* arena;
   const NodeDesc* nodes;
-  const int32_t* succ;
+  const SuccInfo* succ;
   const ClassInfo* classes;
   Control* control;
   TileQueue* queues;             // [N_CLASSES]
