@@ -121,6 +121,7 @@ __device__ inline bool queue_try_pop(const DeviceCtx& ctx, int cls, QueueEntry& 
 // ------------------------------------------------------------------ per-SM state of the persistent kernel
 constexpr int MAX_READY = 6;
 constexpr int DISPATCH_THREADS = 64;     // two service warps per SM (claim, retire), after the worker groups
+constexpr int ACT_BACKLOG_MIN = 128;    // action-head tiles waiting from which on a second worker per SM serves the head first
 constexpr int PREFETCH_MIN_AVAIL = 64;   // tiles are claimed ahead of need only from queues at least this deep
 constexpr int HELD_DEPTH = 2;            // claimed tiles a worker may have waiting
 
@@ -146,7 +147,8 @@ struct WorkerSlot {
   volatile int done_state;       // 0 empty, 1 finished tile posted for the retire warp
   volatile int busy;             // the worker is running a tile (set and cleared by the worker)
   int pad_;
-  WorkerTile done, fin, held[HELD_DEPTH];
+  volatile unsigned prio_tail, prio_head;   // one-deep slot for an action-head tile that goes ahead of the held VLM tiles
+  WorkerTile done, fin, held[HELD_DEPTH], prio;
   int n_ready;
   ReadyItem ready[MAX_READY];
 };
@@ -326,7 +328,7 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     group[c] = ctx.classes[c].group;
   }
   uint64_t idle_start = 0, last_progress = gtimer();
-  unsigned iter = 0, nap = 60;
+  unsigned iter = 0, nap = 60, lost = 0;
   bool leaving = false;
 
   for (;;) {
@@ -335,18 +337,43 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     long long av = lane < N_CLASSES ? ld_volatile_s64(&ctx.queues[lane].avail) : 0;
     const unsigned pending = __ballot_sync(0xffffffffu, av > 0) & ((1u << N_CLASSES) - 1u);
     const unsigned deep = __ballot_sync(0xffffffffu, av >= PREFETCH_MIN_AVAIL) & ((1u << N_CLASSES) - 1u);
+    // committed action-head tiles nobody has claimed yet, over the head's classes: its backlog.  While it is long,
+    // a second worker of the SM joins worker 0 as reserve for the head.
+    long long act_av = (lane >= N_KINDS && lane < N_CLASSES && av > 0) ? av : 0;
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) act_av += __shfl_xor_sync(0xffffffffu, act_av, o);
+    const bool act_backlog = __shfl_sync(0xffffffffu, act_av, 0) >= ACT_BACKLOG_MIN && ctx.policy == POLICY_TWO_PHASE;
     // ---- choose, lane by lane, which class each worker claims from
     int want = -1;
+    bool to_prio = false;
+    const unsigned avoid = lost;      // the class this lane just lost a race for: other SMs drained it
+    lost = 0;
     for (int w = 0; w < n_workers; ++w) {
       const unsigned queued = serving ? slot->held_tail - slot->held_head : 0u;
+#ifdef PRIO_SLOT
+      const unsigned pq = serving ? slot->prio_tail - slot->prio_head : 0u;
+      if (lane == w && !leaving && (queued < (unsigned)HELD_DEPTH || pq == 0u)) {
+        const unsigned act_mask = ((1u << N_KINDS) - 1u) << N_KINDS;
+        const bool busy = slot->busy != 0 || queued > 0 || pq > 0;
+        const bool head_pending = ctx.policy == POLICY_TWO_PHASE && (pending & act_mask & ~avoid) != 0u;
+        unsigned cand;
+        if (!busy) cand = head_pending ? (pending & act_mask) : pending;          // a free worker serves the head first
+        else if (pq == 0u && head_pending) { cand = pending & act_mask; to_prio = true; }   // ahead of the held VLM tiles
+        else if (queued < (unsigned)HELD_DEPTH) cand = deep & ((1u << N_KINDS) - 1u);
+        else cand = 0u;
+        (void)act_backlog;
+#else
       if (lane == w && !leaving && queued < (unsigned)HELD_DEPTH) {
         const bool busy = slot->busy != 0 || queued > 0;   // anything beyond the first tile is claimed ahead of need
-        // early claims (for a worker that is still running) only from deep VLM queues, and never for worker 0:
-        // one worker per SM always returns to the pool, so a short action-head tile is at most one tile away
-        // worker 0 is also the SM's reserve for the action head: it takes VLM tiles only while no action-head tile is pending
+        // early claims (for a worker that is still running) only from deep VLM queues;
+        // worker 0 is the SM's reserve for the action head: nothing is claimed ahead for it (it returns to the pool
+        // when its tile ends) and it takes VLM tiles only while no action-head tile is pending
         const unsigned act_mask = ((1u << N_KINDS) - 1u) << N_KINDS;
-        const unsigned cand = busy ? (w == 0 ? 0u : (deep & ((1u << N_KINDS) - 1u)))
-                                   : ((w == 0 && ctx.policy == POLICY_TWO_PHASE && (pending & act_mask)) ? (pending & act_mask) : pending);
+        const bool reserve = w == 0 || (w == 1 && act_backlog);
+        const bool head_first = reserve && ctx.policy == POLICY_TWO_PHASE && (pending & act_mask & ~avoid) != 0u;
+        unsigned cand = busy ? (reserve ? 0u : (deep & ((1u << N_KINDS) - 1u))) : (head_first ? (pending & act_mask) : pending);
+#endif
+        cand &= ~avoid;
         const unsigned long long smask = *reinterpret_cast<volatile unsigned long long*>(&sm->smem_mask);
         const unsigned tmask = *reinterpret_cast<volatile unsigned*>(&sm->tmem_mask);
         const bool blocked = false;
@@ -375,7 +402,7 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     if (want >= 0) {
       QueueEntry e;
       if (queue_try_pop(ctx, want, e, gtimer() + ctx.wait_limit_ns)) {
-        WorkerTile& h = slot->held[slot->held_tail % HELD_DEPTH];
+        WorkerTile& h = to_prio ? slot->prio : slot->held[slot->held_tail % HELD_DEPTH];
         h.node = (uint32_t)e & ((1u << QW_NODE_BITS) - 1u);
         h.inst = (uint32_t)(e >> QW_NODE_BITS) & ((1u << QW_INST_BITS) - 1u);
         h.tile = (uint32_t)(e >> (QW_NODE_BITS + QW_INST_BITS)) & ((1u << QW_TILE_BITS) - 1u);
@@ -383,11 +410,13 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         h.tmem_units = (int)((e >> (QW_NODE_BITS + QW_INST_BITS + QW_TILE_BITS + QW_SMEM_BITS)) & ((1u << QW_TMEM_BITS) - 1u));
         h.cls = want;
         __threadfence_block();
-        slot->held_tail = slot->held_tail + 1;      // the worker takes it as soon as it is free
+        if (to_prio) slot->prio_tail = slot->prio_tail + 1;
+        else slot->held_tail = slot->held_tail + 1;      // the worker takes it as soon as it is free
         progressed = true;
       } else {                                         // lost the race: undo the count
         atomicSub(&sm->pick.cta_count[want], 1);
         for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[want * 3 + x]);
+        lost = 1u << want;                             // look elsewhere in the next round, which follows at once
       }
     }
     // ---- admission, exit and watchdog (lane 0 decides, every few rounds)
@@ -419,7 +448,8 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     if (verdict) leaving = true;
     if (leaving) {
       // stop claiming; once every worker is idle and nothing is posted, send them home
-      const bool quiet = !serving || (slot->busy == 0 && slot->done_state == 0 && slot->held_tail == slot->held_head);
+      const bool quiet = !serving || (slot->busy == 0 && slot->done_state == 0 && slot->held_tail == slot->held_head &&
+                                      slot->prio_tail == slot->prio_head);
       if (__all_sync(0xffffffffu, quiet)) {
         if (serving) { __threadfence_block(); slot->leave = 1; }
         __syncwarp();
@@ -427,7 +457,7 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         break;
       }
     }
-    if (!__any_sync(0xffffffffu, progressed)) { __nanosleep(nap); if (nap < 240) nap += 60; } else nap = 60;
+    if (!__any_sync(0xffffffffu, progressed || lost != 0u)) { __nanosleep(nap); if (nap < 240) nap += 60; } else nap = 60;
   }
 }
 
@@ -457,6 +487,7 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
     sm->quit = 0;
     for (int w = 0; w < MAX_WORKERS; ++w) {
       sm->slot[w].held_tail = 0; sm->slot[w].held_head = 0; sm->slot[w].leave = 0; sm->slot[w].done_state = 0;
+      sm->slot[w].prio_tail = 0; sm->slot[w].prio_head = 0;
       sm->slot[w].busy = 0;
       sm->slot[w].n_ready = 0;
     }
@@ -487,6 +518,7 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
         const uint64_t tw0 = gtimer();
 #endif
         for (;;) {
+          if (slot->prio_tail != slot->prio_head) { st = 3; break; }
           if (slot->held_tail != slot->held_head) { st = 1; break; }
           if (slot->leave) { st = 2; break; }
           __nanosleep(naps < 64 ? 20 : 100);
@@ -497,11 +529,12 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
         atomicAdd(ctl->dbg + 5, tw1 - tw0); atomicAdd(ctl->dbg + 6, 1ull);
 #endif
         WorkerTile& cur = sm->cur[worker];
-        if (st == 1) {
-          cur = slot->held[slot->held_head % HELD_DEPTH];
+        if (st == 1 || st == 3) {
+          cur = st == 3 ? slot->prio : slot->held[slot->held_head % HELD_DEPTH];
           slot->busy = 1;
           __threadfence_block();
-          slot->held_head = slot->held_head + 1;   // the claim warp may refill the slot
+          if (st == 3) slot->prio_head = slot->prio_head + 1;
+          else slot->held_head = slot->held_head + 1;   // the claim warp may refill the slot
           const uint64_t lim = gtimer() + ctx.wait_limit_ns;
           bool ok = false;
           for (unsigned spin = 0;; ++spin) {

@@ -113,6 +113,16 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 // Epilogue phase 1 (thread = output feature, the TMEM lane it owns): read the accumulators 16 token columns at a
 // time, apply the row scale and the activation, and park the values in shared memory as [token][feature]; a
 // feature of the V^T part of a q|k|v projection is written from here, 16 consecutive tokens per store pair.
@@ -124,14 +134,23 @@ struct Phase1Args {
 template <int ACT, bool DUAL>
 __device__ __forceinline__ void gemm_phase1(const Phase1Args& p) {
   for (int c0 = 0; c0 < p.nt; c0 += 16) {
-    float a[16], b[16], v[16];
+    float a[16], b[16], v[16], sc[16];
     tmem_ld16(p.lane_base + (uint32_t)c0, a);
     if (DUAL) tmem_ld16(p.lane_base + (uint32_t)(p.bt + c0), b);
+    if (p.rs) {                                        // 16 row scales in four broadcast 16-byte loads
+#pragma unroll
+      for (int j = 0; j < 16; j += 4) {
+        const float4 r4 = *reinterpret_cast<const float4*>(p.rs + c0 + j);
+        sc[j] = r4.x; sc[j + 1] = r4.y; sc[j + 2] = r4.z; sc[j + 3] = r4.w;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) sc[j] = 1.0f;
+    }
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      const float sc = p.rs ? p.rs[c0 + j] : 1.0f;
-      float t = apply_act_t<ACT>(a[j] * sc);
-      if (DUAL) t *= b[j] * sc;
+      float t = apply_act_t<ACT>(a[j] * sc[j]);
+      if (DUAL) t *= b[j] * sc[j];
       v[j] = t * p.c_acc;
     }
     if (p.outT_row) {
@@ -165,6 +184,63 @@ __device__ __forceinline__ void gemm_phase1(const Phase1Args& p) {
   }
 }
 
+// Epilogue phase 2, rows of the staged tile (warp = token row, lane = four consecutive features).  A template
+// flag that is false removes that output or addend statically; one that is true is still checked per lane (a
+// lane beyond the last feature, or one whose columns went to V^T, has a null pointer).  Branches cost a lone warp
+// dearly, so the common shapes get straight-line code.
+struct Phase2Args {
+  const float* tab; const float* tab2; float* o32; unsigned short* o16; float* St;
+  float4 vecv;
+  size_t ldo32, ldo16, ldtab, ldtab2;
+  int nt, t0, warp, lane, gf;
+  bool fok, ss;
+};
+template <bool TAB, bool O32, bool O16, bool SS>
+__device__ __forceinline__ void gemm_phase2_row(const Phase2Args& p, int tok, float4 w) {
+  const int r = p.t0 + tok;
+  if (TAB) {
+    w.x += p.vecv.x; w.y += p.vecv.y; w.z += p.vecv.z; w.w += p.vecv.w;
+    if (p.tab) {
+      const float4 t = *reinterpret_cast<const float4*>(p.tab + (size_t)r * p.ldtab + p.gf);
+      w.x += t.x; w.y += t.y; w.z += t.z; w.w += t.w;
+    }
+    if (p.tab2) {
+      const float4 t = *reinterpret_cast<const float4*>(p.tab2 + (size_t)r * p.ldtab2 + p.gf);
+      w.x += t.x; w.y += t.y; w.z += t.z; w.w += t.w;
+    }
+  }
+  if (O32 && p.o32) *reinterpret_cast<float4*>(p.o32 + (size_t)r * p.ldo32 + p.gf) = w;
+  if (O16) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+    if (p.o16)
+      *reinterpret_cast<uint2*>(p.o16 + (size_t)r * p.ldo16 + p.gf) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+  }
+  if (SS && p.ss) {
+    // the lane's share of the row's sum of squares, parked in the row's first 32 words at a position rotated by
+    // the row's slot so that the final per-row additions run without bank conflicts
+    const float sq = p.fok ? (w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w) : 0.f;
+    p.St[(size_t)tok * GEMM_BM + ((p.lane + (tok >> 2)) & 31)] = sq;
+  }
+}
+template <bool TAB, bool O32, bool O16, bool SS>
+__device__ __forceinline__ void gemm_phase2_rows(const Phase2Args& p) {
+  constexpr int RP = 4;                              // token rows per pass
+  int tok0 = p.warp;
+  for (; tok0 + 4 * (RP - 1) < p.nt; tok0 += 4 * RP) {   // full passes: no per-row bound checks
+    float4 v[RP];
+#pragma unroll
+    for (int q = 0; q < RP; ++q) v[q] = *reinterpret_cast<const float4*>(p.St + (size_t)(tok0 + 4 * q) * GEMM_BM + 4 * p.lane);
+    if (SS) __syncwarp();                            // every lane has its part of the rows before partial sums overwrite them
+#pragma unroll
+    for (int q = 0; q < RP; ++q) gemm_phase2_row<TAB, O32, O16, SS>(p, tok0 + 4 * q, v[q]);
+  }
+  for (; tok0 < p.nt; tok0 += 4) {                   // ragged tail, one row at a time
+    const float4 v = *reinterpret_cast<const float4*>(p.St + (size_t)tok0 * GEMM_BM + 4 * p.lane);
+    if (SS) __syncwarp();
+    gemm_phase2_row<TAB, O32, O16, SS>(p, tok0, v);
+  }
+}
+
 constexpr int GEMM_BAR_BYTES = 1024;   // barrier block at the head of the slab (keeps the stages 1024-byte aligned)
 constexpr int GEMM_W_STAGE_BYTES = GEMM_BM * GEMM_BK * 2;
 
@@ -194,6 +270,12 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   }
   worker_sync(c);
 
+  // epilogue pointers and shape facts are resolved now, so their loads overlap the main loop
+  const GemmPtrs ptrs = gemm_ptrs(c, g);
+  const bool vec4 = (g.N % 4 == 0) && (!ptrs.X || g.ldx % 4 == 0) && (!ptrs.tab || g.ldtab % 4 == 0) &&
+                    (!ptrs.tab2 || g.ldtab2 % 4 == 0) && (!ptrs.out32 || g.ldo32 % 4 == 0) && (!ptrs.out16 || g.ldo16 % 4 == 0);
+  const int gf = f0 + 4 * lane;            // epilogue phase 2: this lane's four consecutive features
+  const bool fok = gf < g.N;
   const uint32_t tmem_d = c.tmem;                 // accumulator columns [0, bt) (and [bt, 2 bt) when dual)
   float* rs_smem = reinterpret_cast<float*>(c.smem + 256);       // [bt] row scales, inside the barrier block
 #ifdef VLA_TILE_TIMING
@@ -279,12 +361,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
 #ifdef VLA_TILE_TIMING
   long long ck[6]; ck[0] = clock64();
 #endif
-  GemmPtrs ptrs = gemm_ptrs(c, g);
   float* St = reinterpret_cast<float*>(c.smem + GEMM_BAR_BYTES);   // [bt][128] fp32
-  const bool vec4 = (g.N % 4 == 0) && (!ptrs.X || g.ldx % 4 == 0) && (!ptrs.tab || g.ldtab % 4 == 0) &&
-                    (!ptrs.tab2 || g.ldtab2 % 4 == 0) && (!ptrs.out32 || g.ldo32 % 4 == 0) && (!ptrs.out16 || g.ldo16 % 4 == 0);
-  const int gf = f0 + 4 * lane;            // phase 2: this lane's four consecutive features
-  const bool fok = gf < g.N;
   // The residual rows of this tile start their way into the staging area now (asynchronous 16-byte copies
   // through L2, no registers held), so their latency overlaps the accumulator read-out.
   const bool x_staged = vec4 && ptrs.X != nullptr;
@@ -335,47 +412,16 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       float* const o32 = fok ? ptrs.out32 : nullptr;
       const bool skip16 = ptrs.outT != nullptr && gf >= g.t_col0;      // these columns went to V^T in phase 1
       unsigned short* const o16 = (fok && !skip16) ? ptrs.out16 : nullptr;
-      float4 vecv = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (ptrs.vec && fok) vecv = *reinterpret_cast<const float4*>(ptrs.vec + gf);
-      // four token rows per pass; the lane's share of each row's sum of squares is left in the row's first 32
-      // words (rotated by the row's slot so the final per-row additions run without bank conflicts)
-      constexpr int RP = 4;
-      for (int tok0 = warp; tok0 < nt; tok0 += 4 * RP) {
-        float4 v[RP];
-#pragma unroll
-        for (int q = 0; q < RP; ++q) {
-          const int tok = tok0 + 4 * q;
-          v[q] = tok < nt ? *reinterpret_cast<const float4*>(St + (size_t)tok * GEMM_BM + 4 * lane) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        __syncwarp();
-#pragma unroll
-        for (int q = 0; q < RP; ++q) {
-          const int tok = tok0 + 4 * q;
-          if (tok < nt) {
-            const int r = t0 + tok;
-            float4 w = v[q];
-            w.x += vecv.x; w.y += vecv.y; w.z += vecv.z; w.w += vecv.w;
-            if (tab) {
-              const float4 t = *reinterpret_cast<const float4*>(tab + (size_t)r * ldtab + gf);
-              w.x += t.x; w.y += t.y; w.z += t.z; w.w += t.w;
-            }
-            if (tab2) {
-              const float4 t = *reinterpret_cast<const float4*>(tab2 + (size_t)r * ldtab2 + gf);
-              w.x += t.x; w.y += t.y; w.z += t.z; w.w += t.w;
-            }
-            if (o32) *reinterpret_cast<float4*>(o32 + (size_t)r * ldo32 + gf) = w;
-            if (o16) {
-              __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
-              *reinterpret_cast<uint2*>(o16 + (size_t)r * ldo16 + gf) =
-                  make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
-            }
-            if (ssq_out) {
-              const float sq = fok ? (w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w) : 0.f;
-              St[(size_t)tok * GEMM_BM + ((lane + (tok >> 2)) & 31)] = sq;
-            }
-          }
-        }
-      }
+      Phase2Args p2;
+      p2.vecv = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (ptrs.vec && fok) p2.vecv = *reinterpret_cast<const float4*>(ptrs.vec + gf);
+      p2.tab = tab; p2.tab2 = tab2; p2.o32 = o32; p2.o16 = o16; p2.St = St;
+      p2.ldo32 = ldo32; p2.ldo16 = ldo16; p2.ldtab = ldtab; p2.ldtab2 = ldtab2;
+      p2.nt = nt; p2.t0 = t0; p2.warp = warp; p2.lane = lane; p2.gf = gf; p2.fok = fok; p2.ss = ssq_out != nullptr;
+      const bool has_tab = ptrs.tab || ptrs.tab2 || ptrs.vec;          // warp-uniform choices of the row code
+      if (!has_tab && !ptrs.out32 && !ssq_out) gemm_phase2_rows<false, false, true, false>(p2);      // bf16 only (q|k|v, MLP up)
+      else if (!has_tab) gemm_phase2_rows<false, true, true, true>(p2);                                // residual stream
+      else gemm_phase2_rows<true, true, true, true>(p2);
 #ifdef VLA_TILE_TIMING
       ck[4] = clock64();
 #endif
