@@ -121,7 +121,7 @@ __device__ inline bool queue_try_pop(const DeviceCtx& ctx, int cls, QueueEntry& 
 // ------------------------------------------------------------------ per-SM state of the persistent kernel
 constexpr int MAX_READY = 6;
 constexpr int DISPATCH_THREADS = 64;     // two service warps per SM (claim, retire), after the worker groups
-constexpr int ACT_BACKLOG_MIN = 128;    // action-head tiles waiting from which on a second worker per SM serves the head first
+constexpr long long PRIO_WINDOW_NS = 8000;   // an action-head tile may be claimed for a worker this close to the end of its tile
 constexpr int PREFETCH_MIN_AVAIL = 64;   // tiles are claimed ahead of need only from queues at least this deep
 constexpr int HELD_DEPTH = 2;            // claimed tiles a worker may have waiting
 
@@ -148,6 +148,7 @@ struct WorkerSlot {
   volatile int busy;             // the worker is running a tile (set and cleared by the worker)
   int pad_;
   volatile unsigned prio_tail, prio_head;   // one-deep slot for an action-head tile that goes ahead of the held VLM tiles
+  volatile unsigned long long t_busy;       // when the running tile was taken (worker), for the claim warp's estimate of its end
   WorkerTile done, fin, held[HELD_DEPTH], prio;
   int n_ready;
   ReadyItem ready[MAX_READY];
@@ -161,6 +162,7 @@ struct SmState {
   unsigned tmem_base;
   int waiter;                      // worker whose claimed tile is waiting for room (-1: none); others then admit only memory-free tiles
   volatile int quit;               // claim warp -> retire warp: everyone is leaving
+  volatile int ema_ns[N_CLASSES];  // running mean of tile durations per class on this SM (retire warp)
   WorkerTile cur[MAX_WORKERS];     // the tile each worker is running (written by its leader)
   WorkerSlot slot[MAX_WORKERS];
 };
@@ -287,6 +289,7 @@ __device__ inline void retire_loop(const DeviceCtx& ctx, SmState* sm, int n_work
       slot->done_state = 0;
       have_fin = true;
       const WorkerTile& f = slot->fin;
+      sm->ema_ns[f.cls] = (3 * sm->ema_ns[f.cls] + (int)(f.t1 - f.t0)) >> 2;
       write_trace(ctx, f.inst, f.node, f.tile, lane, f.cls, f.frame, f.t0, f.t1);
       complete_tile(ctx, f, slot);
     } else if (serving) {
@@ -337,12 +340,6 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     long long av = lane < N_CLASSES ? ld_volatile_s64(&ctx.queues[lane].avail) : 0;
     const unsigned pending = __ballot_sync(0xffffffffu, av > 0) & ((1u << N_CLASSES) - 1u);
     const unsigned deep = __ballot_sync(0xffffffffu, av >= PREFETCH_MIN_AVAIL) & ((1u << N_CLASSES) - 1u);
-    // committed action-head tiles nobody has claimed yet, over the head's classes: its backlog.  While it is long,
-    // a second worker of the SM joins worker 0 as reserve for the head.
-    long long act_av = (lane >= N_KINDS && lane < N_CLASSES && av > 0) ? av : 0;
-#pragma unroll
-    for (int o = 4; o > 0; o >>= 1) act_av += __shfl_xor_sync(0xffffffffu, act_av, o);
-    const bool act_backlog = __shfl_sync(0xffffffffu, act_av, 0) >= ACT_BACKLOG_MIN && ctx.policy == POLICY_TWO_PHASE;
     // ---- choose, lane by lane, which class each worker claims from
     int want = -1;
     bool to_prio = false;
@@ -350,29 +347,23 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     lost = 0;
     for (int w = 0; w < n_workers; ++w) {
       const unsigned queued = serving ? slot->held_tail - slot->held_head : 0u;
-#ifdef PRIO_SLOT
       const unsigned pq = serving ? slot->prio_tail - slot->prio_head : 0u;
       if (lane == w && !leaving && (queued < (unsigned)HELD_DEPTH || pq == 0u)) {
+        // A free worker serves the action head first.  A running worker gets VLM tiles claimed ahead of need (from
+        // deep queues only), and an action-head tile when its running tile is within PRIO_WINDOW_NS of its expected
+        // end (this SM's running mean for the class): that tile goes into the priority slot, ahead of the held VLM
+        // tiles, so a short action-head tile is never stuck behind more than the tail of one tile.
         const unsigned act_mask = ((1u << N_KINDS) - 1u) << N_KINDS;
         const bool busy = slot->busy != 0 || queued > 0 || pq > 0;
         const bool head_pending = ctx.policy == POLICY_TWO_PHASE && (pending & act_mask & ~avoid) != 0u;
         unsigned cand;
-        if (!busy) cand = head_pending ? (pending & act_mask) : pending;          // a free worker serves the head first
-        else if (pq == 0u && head_pending) { cand = pending & act_mask; to_prio = true; }   // ahead of the held VLM tiles
+        if (!busy) cand = head_pending ? (pending & act_mask) : pending;
+        else if (pq == 0u && head_pending && slot->busy != 0 &&
+                 (long long)(gtimer() - slot->t_busy) + PRIO_WINDOW_NS >= (long long)sm->ema_ns[sm->cur[w].cls]) {
+          cand = pending & act_mask; to_prio = true;
+        }
         else if (queued < (unsigned)HELD_DEPTH) cand = deep & ((1u << N_KINDS) - 1u);
         else cand = 0u;
-        (void)act_backlog;
-#else
-      if (lane == w && !leaving && queued < (unsigned)HELD_DEPTH) {
-        const bool busy = slot->busy != 0 || queued > 0;   // anything beyond the first tile is claimed ahead of need
-        // early claims (for a worker that is still running) only from deep VLM queues;
-        // worker 0 is the SM's reserve for the action head: nothing is claimed ahead for it (it returns to the pool
-        // when its tile ends) and it takes VLM tiles only while no action-head tile is pending
-        const unsigned act_mask = ((1u << N_KINDS) - 1u) << N_KINDS;
-        const bool reserve = w == 0 || (w == 1 && act_backlog);
-        const bool head_first = reserve && ctx.policy == POLICY_TWO_PHASE && (pending & act_mask & ~avoid) != 0u;
-        unsigned cand = busy ? (reserve ? 0u : (deep & ((1u << N_KINDS) - 1u))) : (head_first ? (pending & act_mask) : pending);
-#endif
         cand &= ~avoid;
         const unsigned long long smask = *reinterpret_cast<volatile unsigned long long*>(&sm->smem_mask);
         const unsigned tmask = *reinterpret_cast<volatile unsigned*>(&sm->tmem_mask);
@@ -485,9 +476,10 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
     sm->tmem_base = 0;
     sm->waiter = -1;
     sm->quit = 0;
+    for (int c = 0; c < N_CLASSES; ++c) sm->ema_ns[c] = 30000;
     for (int w = 0; w < MAX_WORKERS; ++w) {
       sm->slot[w].held_tail = 0; sm->slot[w].held_head = 0; sm->slot[w].leave = 0; sm->slot[w].done_state = 0;
-      sm->slot[w].prio_tail = 0; sm->slot[w].prio_head = 0;
+      sm->slot[w].prio_tail = 0; sm->slot[w].prio_head = 0; sm->slot[w].t_busy = 0;
       sm->slot[w].busy = 0;
       sm->slot[w].n_ready = 0;
     }
@@ -531,6 +523,7 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
         WorkerTile& cur = sm->cur[worker];
         if (st == 1 || st == 3) {
           cur = st == 3 ? slot->prio : slot->held[slot->held_head % HELD_DEPTH];
+          slot->t_busy = gtimer();
           slot->busy = 1;
           __threadfence_block();
           if (st == 3) slot->prio_head = slot->prio_head + 1;

@@ -6,9 +6,10 @@
 // one TMEM column each), K walked in 64-element stages.  The weight tile is
 // the MMA "A" operand and the activation tile the "B" operand, both K-major, so
 // small token counts (the action head's 9..51 rows) still fill the 128-row
-// datapath and stream each weight exactly once.  Gated MLPs run two MMAs per
-// stage (gate and up weights against the same activation tile) into two
-// accumulators.
+// datapath and stream each weight exactly once.  A gated MLP tile covers 64
+// output features: rows 0..63 of its weight tile are gate rows and rows 64..127
+// the matching up rows (two 64-row TMA boxes per stage), so it is one MMA stream
+// and one accumulator like any other tile; the epilogue multiplies act(gate) by up.
 //
 // Roles inside the 128-thread worker: thread 0 of warp 0 issues TMA loads,
 // thread 0 of warp 1 issues MMAs, all four warps run the epilogue (warp w reads
@@ -131,12 +132,11 @@ struct Phase1Args {
   float c_acc, c_x; uint32_t lane_base; int bt, nt, tid, t0;
   bool x_staged;            // the residual rows already sit in St: accumulate on top of them
 };
-template <int ACT, bool DUAL>
+template <int ACT>
 __device__ __forceinline__ void gemm_phase1(const Phase1Args& p) {
   for (int c0 = 0; c0 < p.nt; c0 += 16) {
-    float a[16], b[16], v[16], sc[16];
+    float a[16], v[16], sc[16];
     tmem_ld16(p.lane_base + (uint32_t)c0, a);
-    if (DUAL) tmem_ld16(p.lane_base + (uint32_t)(p.bt + c0), b);
     if (p.rs) {                                        // 16 row scales in four broadcast 16-byte loads
 #pragma unroll
       for (int j = 0; j < 16; j += 4) {
@@ -149,9 +149,7 @@ __device__ __forceinline__ void gemm_phase1(const Phase1Args& p) {
     }
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      float t = apply_act_t<ACT>(a[j] * sc[j]);
-      if (DUAL) t *= b[j] * sc[j];
-      v[j] = t * p.c_acc;
+      v[j] = apply_act_t<ACT>(a[j] * sc[j]) * p.c_acc;
     }
     if (p.outT_row) {
       unsigned short* op = p.outT_row + p.t0 + c0;
@@ -241,12 +239,33 @@ __device__ __forceinline__ void gemm_phase2_rows(const Phase2Args& p) {
   }
 }
 
+// Rows of a gated tile: columns 0..63 of the staged row are gate values, 64..127 the up values of the same 64
+// features.  Sixteen lanes cover a row (four features each), so a warp does two rows per pass.
+template <int ACT>
+__device__ __forceinline__ void gemm_phase2_rows_gated(const Phase2Args& p, float c_acc, int f0, int N) {
+  const int sub = p.lane >> 4, l16 = p.lane & 15;
+  const int gf = f0 + 4 * l16;
+  const bool fok = gf < N;
+  for (int tok0 = p.warp; tok0 < p.nt; tok0 += 8) {
+    const int tok = tok0 + 4 * sub;
+    if (tok < p.nt && fok) {
+      const float4 gt = *reinterpret_cast<const float4*>(p.St + (size_t)tok * GEMM_BM + 4 * l16);
+      const float4 up = *reinterpret_cast<const float4*>(p.St + (size_t)tok * GEMM_BM + GEMM_BM / 2 + 4 * l16);
+      const float w0 = apply_act_t<ACT>(gt.x) * up.x * c_acc, w1 = apply_act_t<ACT>(gt.y) * up.y * c_acc;
+      const float w2 = apply_act_t<ACT>(gt.z) * up.z * c_acc, w3 = apply_act_t<ACT>(gt.w) * up.w * c_acc;
+      __nv_bfloat162 lo = __floats2bfloat162_rn(w0, w1), hi = __floats2bfloat162_rn(w2, w3);
+      *reinterpret_cast<uint2*>(p.o16 + (size_t)(p.t0 + tok) * p.ldo16 + gf) =
+          make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+    }
+  }
+}
+
 constexpr int GEMM_BAR_BYTES = 1024;   // barrier block at the head of the slab (keeps the stages 1024-byte aligned)
 constexpr int GEMM_W_STAGE_BYTES = GEMM_BM * GEMM_BK * 2;
 
 __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   const int ft = tile / g.tiles_t, tt = tile % g.tiles_t;
-  const int f0 = ft * GEMM_BM, t0 = tt * g.bt;
+  const int f0 = ft * (g.dual ? GEMM_BM / 2 : GEMM_BM), t0 = tt * g.bt;    // a gated tile covers 64 output features
   const int nt = min(g.bt, g.M - t0);
   const int warp = c.tid >> 5, lane = c.tid & 31;
   const int nkb = g.Kp / GEMM_BK;
@@ -254,7 +273,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   const int a_bytes = g.bt * GEMM_BK * 2;
   const bool dual = g.dual != 0;            // arguments used inside the loops, out of global memory once
   const int bt = g.bt;
-  const int stage_bytes = GEMM_W_STAGE_BYTES * (dual ? 2 : 1) + a_bytes;
+  const int stage_bytes = GEMM_W_STAGE_BYTES + a_bytes;
 
   uint64_t* bars = reinterpret_cast<uint64_t*>(c.smem);          // full[S], empty[S], accum
   const uint32_t bar0 = smem_u32(bars);
@@ -276,7 +295,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
                     (!ptrs.tab2 || g.ldtab2 % 4 == 0) && (!ptrs.out32 || g.ldo32 % 4 == 0) && (!ptrs.out16 || g.ldo16 % 4 == 0);
   const int gf = f0 + 4 * lane;            // epilogue phase 2: this lane's four consecutive features
   const bool fok = gf < g.N;
-  const uint32_t tmem_d = c.tmem;                 // accumulator columns [0, bt) (and [bt, 2 bt) when dual)
+  const uint32_t tmem_d = c.tmem;                 // accumulator columns [0, bt)
   float* rs_smem = reinterpret_cast<float*>(c.smem + 256);       // [bt] row scales, inside the barrier block
 #ifdef VLA_TILE_TIMING
   uint64_t tt0; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt0));
@@ -297,9 +316,9 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       if (!mbar_wait(c, empty_bar(s), ph ^ 1u)) break;
       mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
       const uint32_t dst = stage0 + (uint32_t)(s * stage_bytes);
-      tma_load_2d(dst, wmap, full_bar(s), kb * GEMM_BK, f0);
-      if (dual) tma_load_2d(dst + GEMM_W_STAGE_BYTES, w2map, full_bar(s), kb * GEMM_BK, f0);
-      tma_load_2d(dst + GEMM_W_STAGE_BYTES * (dual ? 2 : 1), amap, full_bar(s), kb * GEMM_BK, t0);
+      tma_load_2d(dst, wmap, full_bar(s), kb * GEMM_BK, f0);      // 128 rows, or the 64 gate rows of a gated tile
+      if (dual) tma_load_2d(dst + GEMM_W_STAGE_BYTES / 2, w2map, full_bar(s), kb * GEMM_BK, f0);   // its 64 up rows
+      tma_load_2d(dst + GEMM_W_STAGE_BYTES, amap, full_bar(s), kb * GEMM_BK, t0);
     }
     }
     __syncwarp();
@@ -318,14 +337,12 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
 #endif
       tc_fence_after();
       const uint32_t wsm = stage0 + (uint32_t)(s * stage_bytes);
-      const uint32_t asm_ = wsm + GEMM_W_STAGE_BYTES * (dual ? 2 : 1);
+      const uint32_t asm_ = wsm + GEMM_W_STAGE_BYTES;
       const uint64_t wd = umma_desc_sw128(wsm), ad = umma_desc_sw128(asm_);
-      const uint64_t w2d = umma_desc_sw128(wsm + GEMM_W_STAGE_BYTES);
 #pragma unroll
       for (int k = 0; k < GEMM_BK / 16; ++k) {
         const uint32_t accumulate = (kb | k) != 0 ? 1u : 0u;
         umma_bf16(tmem_d, wd + 2u * k, ad + 2u * k, idesc, accumulate);          // 16 bf16 = 32 bytes per K step
-        if (dual) umma_bf16(tmem_d + (uint32_t)bt, w2d + 2u * k, ad + 2u * k, idesc, accumulate);
       }
       umma_commit(empty_bar(s));        // stage reusable once these MMAs have read it
     }
@@ -382,15 +399,10 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
     p1.bt = g.bt; p1.nt = nt; p1.tid = c.tid; p1.t0 = t0;
     const int f = f0 + c.tid;
     p1.outT_row = (ptrs.outT != nullptr && f >= g.t_col0 && f < g.N) ? ptrs.outT + (size_t)(f - g.t_col0) * g.ldoT : nullptr;
-    if (g.dual) {
-      if (g.act == ACT_SILU) gemm_phase1<ACT_SILU, true>(p1);
-      else if (g.act == ACT_GELU) gemm_phase1<ACT_GELU, true>(p1);
-      else gemm_phase1<ACT_NONE, true>(p1);
-    } else {
-      if (g.act == ACT_GELU) gemm_phase1<ACT_GELU, false>(p1);
-      else if (g.act == ACT_SILU) gemm_phase1<ACT_SILU, false>(p1);
-      else gemm_phase1<ACT_NONE, false>(p1);
-    }
+    if (dual) { p1.c_acc = 1.0f; gemm_phase1<ACT_NONE>(p1); }   // gate and up rows parked raw: phase 2 combines them
+    else if (g.act == ACT_GELU) gemm_phase1<ACT_GELU>(p1);
+    else if (g.act == ACT_SILU) gemm_phase1<ACT_SILU>(p1);
+    else gemm_phase1<ACT_NONE>(p1);
   }
 #ifdef VLA_TILE_TIMING
   ck[2] = clock64();
@@ -419,7 +431,12 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       p2.ldo32 = ldo32; p2.ldo16 = ldo16; p2.ldtab = ldtab; p2.ldtab2 = ldtab2;
       p2.nt = nt; p2.t0 = t0; p2.warp = warp; p2.lane = lane; p2.gf = gf; p2.fok = fok; p2.ss = ssq_out != nullptr;
       const bool has_tab = ptrs.tab || ptrs.tab2 || ptrs.vec;          // warp-uniform choices of the row code
-      if (!has_tab && !ptrs.out32 && !ssq_out) gemm_phase2_rows<false, false, true, false>(p2);      // bf16 only (q|k|v, MLP up)
+      if (dual) {
+        p2.o16 = ptrs.out16;
+        if (g.act == ACT_SILU) gemm_phase2_rows_gated<ACT_SILU>(p2, g.c_acc, f0, g.N);
+        else if (g.act == ACT_GELU) gemm_phase2_rows_gated<ACT_GELU>(p2, g.c_acc, f0, g.N);
+        else gemm_phase2_rows_gated<ACT_NONE>(p2, g.c_acc, f0, g.N);
+      } else if (!has_tab && !ptrs.out32 && !ssq_out) gemm_phase2_rows<false, false, true, false>(p2);      // bf16 only (q|k|v, MLP up)
       else if (!has_tab) gemm_phase2_rows<false, true, true, true>(p2);                                // residual stream
       else gemm_phase2_rows<true, true, true, true>(p2);
 #ifdef VLA_TILE_TIMING

@@ -185,12 +185,12 @@ int vla_op_linear(const void* a, const void* w, float* out32, void* out16, int32
   g.act = act; g.c_acc = 1.f; g.c_x = 1.f;
   g.tiles_t = (m + GEMM_MAX_BT - 1) / GEMM_MAX_BT;
   g.bt = (int)op_pad((m + g.tiles_t - 1) / g.tiles_t, 16);
-  g.stages = gemm_stages(g.bt, false, g.Kp);
+  g.stages = gemm_stages(g.bt, g.Kp);
   g.wmap = 0; g.w2map = 0; g.amap = 1;
   OpMaps maps;
   memset(&maps, 0, sizeof maps);
   if (!op_encode(&maps.m[0], w, n, k, k, GEMM_BM) || !op_encode(&maps.m[1], a, m, k, k, g.bt)) return VLA_ERR_CUDA;
-  const int smem = gemm_smem_bytes(g.bt, false, g.stages);
+  const int smem = gemm_smem_bytes(g.bt, g.stages);
   int tmem_cols = 32;
   while (tmem_cols < g.bt) tmem_cols <<= 1;
   static unsigned* err = nullptr;       // one error word per process, allocated on first use

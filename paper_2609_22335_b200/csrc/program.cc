@@ -247,15 +247,21 @@ class Builder {
     g.bt = bt; g.tiles_t = tiles_t;
     {
       // pipeline depth from the stage size; tensor maps for the operands
-      const int S = gemm_stages(bt, g.dual != 0, g.Kp);
+      // A gated tile covers 64 output features: rows 0..63 of its 128-row weight tile come from the gate matrix,
+      // rows 64..127 from the up matrix (two 64-row TMA boxes), so it is one accumulator and has the shared and
+      // tensor-memory shape of a plain tile.
+      const int S = gemm_stages(bt, g.Kp);
       g.stages = S;
-      n.smem_bytes = gemm_smem_bytes(bt, g.dual != 0, S);
-      n.tmem_cols = (int)pad_to((int64_t)bt * (g.dual ? 2 : 1), TMEM_UNIT);
-      g.wmap = weight_map(W, N);
-      g.w2map = o.W2 >= 0 ? weight_map(o.W2, N) : 0;
+      n.smem_bytes = gemm_smem_bytes(bt, S);
+      n.tmem_cols = (int)pad_to((int64_t)bt, TMEM_UNIT);
+      g.wmap = weight_map(W, N, g.dual ? GEMM_BM / 2 : GEMM_BM);
+      g.w2map = o.W2 >= 0 ? weight_map(o.W2, N, GEMM_BM / 2) : 0;
+      if (g.dual && (N % 4 != 0 || o.X.buf >= 0 || o.outT.buf >= 0 || o.out32.buf >= 0 || o.tab || o.tab2 || o.vec))
+        p.error = "internal: a gated GEMM writes bf16 only, width a multiple of 4 (" + name + ")";
       g.amap = act_map(A, g.Kp, bt);
     }
-    n.n_tiles = (int)((g.N + GEMM_BM - 1) / GEMM_BM) * tiles_t;
+    const int feat_per_tile = g.dual ? GEMM_BM / 2 : GEMM_BM;
+    n.n_tiles = (int)((g.N + feat_per_tile - 1) / feat_per_tile) * tiles_t;
     int id = add(n, name, g.dual ? KIND_GEMM2 : KIND_GEMM);
     read(id, A);
     if (o.X.buf >= 0) read(id, o.X);
@@ -270,11 +276,11 @@ class Builder {
     return id;
   }
 
-  int weight_map(int W, int64_t N) {
+  int weight_map(int W, int64_t N, int box_rows = GEMM_BM) {
     const DevTensor& t = p.dev_tensors[W];
-    TmapSpec sp{WEIGHT_BASE + t.offset, false, N, t.ld, t.ld, GEMM_BM};
+    TmapSpec sp{WEIGHT_BASE + t.offset, false, N, t.ld, t.ld, box_rows};
     for (size_t i = 0; i < p.wmaps.size(); ++i)
-      if (p.wmaps[i].offset == sp.offset && p.wmaps[i].rows == sp.rows) return (int)i;
+      if (p.wmaps[i].offset == sp.offset && p.wmaps[i].rows == sp.rows && p.wmaps[i].box_rows == sp.box_rows) return (int)i;
     p.wmaps.push_back(sp);
     return (int)p.wmaps.size() - 1;
   }

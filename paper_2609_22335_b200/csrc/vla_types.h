@@ -42,17 +42,17 @@ constexpr int GEMM_SMEM_BUDGET = 64 * 1024;  // stage memory a token-rich GEMM t
 constexpr int GEMM_SMEM_BUDGET_SMALL = 84 * 1024;  // token-poor tiles (<= 64 tokens) are bound by TMA latency and get deeper
                                                    // pipelines, but must fit the room one finished token-rich tile leaves
                                                    // on an SM that runs three of them (3 x 17 of 56 four-KB units)
-// TMA pipeline depth of a GEMM tile with `bt` tokens per tile.
-inline int gemm_stage_bytes(int bt, bool dual) { return GEMM_BM * GEMM_BK * 2 * (dual ? 2 : 1) + bt * GEMM_BK * 2; }
-inline int gemm_stages(int bt, bool dual, int Kp) {
-  const int stage = gemm_stage_bytes(bt, dual);
+// TMA pipeline depth of a GEMM tile with `bt` tokens per tile (a 128-row weight tile plus the activation tile per stage).
+inline int gemm_stage_bytes(int bt) { return GEMM_BM * GEMM_BK * 2 + bt * GEMM_BK * 2; }
+inline int gemm_stages(int bt, int Kp) {
+  const int stage = gemm_stage_bytes(bt);
   int S = (bt <= 64 ? GEMM_SMEM_BUDGET_SMALL : GEMM_SMEM_BUDGET) / stage;
   S = S < 2 ? 2 : (S > 4 ? 4 : S);
   const int nkb = Kp / GEMM_BK;
   return S < nkb ? S : (nkb < 1 ? 1 : nkb);
 }
-inline int gemm_smem_bytes(int bt, bool dual, int S) {      // the epilogue parks the tile in the stage memory as fp32
-  const int a = S * gemm_stage_bytes(bt, dual), b = bt * GEMM_BM * 4;
+inline int gemm_smem_bytes(int bt, int S) {      // the epilogue parks the tile in the stage memory as fp32
+  const int a = S * gemm_stage_bytes(bt), b = bt * GEMM_BM * 4;
   return 1024 + (a > b ? a : b);
 }
 
@@ -73,7 +73,7 @@ struct GemmArgs {
   int32_t lda, ldx, ldtab, ldtab2, ldo32, ldo16, ldoT, t_col0;
   int32_t M, N, Kp;    // tokens, output features, padded reduction length (multiple of GEMM_BK)
   int32_t bt, tiles_t; // tokens per tile, number of token tiles
-  int32_t act, dual;   // activation; dual: out = act(A W^T) * (A W2^T)
+  int32_t act, dual;   // activation; dual (gated): out = act(A W^T) * (A W2^T), 64 output features per tile
   float c_acc, c_x;    // out = c_x * X + c_acc * acc + vec + tab + tab2
   int32_t wmap, w2map, amap;  // tensor-map indices: shared weight maps, activation map relative to the slot's first
   int32_t stages;             // TMA pipeline depth
