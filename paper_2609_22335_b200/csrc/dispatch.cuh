@@ -162,6 +162,7 @@ struct SmState {
   unsigned tmem_base;
   int waiter;                      // worker whose claimed tile is waiting for room (-1: none); others then admit only memory-free tiles
   volatile int quit;               // claim warp -> retire warp: everyone is leaving
+  int smem_promised, tmem_promised;  // units of tiles handed to free workers that have not allocated them yet
   volatile int ema_ns[N_CLASSES];  // running mean of tile durations per class on this SM (retire warp)
   WorkerTile cur[MAX_WORKERS];     // the tile each worker is running (written by its leader)
   WorkerSlot slot[MAX_WORKERS];
@@ -241,7 +242,7 @@ __device__ inline void complete_tile(const DeviceCtx& ctx, const WorkerTile& f, 
       si[j].node = -1;
       if (i0 + j < n_succ) {
         const int4 v = __ldg(reinterpret_cast<const int4*>(ctx.succ + succ0 + i0 + j));
-        si[j].node = v.x; si[j].n_tiles = v.y; si[j].cls = v.z; si[j].n_pred = v.w;
+        si[j].node = v.x; si[j].n_tiles = v.y; si[j].cls_res = v.z; si[j].n_pred = v.w;
       }
     }
 #pragma unroll
@@ -250,13 +251,15 @@ __device__ inline void complete_tile(const DeviceCtx& ctx, const WorkerTile& f, 
     for (int j = 0; j < 4; ++j) {
       if (left[j] != 0) continue;
       ctx.dep_count[(size_t)inst * ctx.n_nodes + si[j].node] = si[j].n_pred;
+      const int s_cls = si[j].cls_res & 0xFF;
+      const uint32_t s_res = (uint32_t)si[j].cls_res >> 8;
       if (slot->n_ready < MAX_READY) {
         ReadyItem& it = slot->ready[slot->n_ready++];
-        it.base = queue_reserve(ctx, si[j].cls, si[j].n_tiles);
-        it.node = (uint32_t)si[j].node; it.n_tiles = si[j].n_tiles; it.cls = si[j].cls;
-        it.res_units = node_res_units(ctx.nodes[si[j].node]);
+        it.base = queue_reserve(ctx, s_cls, si[j].n_tiles);
+        it.node = (uint32_t)si[j].node; it.n_tiles = si[j].n_tiles; it.cls = s_cls;
+        it.res_units = s_res;
       } else {
-        queue_push(ctx, si[j].cls, inst, (uint32_t)si[j].node, si[j].n_tiles);
+        queue_push(ctx, s_cls, inst, (uint32_t)si[j].node, si[j].n_tiles);
       }
     }
   }
@@ -331,7 +334,7 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     group[c] = ctx.classes[c].group;
   }
   uint64_t idle_start = 0, last_progress = gtimer();
-  unsigned iter = 0, nap = 60, lost = 0;
+  unsigned iter = 0, nap = 60, lost = 0, prev_pending = 0;
   bool leaving = false;
 
   for (;;) {
@@ -340,8 +343,10 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     long long av = lane < N_CLASSES ? ld_volatile_s64(&ctx.queues[lane].avail) : 0;
     const unsigned pending = __ballot_sync(0xffffffffu, av > 0) & ((1u << N_CLASSES) - 1u);
     const unsigned deep = __ballot_sync(0xffffffffu, av >= PREFETCH_MIN_AVAIL) & ((1u << N_CLASSES) - 1u);
+    const unsigned waiting = pending & prev_pending;   // classes that free workers elsewhere did not drain within a round
+    prev_pending = pending;
     // ---- choose, lane by lane, which class each worker claims from
-    int want = -1;
+    int want = -1, promised_s = 0, promised_t = 0;
     bool to_prio = false;
     const unsigned avoid = lost;      // the class this lane just lost a race for: other SMs drained it
     lost = 0;
@@ -350,30 +355,34 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
       const unsigned pq = serving ? slot->prio_tail - slot->prio_head : 0u;
       if (lane == w && !leaving && (queued < (unsigned)HELD_DEPTH || pq == 0u)) {
         // A free worker serves the action head first.  A running worker gets VLM tiles claimed ahead of need (from
-        // deep queues only), and an action-head tile when its running tile is within PRIO_WINDOW_NS of its expected
-        // end (this SM's running mean for the class): that tile goes into the priority slot, ahead of the held VLM
-        // tiles, so a short action-head tile is never stuck behind more than the tail of one tile.
+        // deep queues only), and an action-head tile when that tile has been waiting for more than a round (no
+        // free worker anywhere took it) and the running tile is within PRIO_WINDOW_NS of its expected end (this
+        // SM's running mean for the class): it goes into the priority slot, ahead of the held VLM tiles, so a
+        // short action-head tile is never stuck behind more than the tail of one tile.
         const unsigned act_mask = ((1u << N_KINDS) - 1u) << N_KINDS;
         const bool busy = slot->busy != 0 || queued > 0 || pq > 0;
         const bool head_pending = ctx.policy == POLICY_TWO_PHASE && (pending & act_mask & ~avoid) != 0u;
         unsigned cand;
         if (!busy) cand = head_pending ? (pending & act_mask) : pending;
-        else if (pq == 0u && head_pending && slot->busy != 0 &&
+        else if (pq == 0u && head_pending && (waiting & act_mask & ~avoid) != 0u && slot->busy != 0 &&
                  (long long)(gtimer() - slot->t_busy) + PRIO_WINDOW_NS >= (long long)sm->ema_ns[sm->cur[w].cls]) {
-          cand = pending & act_mask; to_prio = true;
+          cand = waiting & act_mask; to_prio = true;
         }
         else if (queued < (unsigned)HELD_DEPTH) cand = deep & ((1u << N_KINDS) - 1u);
         else cand = 0u;
         cand &= ~avoid;
         const unsigned long long smask = *reinterpret_cast<volatile unsigned long long*>(&sm->smem_mask);
         const unsigned tmask = *reinterpret_cast<volatile unsigned*>(&sm->tmem_mask);
-        const bool blocked = false;
+        // room: a free run of units now, and enough units left after what was promised to tiles already handed
+        // to free workers of this SM (they allocate a moment later)
+        const int smem_left = sm->n_smem_units - __popcll(smask) - *reinterpret_cast<volatile int*>(&sm->smem_promised);
+        const int tmem_left = sm->n_tmem_units - __popc(tmask) - *reinterpret_cast<volatile int*>(&sm->tmem_promised);
         unsigned feasible = 0;
         for (int c = 0; c < N_CLASSES; ++c) {
           const int su = ctx.classes[c].smem_units, tu = ctx.classes[c].tmem_units;
           if (busy) { feasible |= 1u << c; continue; }
-          if (blocked && (su > 0 || tu > 0)) continue;
-          if (find_free(smask, su, sm->n_smem_units) >= 0 && find_free((unsigned long long)tmask, tu, sm->n_tmem_units) >= 0)
+          if (su <= smem_left && tu <= tmem_left && find_free(smask, su, sm->n_smem_units) >= 0 &&
+              find_free((unsigned long long)tmask, tu, sm->n_tmem_units) >= 0)
             feasible |= 1u << c;
         }
         PickState ps;
@@ -382,6 +391,10 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         int phase;
         want = pick_choose(N_CLASSES, tau, group, cand, feasible, ps, sm->pick.rr, ctx.policy, ctx.u_max, &phase);
         if (want >= 0) {
+          if (!busy) {                                   // promised until the worker has allocated (or the pop is lost)
+            promised_s = ctx.classes[want].smem_units; promised_t = ctx.classes[want].tmem_units;
+            atomicAdd(&sm->smem_promised, promised_s); atomicAdd(&sm->tmem_promised, promised_t);
+          }
           atomicAdd(&sm->pick.cta_count[want], 1);     // counted from the claim on, so the next lane sees it
           for (int x = 0; x < 3; ++x) atomicAdd(&sm->pick.u[x], tau[want * 3 + x]);
           sm->pick.rr = (want + 1) % N_CLASSES;
@@ -400,6 +413,7 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         h.smem_units = (int)((e >> (QW_NODE_BITS + QW_INST_BITS + QW_TILE_BITS)) & ((1u << QW_SMEM_BITS) - 1u));
         h.tmem_units = (int)((e >> (QW_NODE_BITS + QW_INST_BITS + QW_TILE_BITS + QW_SMEM_BITS)) & ((1u << QW_TMEM_BITS) - 1u));
         h.cls = want;
+        h.succ_begin = promised_s; h.succ_count = promised_t;   // (fields reused until the worker fills them in) units to un-promise
         __threadfence_block();
         if (to_prio) slot->prio_tail = slot->prio_tail + 1;
         else slot->held_tail = slot->held_tail + 1;      // the worker takes it as soon as it is free
@@ -407,6 +421,7 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
       } else {                                         // lost the race: undo the count
         atomicSub(&sm->pick.cta_count[want], 1);
         for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[want * 3 + x]);
+        if (promised_s | promised_t) { atomicSub(&sm->smem_promised, promised_s); atomicSub(&sm->tmem_promised, promised_t); }
         lost = 1u << want;                             // look elsewhere in the next round, which follows at once
       }
     }
@@ -476,6 +491,7 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
     sm->tmem_base = 0;
     sm->waiter = -1;
     sm->quit = 0;
+    sm->smem_promised = 0; sm->tmem_promised = 0;
     for (int c = 0; c < N_CLASSES; ++c) sm->ema_ns[c] = 30000;
     for (int w = 0; w < MAX_WORKERS; ++w) {
       sm->slot[w].held_tail = 0; sm->slot[w].held_head = 0; sm->slot[w].leave = 0; sm->slot[w].done_state = 0;
@@ -553,6 +569,9 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
 #ifdef VLA_TILE_TIMING
           atomicAdd(ctl->dbg + 7, gtimer() - tw1); atomicAdd(ctl->dbg + 8, 1ull);
 #endif
+          if (cur.succ_begin | cur.succ_count) {     // the claim warp's promise of room is settled either way
+            atomicSub(&sm->smem_promised, cur.succ_begin); atomicSub(&sm->tmem_promised, cur.succ_count);
+          }
           if (!ok) set_error(ctx, DEV_ERR_IDLE_LIMIT, 0x2000u + (unsigned)blockIdx.x);
           cur.t0 = ok ? 1 : 2;              // 1 run, 2 skip (error), 0 leave
         } else {

@@ -343,7 +343,8 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
     std::vector<SuccInfo> si(p.succ.size());
     for (size_t i = 0; i < si.size(); ++i) {
       const NodeDesc& sn = p.nodes[p.succ[i]];
-      si[i] = SuccInfo{p.succ[i], sn.n_tiles, sn.cls, sn.n_pred};
+      const int res = ((sn.smem_bytes + SMEM_UNIT - 1) / SMEM_UNIT) | (((sn.tmem_cols + TMEM_UNIT - 1) / TMEM_UNIT) << QW_SMEM_BITS);
+      si[i] = SuccInfo{p.succ[i], sn.n_tiles, sn.cls | (res << 8), sn.n_pred};
     }
     CU(cudaMemcpy(at<char>(c, p.off_succ), si.data(), sizeof(SuccInfo) * si.size(), cudaMemcpyHostToDevice));
   }

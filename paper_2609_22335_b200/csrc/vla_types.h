@@ -223,7 +223,7 @@ enum DevError : uint32_t {
 
 // Everything a kernel needs, passed by value.
 // One successor edge as the retire path reads it: everything needed to release the node in one 16-byte load.
-struct SuccInfo { int32_t node, n_tiles, cls, n_pred; };
+struct SuccInfo { int32_t node, n_tiles, cls_res, n_pred; };   // cls_res = class | resource units of one tile << 8
 
 struct DeviceCtx {
   char* arena;
