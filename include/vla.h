@@ -86,7 +86,7 @@ typedef struct {
   int32_t n_streams;        /* request streams R */
   int32_t ring_depth;       /* frames in flight per request stream, >= 2 */
   int32_t policy;           /* COSCHED pick: 0 = two-phase resource-aware pick, 1 = first-in-first-out */
-  uint64_t wait_limit_ns;   /* bound of every device-side wait; 0 = default (2 s) */
+  uint64_t wait_limit_ns;   /* bound of every device-side wait; 0 = default (5 s) */
   uint32_t trace_capacity;  /* tile records kept by the device trace; 0 = tracing off */
   int32_t workers_per_sm;   /* COSCHED worker groups per SM; 0 = default */
   int32_t u_max;            /* saturation value of the per-SM utilisation counters in the pick's Phase-2 score
