@@ -122,8 +122,8 @@ __device__ inline bool queue_try_pop(const DeviceCtx& ctx, int cls, QueueEntry& 
 constexpr int MAX_READY = 6;
 constexpr int DISPATCH_THREADS = 64;     // two service warps per SM (claim, retire), after the worker groups
 constexpr long long PRIO_WINDOW_NS = 8000;   // an action-head tile may be claimed for a worker this close to the end of its tile
-constexpr int PREFETCH_MIN_AVAIL = 64;   // tiles are claimed ahead of need only from queues at least this deep
-constexpr int HELD_DEPTH = 2;            // claimed tiles a worker may have waiting
+constexpr int PREFETCH_MIN_AVAIL = 128;   // tiles are claimed ahead of need only from queues at least this deep
+constexpr int HELD_DEPTH = 1;            // claimed tiles a worker may have waiting
 
 struct ReadyItem {
   unsigned long long base;   // reserved queue range
@@ -318,7 +318,7 @@ __device__ inline void retire_loop(const DeviceCtx& ctx, SmState* sm, int n_work
     } else {
       if (sm->quit) break;
       __nanosleep(nap);
-      if (nap < 400) nap += 40;
+      if (nap < 120) nap += 40;
     }
   }
 }
@@ -413,6 +413,11 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         h.smem_units = (int)((e >> (QW_NODE_BITS + QW_INST_BITS + QW_TILE_BITS)) & ((1u << QW_SMEM_BITS) - 1u));
         h.tmem_units = (int)((e >> (QW_NODE_BITS + QW_INST_BITS + QW_TILE_BITS + QW_SMEM_BITS)) & ((1u << QW_TMEM_BITS) - 1u));
         h.cls = want;
+        {   // the worker's first loads are from the node's description: bring its two lines into this SM's L1 now
+          const char* ndp = reinterpret_cast<const char*>(ctx.nodes + h.node);
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(ndp));
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(ndp + 128));
+        }
         h.succ_begin = promised_s; h.succ_count = promised_t;   // (fields reused until the worker fills them in) units to un-promise
         __threadfence_block();
         if (to_prio) slot->prio_tail = slot->prio_tail + 1;
@@ -598,6 +603,10 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
       tc.deadline = t0 + ctx.wait_limit_ns;
       // the frame id is only needed by the emit tile and by the trace
       const int n_op = __ldg(&n.op);
+      if (wt == 0) {     // the retire warp of this SM will read the node's successor records when the tile ends
+        const char* sp = reinterpret_cast<const char*>(ctx.succ + __ldg(&n.succ_begin));
+        asm volatile("prefetch.global.L1 [%0];" ::"l"(sp));
+      }
       const uint64_t frame = (ctx.trace_capacity != 0 || n_op == OP_EMIT)
                                  ? *reinterpret_cast<const volatile uint64_t*>(ctx.inst_frame + cmd.inst) : 0ull;
       if (cmd.t0 == 1) run_tile(ctx, tc, n, (int)cmd.tile, (int)cmd.inst, frame);
@@ -622,7 +631,11 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
         atomicAdd(ctl->dbg + 9, gtimer() - t1); atomicAdd(ctl->dbg + 10, 1ull);
 #endif
         slot->done = d;
-        __threadfence();       // the tile's writes (all threads, ordered by the barrier) before the completion is seen
+        // The tile's writes (all threads, ordered by the barrier above) must be visible device-wide before any
+        // successor is released.  That fence is the retire warp's (first statement of complete_tile, after it has
+        // read this flag): fences are cumulative, and barrier -> block-scope fence -> flag -> device-scope fence
+        // keeps the writes ahead of the counter atomics without a device-scope round trip on the worker's path.
+        __threadfence_block();
         slot->done_state = 1;
         slot->busy = 0;
         atomicSub(&sm->pick.cta_count[cmd.cls], 1);    // the pick's view of this SM, after the completion is on its way
