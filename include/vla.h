@@ -138,7 +138,9 @@ int vla_load_weights(vla_ctx* ctx, const vla_tensor* tensors, size_t n, int32_t 
 
 /* Enqueues one frame of request stream `stream` (Section 2.1: each frame = image(s) +
  * instruction tokens; the head also gets robot state and the initial noise sample).
- * All pointers are HOST memory and are copied before the call returns:
+ * All pointers are HOST memory.  They are copied before the call returns, with one exception:
+ * an image of 64 KiB or more in page-locked (pinned) memory is read by an asynchronous copy,
+ * so that buffer must stay valid and unmodified until this frame's chunk has been polled:
  * image fp32 [n_cam,3,img,img]; text_ids int32 [n_text]; state fp32 [state_dim] or NULL
  * when the model has none; noise fp32 [horizon,act_dim].  Non-blocking with respect to
  * the GPU.  Ring full -> VLA_ERR_BUSY.  frame_id (optional) gets the per-stream frame number. */

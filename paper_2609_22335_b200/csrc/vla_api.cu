@@ -231,11 +231,25 @@ int submit_common(vla_ctx* c, int32_t stream, const float* image, const int32_t*
     ip[2] = reinterpret_cast<uint64_t>(state); ip[3] = reinterpret_cast<uint64_t>(noise);
   } else {
     char* st = c->staging + (size_t)inst * c->staging_bytes;
-    std::memcpy(st + (p.in_image - c->in_lo), image, p.image_bytes);
+    // The image is by far the largest input.  From page-locked memory it is copied straight from the caller's
+    // buffer (no staging pass on the host, which would keep this thread from polling the other streams);
+    // everything else, and images in pageable memory, go through the pinned staging block.
+    uint64_t rest_lo = std::min(p.in_text, p.in_noise);
+    if (d.state_dim > 0) rest_lo = std::min(rest_lo, p.in_state);
+    cudaPointerAttributes pa;
+    const bool direct = p.image_bytes >= (64u << 10) && rest_lo >= p.in_image + p.image_bytes &&
+                        cudaPointerGetAttributes(&pa, image) == cudaSuccess && pa.type == cudaMemoryTypeHost;
+    if (!direct) { cudaGetLastError(); std::memcpy(st + (p.in_image - c->in_lo), image, p.image_bytes); }
     std::memcpy(st + (p.in_text - c->in_lo), text_ids, p.text_bytes);
     if (d.state_dim > 0) std::memcpy(st + (p.in_state - c->in_lo), state, p.state_bytes);
     std::memcpy(st + (p.in_noise - c->in_lo), noise, p.noise_bytes);
-    CU(cudaMemcpyAsync(slot_dev + c->in_lo, st, c->staging_bytes, cudaMemcpyHostToDevice, c->scopy));
+    if (direct) {
+      CU(cudaMemcpyAsync(slot_dev + p.in_image, image, p.image_bytes, cudaMemcpyHostToDevice, c->scopy));
+      CU(cudaMemcpyAsync(slot_dev + rest_lo, st + (rest_lo - c->in_lo), c->in_lo + c->staging_bytes - rest_lo,
+                         cudaMemcpyHostToDevice, c->scopy));
+    } else {
+      CU(cudaMemcpyAsync(slot_dev + c->in_lo, st, c->staging_bytes, cudaMemcpyHostToDevice, c->scopy));
+    }
     ip[0] = reinterpret_cast<uint64_t>(slot_dev + p.in_image); ip[1] = reinterpret_cast<uint64_t>(slot_dev + p.in_text);
     ip[2] = reinterpret_cast<uint64_t>(slot_dev + p.in_state); ip[3] = reinterpret_cast<uint64_t>(slot_dev + p.in_noise);
   }

@@ -190,6 +190,45 @@ def test_api_errors():
         eng.close()
 
 
+def test_pinned_host_inputs_match_pageable_ones():
+    """Images in page-locked memory are copied straight from the caller's buffer, pageable ones are staged: same chunks."""
+    import torch
+    from paper_2609_22335_b200 import Engine
+    from paper_2609_22335_b200.api import VLA_ERR_BUSY
+    m = SMALL["cfg2s"]
+    w = make_weights(m, seed=0)
+    frames = _frames(m)
+    ref, _ = _run(m, w, frames, "cosched")
+    eng = Engine(m, mode="cosched", n_streams=len(frames))
+    try:
+        eng.load_weights(w)
+        pinned = [[{k: (None if v is None else torch.from_numpy(np.ascontiguousarray(v)).pin_memory()) for k, v in fr.items()}
+                   for fr in s] for s in frames]
+        ptr = lambda t: None if t is None else t.data_ptr()  # noqa: E731
+        got = [[None] * m.n_frames for _ in frames]
+        nxt = [0] * len(frames)
+        left = len(frames) * m.n_frames
+        import time
+        t0 = time.time()
+        while left and time.time() - t0 < 120:
+            for r in range(len(frames)):
+                while nxt[r] < m.n_frames:
+                    d = pinned[r][nxt[r]]
+                    if eng.submit_ptrs(r, ptr(d["image"]), ptr(d["text"]), ptr(d["state"]), ptr(d["noise"])) == VLA_ERR_BUSY:
+                        break
+                    nxt[r] += 1
+                res = eng.poll(r)
+                if res is not None:
+                    got[r][res[1]] = res[0]
+                    left -= 1
+        assert left == 0
+    finally:
+        eng.close()
+    for r in range(len(frames)):
+        for n in range(m.n_frames):
+            assert np.array_equal(got[r][n], ref[r][n]), (r, n)
+
+
 def test_policy_probe_matches_algorithm_1():
     """The device pick, run on the GPU, agrees with the CPU oracle of Algorithm 1 on random states."""
     import random
