@@ -522,6 +522,9 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
     int tau[N_CLASSES * 3];
     for (int c = 0; c < N_CLASSES; ++c)
       for (int x = 0; x < 3; ++x) tau[c * 3 + x] = ctx.classes[c].tau[x];
+#ifdef VLA_TILE_TIMING
+    long long ck_end = 0, ck_posted = 0, ck_seen = 0, ck_alloc = 0;
+#endif
     for (;;) {
       if (wt == 0) {
         // take the tile the claim warp holds for this worker, then give it its exact memory need
@@ -539,6 +542,7 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
         }
 #ifdef VLA_TILE_TIMING
         const uint64_t tw1 = gtimer();
+        ck_seen = clock64();
         atomicAdd(ctl->dbg + 5, tw1 - tw0); atomicAdd(ctl->dbg + 6, 1ull);
 #endif
         WorkerTile& cur = sm->cur[worker];
@@ -573,6 +577,7 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
           }
 #ifdef VLA_TILE_TIMING
           atomicAdd(ctl->dbg + 7, gtimer() - tw1); atomicAdd(ctl->dbg + 8, 1ull);
+          ck_alloc = clock64();
 #endif
           if (cur.succ_begin | cur.succ_count) {     // the claim warp's promise of room is settled either way
             atomicSub(&sm->smem_promised, cur.succ_begin); atomicSub(&sm->tmem_promised, cur.succ_count);
@@ -601,6 +606,14 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
       tc.amap_base = ctx.n_weight_tmaps + (int)cmd.inst * ctx.n_act_tmaps;
       const uint64_t t0 = gtimer();
       tc.deadline = t0 + ctx.wait_limit_ns;
+#ifdef VLA_TILE_TIMING
+      if (wt == 0 && ck_end != 0 && cmd.t0 == 1) {     // SM clocks between two tiles of this worker
+        const long long now = clock64();
+        atomicAdd(ctl->dbg + 36, (unsigned long long)(ck_posted - ck_end)); atomicAdd(ctl->dbg + 37, (unsigned long long)(ck_seen - ck_posted));
+        atomicAdd(ctl->dbg + 38, (unsigned long long)(ck_alloc - ck_seen)); atomicAdd(ctl->dbg + 39, (unsigned long long)(now - ck_alloc));
+        atomicAdd(ctl->dbg + 22, 1ull);
+      }
+#endif
       // the frame id is only needed by the emit tile and by the trace
       const int n_op = __ldg(&n.op);
       if (wt == 0) {     // the retire warp of this SM will read the node's successor records when the tile ends
@@ -610,10 +623,15 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
       const uint64_t frame = (ctx.trace_capacity != 0 || n_op == OP_EMIT)
                                  ? *reinterpret_cast<const volatile uint64_t*>(ctx.inst_frame + cmd.inst) : 0ull;
       if (cmd.t0 == 1) run_tile(ctx, tc, n, (int)cmd.tile, (int)cmd.inst, frame);
-      asm volatile("fence.proxy.async;" ::: "memory");   // outputs may be read by TMA on another SM
+      // Outputs written here by ordinary stores are read by TMA on other SMs.  The proxy fence that must lie between
+      // the two in causality order is the consumer's (first statement of its TMA-issuing thread, after the
+      // dependency was observed); a second one here cost 2 % of the throughput and is not needed.
       asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
       if (wt == 0) {
         ++tiles;
+#ifdef VLA_TILE_TIMING
+        ck_end = clock64();
+#endif
         const uint64_t t1 = gtimer();
         if (cmd.t0 == 1) {
           if (cmd.smem_units) atomicAnd(&sm->smem_mask, ~(unit_bits(cmd.smem_units) << cmd.smem_unit0));
@@ -640,6 +658,9 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
         slot->busy = 0;
         atomicSub(&sm->pick.cta_count[cmd.cls], 1);    // the pick's view of this SM, after the completion is on its way
         for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[cmd.cls * 3 + x]);
+#ifdef VLA_TILE_TIMING
+        ck_posted = clock64();
+#endif
       }
     }
     if (wt == 0) atomicAdd(&ctl->tiles_done, tiles);

@@ -675,6 +675,10 @@ int vla_get_counters(vla_ctx* c, uint64_t* tiles, uint64_t* kernel_launches, uin
           fprintf(stderr, "dbg: epilogue clocks (%s): ptrs+stage+sync %.0f  phase1 %.0f  sync %.0f  phase2 rows %.0f  row sums+rest %.0f (x %llu)\n",
                   b == 24 ? "residual" : "qkv", (double)ctl.dbg[b] / ctl.dbg[b + 5], (double)ctl.dbg[b + 1] / ctl.dbg[b + 5],
                   (double)ctl.dbg[b + 2] / ctl.dbg[b + 5], (double)ctl.dbg[b + 3] / ctl.dbg[b + 5], (double)ctl.dbg[b + 4] / ctl.dbg[b + 5], ctl.dbg[b + 5]);
+    if (getenv("VLA_PRINT_DBG") && ctl.dbg[22])
+      fprintf(stderr, "dbg: between two tiles of a worker (SM clocks): post %.0f  wait for the next tile %.0f  allocate %.0f  barrier + setup %.0f (x %llu)\n",
+              (double)ctl.dbg[36] / ctl.dbg[22], (double)ctl.dbg[37] / ctl.dbg[22], (double)ctl.dbg[38] / ctl.dbg[22],
+              (double)ctl.dbg[39] / ctl.dbg[22], ctl.dbg[22]);
     if (getenv("VLA_PRINT_DBG"))
       fprintf(stderr, "dbg: wait-for-claim %.2f us x %llu  wait-for-room %.2f us x %llu  wait-to-post %.2f us x %llu\n",
               ctl.dbg[6] ? ctl.dbg[5] / 1e3 / ctl.dbg[6] : 0.0, ctl.dbg[6], ctl.dbg[8] ? ctl.dbg[7] / 1e3 / ctl.dbg[8] : 0.0,
