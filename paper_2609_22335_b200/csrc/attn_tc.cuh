@@ -95,8 +95,9 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a_in, int tile)
 
   // shared-memory carve-up (all tile bases 1024-byte aligned)
   const uint32_t base = smem_u32(c.smem);
-  const uint32_t bar_q = base, bar_k = base + 8, bar_v = base + 16, bar_s = base + 24, bar_o = base + 32;
-  const uint32_t Qs = base + 1024;
+  const uint32_t bar0 = smem_u32(c.ctl);                       // the five barriers live in the worker's control block
+  const uint32_t bar_q = bar0, bar_k = bar0 + 8, bar_v = bar0 + 16, bar_s = bar0 + 24, bar_o = bar0 + 32;
+  const uint32_t Qs = base;
   const uint32_t Ks = Qs + (uint32_t)nbox * (ATTN_BQ * 128);
   const uint32_t Vs = Ks + (uint32_t)nbox * (ATTN_BN * 128);
   const uint32_t Ps = Vs + (uint32_t)(hs * 128);

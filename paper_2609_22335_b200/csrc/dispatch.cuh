@@ -8,7 +8,9 @@ namespace vla {
 
 constexpr unsigned CTRL_EXITING = 0x80000000u;
 constexpr int MAX_WORKERS = 3;
-constexpr int SM_STATE_BYTES = 2048;
+constexpr int SM_CTL_BYTES = 1024;       // per-worker control block (mbarriers, row scales) handed to the tile bodies
+constexpr int SM_STATE_BASE = 2048;      // dispatcher state of the SM
+constexpr int SM_STATE_BYTES = SM_STATE_BASE + MAX_WORKERS * SM_CTL_BYTES;   // then the tile slab, 1024-byte aligned
 
 __device__ __forceinline__ uint64_t gtimer() {
   uint64_t t;
@@ -167,7 +169,7 @@ struct SmState {
   WorkerTile cur[MAX_WORKERS];     // the tile each worker is running (written by its leader)
   WorkerSlot slot[MAX_WORKERS];
 };
-static_assert(sizeof(SmState) <= SM_STATE_BYTES, "SM state too large");
+static_assert(sizeof(SmState) <= SM_STATE_BASE, "SM state too large");
 
 __device__ __forceinline__ unsigned long long unit_bits(int n) { return n >= 64 ? ~0ull : ((1ull << n) - 1ull); }
 // Lowest position of `need` consecutive free units among the first `total` (bit set = in use), or -1.
@@ -596,6 +598,7 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
       tc.arena = ctx.arena;
       tc.slot_base = ctx.slot_base[cmd.inst];
       tc.smem = slab + (size_t)cmd.smem_unit0 * SMEM_UNIT;
+      tc.ctl = smem_raw + SM_STATE_BASE + worker * SM_CTL_BYTES;
       tc.tmem = sm->tmem_base + (unsigned)cmd.tmem_unit0 * TMEM_UNIT;
       tc.tid = wt;
       tc.bar_id = bar_id;
@@ -674,6 +677,7 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
 __global__ void __launch_bounds__(WORKER_THREADS) vla_node_kernel(DeviceCtx ctx, const NodeDesc* nodes, int node_idx, int inst) {
   extern __shared__ __align__(1024) char smem_raw[];
   __shared__ uint32_t tmem_base_s;
+  __shared__ __align__(16) char ctl_block[1024];
   const NodeDesc& n = nodes[node_idx];
   uint32_t tmem_cols = 0;
   if (n.tmem_cols > 0) {
@@ -688,6 +692,7 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_node_kernel(DeviceCtx ctx,
   tc.arena = ctx.arena;
   tc.slot_base = inst >= 0 ? ctx.slot_base[inst] : 0;
   tc.smem = smem_raw;
+  tc.ctl = ctl_block;
   tc.tmem = tmem_cols ? tmem_base_s : 0;
   tc.tid = threadIdx.x;
   tc.bar_id = 1;

@@ -260,7 +260,6 @@ __device__ __forceinline__ void gemm_phase2_rows_gated(const Phase2Args& p, floa
   }
 }
 
-constexpr int GEMM_BAR_BYTES = 1024;   // barrier block at the head of the slab (keeps the stages 1024-byte aligned)
 constexpr int GEMM_W_STAGE_BYTES = GEMM_BM * GEMM_BK * 2;
 
 __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
@@ -275,9 +274,9 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   const int bt = g.bt;
   const int stage_bytes = GEMM_W_STAGE_BYTES + a_bytes;
 
-  uint64_t* bars = reinterpret_cast<uint64_t*>(c.smem);          // full[S], empty[S], accum
+  uint64_t* bars = reinterpret_cast<uint64_t*>(c.ctl);           // full[S], empty[S], accum (the worker's control block)
   const uint32_t bar0 = smem_u32(bars);
-  const uint32_t stage0 = smem_u32(c.smem + GEMM_BAR_BYTES);
+  const uint32_t stage0 = smem_u32(c.smem);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
   const uint32_t accum_bar = bar0 + 8u * (2 * S);
@@ -296,7 +295,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   const int gf = f0 + 4 * lane;            // epilogue phase 2: this lane's four consecutive features
   const bool fok = gf < g.N;
   const uint32_t tmem_d = c.tmem;                 // accumulator columns [0, bt)
-  float* rs_smem = reinterpret_cast<float*>(c.smem + 256);       // [bt] row scales, inside the barrier block
+  float* rs_smem = reinterpret_cast<float*>(c.ctl + 256);        // [bt] row scales, in the control block
 #ifdef VLA_TILE_TIMING
   uint64_t tt0; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt0));
 #endif
@@ -378,7 +377,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
 #ifdef VLA_TILE_TIMING
   long long ck[6]; ck[0] = clock64();
 #endif
-  float* St = reinterpret_cast<float*>(c.smem + GEMM_BAR_BYTES);   // [bt][128] fp32
+  float* St = reinterpret_cast<float*>(c.smem);   // [bt][128] fp32
   // The residual rows of this tile start their way into the staging area now (asynchronous 16-byte copies
   // through L2, no registers held), so their latency overlaps the accumulator read-out.
   const bool x_staged = vec4 && ptrs.X != nullptr;

@@ -44,11 +44,12 @@ inline bool op_encode(CUtensorMap* out, const void* base, int64_t rows, int64_t 
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-__device__ __forceinline__ TileCtx op_tile_ctx(char* smem, uint32_t tmem, const void* maps, unsigned* err) {
+__device__ __forceinline__ TileCtx op_tile_ctx(char* smem, char* ctl, uint32_t tmem, const void* maps, unsigned* err) {
   TileCtx tc;
   tc.arena = nullptr;          // Refs of the stand-alone operators are absolute device addresses
   tc.slot_base = 0;
   tc.smem = smem;
+  tc.ctl = ctl;
   tc.tmem = tmem;
   tc.tid = threadIdx.x;
   tc.bar_id = 1;
@@ -65,11 +66,12 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_op_attention_kernel(AttnAr
                                                                           int tmem_cols, unsigned* err) {
   extern __shared__ __align__(1024) char smem_raw[];
   __shared__ uint32_t tmem_base_s;
+  __shared__ __align__(16) char ctl_block[1024];
   if (threadIdx.x < 32) tmem_alloc(&tmem_base_s, (uint32_t)tmem_cols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  TileCtx tc = op_tile_ctx(smem_raw, tmem_base_s, &maps, err);
+  TileCtx tc = op_tile_ctx(smem_raw, ctl_block, tmem_base_s, &maps, err);
   tile_attention(tc, a, (int)blockIdx.x);
   tc_fence_before();
   __syncthreads();
@@ -80,11 +82,12 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_op_linear_kernel(GemmArgs 
                                                                        int tmem_cols, unsigned* err) {
   extern __shared__ __align__(1024) char smem_raw[];
   __shared__ uint32_t tmem_base_s;
+  __shared__ __align__(16) char ctl_block[1024];
   if (threadIdx.x < 32) tmem_alloc(&tmem_base_s, (uint32_t)tmem_cols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  TileCtx tc = op_tile_ctx(smem_raw, tmem_base_s, &maps, err);
+  TileCtx tc = op_tile_ctx(smem_raw, ctl_block, tmem_base_s, &maps, err);
   tile_gemm(tc, g, (int)blockIdx.x);
   tc_fence_before();
   __syncthreads();

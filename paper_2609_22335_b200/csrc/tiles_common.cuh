@@ -15,7 +15,9 @@ namespace vla {
 struct TileCtx {
   char* arena;
   uint64_t slot_base;   // arena offset of this frame slot's buffers
-  char* smem;           // this worker's shared-memory slab (16-byte aligned)
+  char* smem;           // this tile's shared-memory slab (1024-byte aligned): operand stages, staging tiles
+  char* ctl;            // this worker's 1 KB control block (mbarriers, row scales): outside the slab, so tile
+                        // slabs are whole powers-of-two-friendly sizes (64 KB, 72 KB, 48 KB)
   uint32_t tmem;        // this worker's tensor-memory column base
   int tid;              // 0 .. WORKER_THREADS-1
   int bar_id;           // named barrier of this worker

@@ -41,7 +41,7 @@ constexpr int GEMM_MAX_BT = 128;     // most tokens per GEMM tile (MMA N)
 constexpr int GEMM_SMEM_BUDGET = 64 * 1024;  // stage memory a token-rich GEMM tile aims for (at least two stages are always taken)
 constexpr int GEMM_SMEM_BUDGET_SMALL = 84 * 1024;  // token-poor tiles (<= 64 tokens) are bound by TMA latency and get deeper
                                                    // pipelines, but must fit the room one finished token-rich tile leaves
-                                                   // on an SM that runs three of them (3 x 17 of 56 four-KB units)
+                                                   // on an SM that runs three of them (3 x 18 of 55 four-KB units)
 // TMA pipeline depth of a GEMM tile with `bt` tokens per tile (a 128-row weight tile plus the activation tile per stage).
 inline int gemm_stage_bytes(int bt) { return GEMM_BM * GEMM_BK * 2 + bt * GEMM_BK * 2; }
 inline int gemm_stages(int bt, int Kp) {
@@ -53,14 +53,14 @@ inline int gemm_stages(int bt, int Kp) {
 }
 inline int gemm_smem_bytes(int bt, int S) {      // the epilogue parks the tile in the stage memory as fp32
   const int a = S * gemm_stage_bytes(bt), b = bt * GEMM_BM * 4;
-  return 1024 + (a > b ? a : b);
+  return a > b ? a : b;
 }
 
-// Shared memory of one attention tile: barrier block, Q (128 rows), one K block and one V^T block of 64 keys,
+// Shared memory of one attention tile: Q (128 rows), one K block and one V^T block of 64 keys,
 // and the probability tile.  hs = head stride (head dim padded to a multiple of 16).
 inline int attn_smem_bytes(int hs) {
   const int nbox = (hs + 63) / 64;
-  return 1024 + nbox * 128 * 128 + nbox * 64 * 128 + hs * 128 + 128 * 128;
+  return nbox * 128 * 128 + nbox * 64 * 128 + hs * 128 + 128 * 128;
 }
 
 struct GemmArgs {
