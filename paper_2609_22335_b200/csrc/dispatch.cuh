@@ -559,12 +559,20 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
           bool ok = false;
           for (unsigned spin = 0;; ++spin) {
             const unsigned long long sm_old = *reinterpret_cast<volatile unsigned long long*>(&sm->smem_mask);
-            const int s0 = find_free(sm_old, cur.smem_units, sm->n_smem_units);
+            // every worker has a home region (a third of the slab, a third of the columns): a tile that fits it goes
+            // there whenever it is free, so tiles of the common shapes never fragment the slab; larger tiles and a
+            // home occupied by one of them fall back to the first free run
+            const int home_s = worker * (sm->n_smem_units / n_workers), home_t = worker * (sm->n_tmem_units / n_workers);
+            int s0 = -1;
+            if (cur.smem_units <= sm->n_smem_units / n_workers && ((sm_old >> home_s) & unit_bits(cur.smem_units)) == 0ull) s0 = home_s;
+            else s0 = find_free(sm_old, cur.smem_units, sm->n_smem_units);
             if (s0 >= 0) {
               const unsigned long long sbits = unit_bits(cur.smem_units) << s0;
               if (cur.smem_units == 0 || atomicCAS(&sm->smem_mask, sm_old, sm_old | sbits) == sm_old) {
                 const unsigned tm_old = *reinterpret_cast<volatile unsigned*>(&sm->tmem_mask);
-                const int t0 = find_free((unsigned long long)tm_old, cur.tmem_units, sm->n_tmem_units);
+                int t0 = -1;
+                if (cur.tmem_units <= sm->n_tmem_units / n_workers && ((tm_old >> home_t) & (unsigned)unit_bits(cur.tmem_units)) == 0u) t0 = home_t;
+                else t0 = find_free((unsigned long long)tm_old, cur.tmem_units, sm->n_tmem_units);
                 const unsigned tbits = (unsigned)(unit_bits(cur.tmem_units) << (t0 < 0 ? 0 : t0));
                 if (t0 >= 0 && (cur.tmem_units == 0 || atomicCAS(&sm->tmem_mask, tm_old, tm_old | tbits) == tm_old)) {
                   cur.smem_unit0 = s0; cur.tmem_unit0 = t0;
