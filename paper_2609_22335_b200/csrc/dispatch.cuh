@@ -627,8 +627,10 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
 #endif
       // the frame id is only needed by the emit tile and by the trace
       const int n_op = __ldg(&n.op);
-      if (wt == 0) {     // the retire warp of this SM will read the node's successor records when the tile ends
-        const char* sp = reinterpret_cast<const char*>(ctx.succ + __ldg(&n.succ_begin));
+      // the node's successor range travels with the finished tile; read it now, while the description is hot
+      const int n_succ_begin = __ldg(&n.succ_begin), n_succ_count = __ldg(&n.succ_count);
+      if (wt == 0) {     // the retire warp of this SM will read the successor records when the tile ends
+        const char* sp = reinterpret_cast<const char*>(ctx.succ + n_succ_begin);
         asm volatile("prefetch.global.L1 [%0];" ::"l"(sp));
       }
       const uint64_t frame = (ctx.trace_capacity != 0 || n_op == OP_EMIT)
@@ -650,7 +652,7 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
         }
         WorkerTile d = cmd;
         d.t0 = t0; d.t1 = t1; d.frame = frame;
-        d.succ_begin = __ldg(&n.succ_begin); d.succ_count = __ldg(&n.succ_count); d.op = n_op;
+        d.succ_begin = n_succ_begin; d.succ_count = n_succ_count; d.op = n_op;
         unsigned naps = 0;
         while (slot->done_state != 0) {
           __nanosleep(40);
