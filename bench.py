@@ -37,7 +37,7 @@ METRIC = "action_chunks_per_sec"
 UNIT = "chunks/s"
 # DRAM bytes per action chunk of the persistent kernel, from the ncu capture summarised in
 # profiles/cosched_kernel_cfg2_small_dram.md (small case, scaled by chunks: an upper bound at full size)
-MEASURED_DRAM_BYTES_PER_CHUNK = {"cfg2_smolvla": 2.659e9 + 0.097e9}
+MEASURED_DRAM_BYTES_PER_CHUNK = {"cfg2_smolvla": 2.655e9 + 0.091e9}
 
 
 def measured_peaks():
