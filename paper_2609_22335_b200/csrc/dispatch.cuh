@@ -640,16 +640,22 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
       // the two in causality order is the consumer's (first statement of its TMA-issuing thread, after the
       // dependency was observed); a second one here cost 2 % of the throughput and is not needed.
       asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(WORKER_THREADS) : "memory");
+      // Two lanes share the end of a tile: lane 0 frees the tile's memory and goes straight on to take the next
+      // tile, the first lane of warp 1 posts the finished one to the retire warp meanwhile (both meet again at the
+      // barrier that opens the next tile).
       if (wt == 0) {
         ++tiles;
 #ifdef VLA_TILE_TIMING
         ck_end = clock64();
+        ck_posted = ck_end;
 #endif
-        const uint64_t t1 = gtimer();
         if (cmd.t0 == 1) {
           if (cmd.smem_units) atomicAnd(&sm->smem_mask, ~(unit_bits(cmd.smem_units) << cmd.smem_unit0));
           if (cmd.tmem_units) atomicAnd(&sm->tmem_mask, ~(unsigned)(unit_bits(cmd.tmem_units) << cmd.tmem_unit0));
         }
+        slot->busy = 0;
+      } else if (wt == 32) {
+        const uint64_t t1 = gtimer();
         WorkerTile d = cmd;
         d.t0 = t0; d.t1 = t1; d.frame = frame;
         d.succ_begin = n_succ_begin; d.succ_count = n_succ_count; d.op = n_op;
@@ -668,12 +674,8 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
         // keeps the writes ahead of the counter atomics without a device-scope round trip on the worker's path.
         __threadfence_block();
         slot->done_state = 1;
-        slot->busy = 0;
         atomicSub(&sm->pick.cta_count[cmd.cls], 1);    // the pick's view of this SM, after the completion is on its way
         for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[cmd.cls * 3 + x]);
-#ifdef VLA_TILE_TIMING
-        ck_posted = clock64();
-#endif
       }
     }
     if (wt == 0) atomicAdd(&ctl->tiles_done, tiles);
