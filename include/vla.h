@@ -85,7 +85,8 @@ typedef struct {
   int32_t mode;             /* VLA_MODE_* */
   int32_t n_streams;        /* request streams R */
   int32_t ring_depth;       /* frames in flight per request stream, >= 2 */
-  int32_t policy;           /* COSCHED pick: 0 = two-phase resource-aware pick, 1 = first-in-first-out */
+  int32_t policy;           /* COSCHED pick: 0 = two-phase resource-aware pick (Algorithm 1), 1 = fixed class order,
+                             * 2 = round robin over the classes */
   uint64_t wait_limit_ns;   /* bound of every device-side wait; 0 = default (5 s) */
   uint32_t trace_capacity;  /* tile records kept by the device trace; 0 = tracing off */
   int32_t workers_per_sm;   /* COSCHED worker groups per SM; 0 = default */
