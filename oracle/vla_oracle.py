@@ -27,7 +27,9 @@ to bf16-representable values.
 Pins (see tests/test_oracle_pins.py): every function here is checked against
 something other than itself -- brute-force loops, closed forms, invariants or
 a library routine.  The end-to-end chunk has no printed reference value in the
-paper; it is pinned through those parts plus the whole-tower closed forms
+paper; it is pinned through those parts, the layer compositions (one vision
+encoder layer, one LLM layer, every head kind end to end: explicit-loop
+restatements in tests/test_oracle_layer_pins.py), the whole-tower closed forms
 (zeroed residual branches) and the dependency rule.
 """
 from __future__ import annotations
@@ -173,6 +175,26 @@ def vision_tokens(m, w, image, dtype):
     return np.concatenate(outs, axis=0)
 
 
+def llm_layer(m, w, i, x, pos, dtype):
+    """Decoder layer i of the prefix LLM on the stream x [S,d] at positions pos.
+
+    Returns (x after the layer, K [S,Hkv,hd] as cached -- after RoPE where used --, V [S,Hkv,hd]).
+    """
+    s = x.shape[0]
+    p = f"llm.L{i}."
+    h = rmsnorm(x, w[p + "n1"].astype(dtype))
+    q = linear(h, w[p + "wq"].astype(dtype)).reshape(s, m.hq, m.hd)
+    k = linear(h, w[p + "wk"].astype(dtype)).reshape(s, m.hkv, m.hd)
+    v = linear(h, w[p + "wv"].astype(dtype)).reshape(s, m.hkv, m.hd)
+    if m.rope:
+        q, k = rope(q, pos), rope(k, pos)
+    a = attention(q, k, v, causal=m.causal).reshape(s, m.hq * m.hd)
+    x = x + linear(a, w[p + "wo"].astype(dtype))
+    h = rmsnorm(x, w[p + "n2"].astype(dtype))
+    x = x + mlp(h, w, p, m.mlp_kind, dtype)
+    return x, k, v
+
+
 def vlm_forward(m, w, image, text, dtype=np.float32):
     """VLM phase of one frame.  Returns the handoff the action head consumes.
 
@@ -190,18 +212,8 @@ def vlm_forward(m, w, image, text, dtype=np.float32):
     pos = np.arange(s)
     kv = []
     for i in range(m.llm_layers):
-        p = f"llm.L{i}."
-        h = rmsnorm(x, w[p + "n1"].astype(dtype))
-        q = linear(h, w[p + "wq"].astype(dtype)).reshape(s, m.hq, m.hd)
-        k = linear(h, w[p + "wk"].astype(dtype)).reshape(s, m.hkv, m.hd)
-        v = linear(h, w[p + "wv"].astype(dtype)).reshape(s, m.hkv, m.hd)
-        if m.rope:
-            q, k = rope(q, pos), rope(k, pos)
+        x, k, v = llm_layer(m, w, i, x, pos, dtype)
         kv.append((k, v))
-        a = attention(q, k, v, causal=m.causal).reshape(s, m.hq * m.hd)
-        x = x + linear(a, w[p + "wo"].astype(dtype))
-        h = rmsnorm(x, w[p + "n2"].astype(dtype))
-        x = x + mlp(h, w, p, m.mlp_kind, dtype)
     hidden = rmsnorm(x, w["llm.norm"].astype(dtype))
     return {"kv": kv, "hidden": hidden, "prefix": prefix}
 

@@ -1,0 +1,375 @@
+"""Pins of the oracle's layer COMPOSITIONS: which norm feeds which projection, where RoPE is applied, what is
+cached, how the four head kinds combine their own tokens with the VLM handoff.
+
+Each oracle function is compared with a restatement written here from the readings of the workload
+descriptions, in plain Python floats with explicit loops over tokens, heads and features.  The restatements
+call nothing in ``oracle/`` and no array library routine beyond building the random inputs: a wrong norm, a
+swapped concatenation, a missing RoPE offset, a transposed matrix or a dropped residual in the oracle fails one
+of these pins.  Weights are drawn large enough that attention logits are of order 1..10 (far from uniform
+softmax rows), every residual-branch output matrix is non-zero, and the norm gains differ from one another.
+"""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import vla_oracle as O
+from vla_synth.configs import CFG1, CFG2, CFG3, CFG4, CFG5, mini, weight_shapes, is_gain
+
+F64 = np.float64
+EPS = 1e-6
+
+
+# ------------------------------------------------------------------ scalar building blocks (lists of floats)
+def matvec(W, x):
+    """y[o] = sum_k W[o][k] x[k]   (matrices are stored [out][in])."""
+    assert len(W[0]) == len(x)
+    return [sum(W[o][k] * x[k] for k in range(len(x))) for o in range(len(W))]
+
+
+def rms(x, g):
+    ms = sum(v * v for v in x) / len(x)
+    return [g[i] * x[i] / math.sqrt(ms + EPS) for i in range(len(x))]
+
+
+def gelu(v):
+    return 0.5 * v * (1.0 + math.tanh(math.sqrt(2.0 / math.pi) * (v + 0.044715 * v ** 3)))
+
+
+def silu(v):
+    return v / (1.0 + math.exp(-v))
+
+
+def add(a, b):
+    return [a[i] + b[i] for i in range(len(a))]
+
+
+def rotate(vec, pos):
+    """Rotary embedding of one head vector: pairs (i, i + hd/2), angle pos * 10000^(-2i/hd)."""
+    hd = len(vec)
+    half = hd // 2
+    out = [0.0] * hd
+    for i in range(half):
+        ang = pos * 10000.0 ** (-2.0 * i / hd)
+        c, s = math.cos(ang), math.sin(ang)
+        out[i] = vec[i] * c - vec[i + half] * s
+        out[i + half] = vec[i + half] * c + vec[i] * s
+    return out
+
+
+def attend_one(q, keys, vals):
+    """One query vector of one head over the visible keys: softmax(q.k / sqrt(hd)) weighted sum of values."""
+    hd = len(q)
+    logits = [sum(q[c] * k[c] for c in range(hd)) / math.sqrt(hd) for k in keys]
+    mx = max(logits)
+    e = [math.exp(l - mx) for l in logits]
+    z = sum(e)
+    return [sum(e[j] / z * vals[j][c] for j in range(len(keys))) for c in range(hd)]
+
+
+def heads_of(vec, n_heads, hd):
+    assert len(vec) == n_heads * hd
+    return [vec[h * hd:(h + 1) * hd] for h in range(n_heads)]
+
+
+def mha(q_rows, k_rows, v_rows, hq, hkv, hd, causal=False):
+    """q_rows[t] = list of hq head vectors; k_rows/v_rows[t] = list of hkv head vectors.  Returns rows of hq*hd."""
+    out = []
+    for i, qh in enumerate(q_rows):
+        row = []
+        for h in range(hq):
+            g = (h * hkv) // hq                     # query head h reads KV head floor(h * Hkv / Hq)
+            vis = range(i + 1) if causal else range(len(k_rows))
+            row += attend_one(qh[h], [k_rows[j][g] for j in vis], [v_rows[j][g] for j in vis])
+        out.append(row)
+    return out
+
+
+def mlp_plain(x, W1, W2):
+    return matvec(W2, [gelu(v) for v in matvec(W1, x)])
+
+
+def mlp_gated(x, Wg, Wu, Wd, act):
+    g, u = matvec(Wg, x), matvec(Wu, x)
+    return matvec(Wd, [act(g[i]) * u[i] for i in range(len(g))])
+
+
+def L(a):
+    """numpy -> nested lists of Python floats."""
+    return np.asarray(a, dtype=F64).tolist()
+
+
+# ------------------------------------------------------------------ random tables with O(1) activations
+def random_weights(m, rng, only=None):
+    """name -> fp64 array; matrices ~ N(0, 2/sqrt(in)) so projections keep O(1..3) entries, gains in [0.5, 1.5]."""
+    w = {}
+    for name, shp in weight_shapes(m).items():
+        if only and not name.startswith(only):
+            continue
+        if is_gain(name):
+            w[name] = rng.uniform(0.5, 1.5, size=shp)
+        elif len(shp) == 2 and name not in ("vis.pos", "llm.pos", "act.pos", "txt.emb"):
+            w[name] = rng.standard_normal(shp) * (2.0 / math.sqrt(shp[1]))
+        else:
+            w[name] = rng.standard_normal(shp)
+    return w
+
+
+def close(a, b):
+    a, b = np.asarray(a, dtype=F64), np.asarray(b, dtype=F64)
+    assert a.shape == b.shape, (a.shape, b.shape)
+    assert np.max(np.abs(a - b)) <= 1e-9 * max(1.0, float(np.max(np.abs(b)))), float(np.max(np.abs(a - b)))
+
+
+# ------------------------------------------------------------------ vision encoder layer
+def test_vision_encoder_layer_composition():
+    rng = np.random.default_rng(101)
+    T, d, heads, hd, mlp = 6, 12, 2, 8, 20                      # heads*hd != d: a transposed W_o would not even fit
+    p = "vis.L0."
+    w = {p + "n1": rng.uniform(0.5, 1.5, d), p + "n2": rng.uniform(0.5, 1.5, d),
+         p + "wq": rng.standard_normal((heads * hd, d)), p + "wk": rng.standard_normal((heads * hd, d)),
+         p + "wv": rng.standard_normal((heads * hd, d)) * 0.5, p + "wo": rng.standard_normal((d, heads * hd)) * 0.3,
+         p + "w1": rng.standard_normal((mlp, d)) * 0.5, p + "w2": rng.standard_normal((d, mlp)) * 0.3}
+    x = rng.standard_normal((T, d))
+    got = O._encoder_layer(x.copy(), w, p, heads, hd, F64)
+
+    W = {k: L(v) for k, v in w.items()}
+    xs = L(x)
+    h = [rms(r, W[p + "n1"]) for r in xs]
+    q = [heads_of(matvec(W[p + "wq"], r), heads, hd) for r in h]
+    k = [heads_of(matvec(W[p + "wk"], r), heads, hd) for r in h]
+    v = [heads_of(matvec(W[p + "wv"], r), heads, hd) for r in h]
+    a = mha(q, k, v, heads, heads, hd)                           # bidirectional, no positions inside the layer
+    xs = [add(xs[t], matvec(W[p + "wo"], a[t])) for t in range(T)]
+    h2 = [rms(r, W[p + "n2"]) for r in xs]                       # second norm reads the UPDATED stream
+    want = [add(xs[t], mlp_plain(h2[t], W[p + "w1"], W[p + "w2"])) for t in range(T)]
+    close(got, want)
+    # the softmax rows really are far from uniform at this weight scale
+    lg = [sum(q[0][0][c] * k[j][0][c] for c in range(hd)) / math.sqrt(hd) for j in range(T)]
+    assert max(lg) - min(lg) > 1.0
+
+
+# ------------------------------------------------------------------ LLM decoder layer
+LLM_CASES = {
+    # GQA + RoPE + causal + SwiGLU (the Llama-style prefix decoder)
+    "gqa_rope_causal_swiglu": mini(CFG5, n_cam=1, img=28, patch=14, vis_layers=0, n_text=3, vocab=16, llm_layers=1, d=24,
+                                   hq=4, hkv=2, hd=8, mlp=20, mlp_kind="swiglu", rope=True, causal=True),
+    # MQA + RoPE + bidirectional + GeGLU
+    "mqa_rope_bidir_geglu": mini(CFG4, n_cam=1, img=28, patch=14, vis_layers=0, n_text=3, vocab=16, llm_layers=1, d=24,
+                                 hq=4, hkv=1, hd=8, mlp=20, mlp_kind="geglu", rope=True, causal=False),
+    # MHA, learned positions (none inside the layer), bidirectional, plain GeLU MLP
+    "mha_nope_bidir_gelu": mini(CFG1, n_text=3, vocab=16, llm_layers=1, d=24, hq=3, hkv=3, hd=8, mlp=20),
+}
+
+
+@pytest.mark.parametrize("key", list(LLM_CASES))
+def test_llm_layer_composition(key):
+    m = LLM_CASES[key]
+    rng = np.random.default_rng(202)
+    w = random_weights(m, rng, only="llm.L0.")
+    S = 7
+    x = rng.standard_normal((S, m.d))
+    pos = np.arange(3, 3 + S)                                    # positions are an argument: a non-zero start shows they are used
+    got_x, got_k, got_v = O.llm_layer(m, w, 0, x.copy(), pos, F64)
+
+    p = "llm.L0."
+    W = {k: L(v) for k, v in w.items()}
+    xs = L(x)
+    h = [rms(r, W[p + "n1"]) for r in xs]
+    q = [heads_of(matvec(W[p + "wq"], r), m.hq, m.hd) for r in h]
+    k = [heads_of(matvec(W[p + "wk"], r), m.hkv, m.hd) for r in h]
+    v = [heads_of(matvec(W[p + "wv"], r), m.hkv, m.hd) for r in h]
+    if m.rope:                                                   # q and k rotated, v not; the cache holds the rotated k
+        q = [[rotate(q[t][hh], int(pos[t])) for hh in range(m.hq)] for t in range(S)]
+        k = [[rotate(k[t][hh], int(pos[t])) for hh in range(m.hkv)] for t in range(S)]
+    a = mha(q, k, v, m.hq, m.hkv, m.hd, causal=m.causal)
+    xs = [add(xs[t], matvec(W[p + "wo"], a[t])) for t in range(S)]
+    h2 = [rms(r, W[p + "n2"]) for r in xs]
+    if m.mlp_kind == "gelu":
+        br = [mlp_plain(r, W[p + "w1"], W[p + "w2"]) for r in h2]
+    else:
+        act = silu if m.mlp_kind == "swiglu" else gelu
+        br = [mlp_gated(r, W[p + "wg"], W[p + "wu"], W[p + "wd"], act) for r in h2]
+    want = [add(xs[t], br[t]) for t in range(S)]
+    close(got_x, want)
+    close(got_k, k)
+    close(got_v, v)
+
+
+def test_vlm_forward_chains_the_layers_and_caches_every_layers_kv():
+    """vlm_forward = embed -> layer 0 -> layer 1 -> final norm, with kv[i] the K,V of layer i."""
+    m = mini(CFG4, n_cam=1, img=28, patch=14, vis_layers=0, vis_d=12, connector=True, n_text=3, vocab=16, llm_layers=2,
+             d=24, hq=4, hkv=1, hd=8, mlp=20)
+    rng = np.random.default_rng(203)
+    w = random_weights(m, rng)
+    image = rng.uniform(0, 1, (1, 3, 28, 28))
+    text = np.array([5, 0, 11])
+    out = O.vlm_forward(m, w, image, text, F64)
+    x = out["prefix"]
+    assert x.shape == (m.prefix_len, m.d)
+    pos = np.arange(m.prefix_len)
+    for i in range(2):
+        x, k, v = O.llm_layer(m, w, i, x, pos, F64)
+        close(out["kv"][i][0], k)
+        close(out["kv"][i][1], v)
+    g = L(w["llm.norm"])
+    close(out["hidden"], [rms(r, g) for r in L(x)])
+    # prefix rows: image tokens (patch (c,py,px) . W_patch + pos, connector) then the text-embedding rows
+    patch0 = [float(image[0, c, py, px]) for c in range(3) for py in range(14) for px in range(14)]
+    tok = add(matvec(L(w["vis.patch.w"]), patch0), L(w["vis.pos"][0]))
+    close(out["prefix"][0], matvec(L(w["conn.w"]), tok))
+    close(out["prefix"][m.n_img_tokens + 1], w["txt.emb"][0])
+
+
+# ------------------------------------------------------------------ action heads, end to end (one evaluation)
+def time_condition(W, t_arg, da):
+    half = da // 2
+    om = [math.exp(-math.log(10000.0) * i / half) for i in range(half)]
+    e = [math.sin(t_arg * o) for o in om] + [math.cos(t_arg * o) for o in om]
+    return matvec(W["act.t2"], [silu(v) for v in matvec(W["act.t1"], e)])
+
+
+def self_attention_rows(h, W, p, heads, hd):
+    q = [heads_of(matvec(W[p + "wq"], r), heads, hd) for r in h]
+    k = [heads_of(matvec(W[p + "wk"], r), heads, hd) for r in h]
+    v = [heads_of(matvec(W[p + "wv"], r), heads, hd) for r in h]
+    a = mha(q, k, v, heads, heads, hd)
+    return [matvec(W[p + "wo"], r) for r in a]
+
+
+def head_mlp(m, W, p, r):
+    if m.act_mlp_kind == "gelu":
+        return mlp_plain(r, W[p + "w1"], W[p + "w2"])
+    return mlp_gated(r, W[p + "wg"], W[p + "wu"], W[p + "wd"], silu if m.act_mlp_kind == "swiglu" else gelu)
+
+
+def restated_head(m, w, vlm, state, x, t_arg):
+    """v (or eps) [H][A] for one evaluation of the head, all four kinds, from the readings of the workloads."""
+    W = {k: L(v) for k, v in w.items() if k.startswith("act.")}
+    da, H, S = m.act_d, m.horizon, m.prefix_len
+    c_t = time_condition(W, t_arg, da)
+    tok = [matvec(W["act.in"], L(x[i])) for i in range(H)]
+    if m.head in ("A", "B"):                                     # time enters the action tokens additively
+        tok = [add(r, c_t) for r in tok]
+    if m.head in ("A", "C") or (m.head == "B" and m.state_dim > 0):
+        tok = [matvec(W["act.state"], L(state))] + tok           # state token first, no time on it
+    elif m.head == "D":
+        cog = L(vlm["hidden"][S - 1])                            # last prefix position = cognition feature
+        tok = [add(matvec(W["act.cond"], cog), c_t)] + tok       # condition token carries the time
+    if not (m.head == "B" and m.rope):                           # learned positions unless the head uses RoPE
+        tok = [add(tok[t], W["act.pos"][t]) for t in range(len(tok))]
+    Ta = len(tok)
+    z = tok
+    for i in range(m.act_layers):
+        p = f"act.L{i}."
+        if m.head == "A":
+            hd = da // m.act_heads
+            br = self_attention_rows([rms(r, W[p + "n1"]) for r in z], W, p, m.act_heads, hd)
+            z = [add(z[t], br[t]) for t in range(Ta)]
+            h = [rms(r, W[p + "n2"]) for r in z]
+            q = [heads_of(matvec(W[p + "cq"], r), m.hq, m.hd) for r in h]     # queries in the VLM's head geometry
+            Kc, Vc = vlm["kv"][m.llm_layers - 1]                              # the LAST LLM layer's cache, attended as is
+            a = mha(q, L(Kc), L(Vc), m.hq, m.hkv, m.hd)
+            z = [add(z[t], matvec(W[p + "co"], a[t])) for t in range(Ta)]
+            h = [rms(r, W[p + "n3"]) for r in z]
+            z = [add(z[t], head_mlp(m, W, p, h[t])) for t in range(Ta)]
+        elif m.head == "B":
+            h = [rms(r, W[p + "n1"]) for r in z]
+            q = [heads_of(matvec(W[p + "wq"], r), m.hq, m.hd) for r in h]
+            k = [heads_of(matvec(W[p + "wk"], r), m.hkv, m.hd) for r in h]
+            v = [heads_of(matvec(W[p + "wv"], r), m.hkv, m.hd) for r in h]
+            if m.rope:                                                         # positions continue after the prefix
+                q = [[rotate(q[t][hh], S + t) for hh in range(m.hq)] for t in range(Ta)]
+                k = [[rotate(k[t][hh], S + t) for hh in range(m.hkv)] for t in range(Ta)]
+            Kp, Vp = vlm["kv"][i]                                              # prefix cache of the SAME layer index
+            keys, vals = L(Kp) + k, L(Vp) + v                                  # [prefix ; own], no mask
+            a = mha(q, keys, vals, m.hq, m.hkv, m.hd)
+            z = [add(z[t], matvec(W[p + "wo"], a[t])) for t in range(Ta)]
+            h = [rms(r, W[p + "n2"]) for r in z]
+            z = [add(z[t], head_mlp(m, W, p, h[t])) for t in range(Ta)]
+        elif m.head == "C":
+            hd = da // m.act_heads
+            sc = [silu(v) for v in c_t]
+            mod = matvec(W[p + "ada1"], sc)
+            gam, bet = mod[:da], mod[da:]
+            h = [[n[c] * (1.0 + gam[c]) + bet[c] for c in range(da)] for n in (rms(r, W[p + "n1"]) for r in z)]
+            if i % 2 == 0:
+                br = self_attention_rows(h, W, p, m.act_heads, hd)
+            else:
+                F = L(vlm["hidden"])                                           # final-norm VLM features, all S positions
+                q = [heads_of(matvec(W[p + "cq"], r), m.act_heads, hd) for r in h]
+                k = [heads_of(matvec(W[p + "ck"], f), m.act_heads, hd) for f in F]
+                v = [heads_of(matvec(W[p + "cv"], f), m.act_heads, hd) for f in F]
+                br = [matvec(W[p + "co"], r) for r in mha(q, k, v, m.act_heads, m.act_heads, hd)]
+            z = [add(z[t], br[t]) for t in range(Ta)]
+            mod = matvec(W[p + "ada2"], sc)
+            gam, bet = mod[:da], mod[da:]
+            h = [[n[c] * (1.0 + gam[c]) + bet[c] for c in range(da)] for n in (rms(r, W[p + "n2"]) for r in z)]
+            z = [add(z[t], head_mlp(m, W, p, h[t])) for t in range(Ta)]
+        else:                                                                  # D: plain pre-norm layers
+            hd = da // m.act_heads
+            br = self_attention_rows([rms(r, W[p + "n1"]) for r in z], W, p, m.act_heads, hd)
+            z = [add(z[t], br[t]) for t in range(Ta)]
+            h = [rms(r, W[p + "n2"]) for r in z]
+            z = [add(z[t], head_mlp(m, W, p, h[t])) for t in range(Ta)]
+    first = Ta - H
+    return [matvec(W["act.out"], rms(z[first + i], W["act.norm"])) for i in range(H)]
+
+
+_VLM = dict(n_cam=1, img=28, patch=14, vis_layers=0, n_text=3, vocab=16)        # prefix of 4 + 3 = 7 positions
+HEAD_CASES = {
+    "A": mini(CFG1, img=16, n_text=3, vocab=16, llm_layers=2, d=24, hq=2, hkv=2, hd=8, mlp=20, act_layers=2, act_d=12,
+              act_heads=2, act_mlp=20, state_dim=5, horizon=4, act_dim=3),
+    "B_nope": mini(CFG2, **_VLM, llm_layers=2, d=24, hq=4, hkv=2, hd=8, mlp=20, act_layers=2, act_d=12, act_mlp=20,
+                   horizon=4, act_dim=3),
+    "B_rope": mini(CFG4, **_VLM, llm_layers=2, d=24, hq=4, hkv=1, hd=8, mlp=20, act_layers=2, act_d=12, act_mlp=20,
+                   state_dim=5, horizon=4, act_dim=3),
+    "C": mini(CFG3, **_VLM, shuffle=1, llm_layers=1, d=24, hq=2, hkv=2, hd=8, mlp=20, act_layers=2, act_d=12, act_heads=2,
+              act_mlp=20, state_dim=5, horizon=4, act_dim=3),
+    "D": mini(CFG5, **_VLM, llm_layers=1, d=24, hq=2, hkv=2, hd=8, mlp=20, act_layers=2, act_d=12, act_heads=2, act_mlp=20,
+              horizon=4, act_dim=3),
+}
+
+
+@pytest.mark.parametrize("key", list(HEAD_CASES))
+def test_head_velocity_composition(key):
+    m = HEAD_CASES[key]
+    rng = np.random.default_rng(300 + len(key))
+    w = random_weights(m, rng, only="act.")
+    S = m.prefix_len
+    # a hand-made VLM handoff (the head reads nothing else of the VLM): distinct K,V per LLM layer, distinct features
+    vlm = {"kv": [(rng.standard_normal((S, m.hkv, m.hd)) * 1.5, rng.standard_normal((S, m.hkv, m.hd)))
+                  for _ in range(m.llm_layers)],
+           "hidden": rng.standard_normal((S, m.d))}
+    state = rng.standard_normal(m.state_dim) if m.state_dim else None
+    x = rng.standard_normal((m.horizon, m.act_dim))
+    for t_arg in (0.0, 730.0):
+        got = O.head_velocity(m, w, vlm, state, x, t_arg, F64)
+        want = restated_head(m, w, vlm, state, x, t_arg)
+        close(got, want)
+    # the time argument matters for every head kind (it reaches C and D only through the layers / condition token)
+    a = O.head_velocity(m, w, vlm, state, x, 0.0, F64)
+    b = O.head_velocity(m, w, vlm, state, x, 730.0, F64)
+    assert np.max(np.abs(a - b)) > 1e-3
+    # and so does the handoff: another prefix cache / feature map changes the result
+    vlm2 = {"kv": [(k + 0.5 * rng.standard_normal(k.shape), v) for k, v in vlm["kv"]],
+            "hidden": vlm["hidden"] + 0.5 * rng.standard_normal(vlm["hidden"].shape)}
+    c = O.head_velocity(m, w, vlm2, state, x, 0.0, F64)
+    assert np.max(np.abs(a - c)) > 1e-3
+
+
+def test_action_chunk_is_solver_of_head_on_vlm_output():
+    """action_chunk feeds frame n's own VLM output, state and noise to the solver (Euler: x += v/n, t_k = k/n,
+    time argument 1000 t_k)."""
+    m = HEAD_CASES["B_rope"]
+    rng = np.random.default_rng(404)
+    w = random_weights(mini(m, vis_d=m.d), rng)
+    m2 = mini(m, vis_d=m.d, connector=False)
+    fr = {"image": rng.uniform(0, 1, (1, 3, 28, 28)), "text": np.array([1, 2, 3]), "state": rng.standard_normal(5),
+          "noise": rng.standard_normal((m.horizon, m.act_dim))}
+    vlm = O.vlm_forward(m2, w, fr["image"], fr["text"], F64)
+    x = [list(r) for r in L(fr["noise"])]
+    for k in range(m2.n_steps):
+        v = restated_head(m2, w, vlm, fr["state"], np.array(x), 1000.0 * k / m2.n_steps)
+        x = [[x[i][j] + v[i][j] / m2.n_steps for j in range(m2.act_dim)] for i in range(m2.horizon)]
+    close(O.action_chunk(m2, w, fr, F64), x)
