@@ -54,6 +54,13 @@ enum { VLA_MODE_COSCHED = 0, VLA_MODE_TWO_STREAM = 1, VLA_MODE_SERIAL = 2, VLA_M
 /* VLA_MODE_MULTI_STREAM: like TWO_STREAM but one (VLM, head) pair of CUDA streams per
  * request stream, created by the library; reported as extra context next to TWO_STREAM. */
 
+/* Pick policies of the persistent kernel.  TWO_PHASE is Algorithm 1; TWO_PHASE_G and TWO_PHASE_R are the two
+ * fairness-augmented variants of its Phase-2 score (Section 4, "Implementations"): s * G_k / (c_k + 1) with G_k the
+ * class's tiles still queued, and s / (c_k * R_k + 1) with R_k the class's shared-memory units per tile (registers
+ * are fixed per worker group here).  CLASS_ORDER and ROUND_ROBIN are resource-blind comparison points. */
+enum { VLA_POLICY_TWO_PHASE = 0, VLA_POLICY_CLASS_ORDER = 1, VLA_POLICY_ROUND_ROBIN = 2, VLA_POLICY_TWO_PHASE_G = 3,
+       VLA_POLICY_TWO_PHASE_R = 4 };
+
 enum { VLA_MLP_GELU = 0, VLA_MLP_SWIGLU = 1, VLA_MLP_GEGLU = 2 };
 enum { VLA_HANDOFF_KV_LAST = 0, VLA_HANDOFF_KV_ALL = 1, VLA_HANDOFF_FEATURES = 2, VLA_HANDOFF_COG = 3 };
 enum { VLA_HEAD_A = 0, VLA_HEAD_B = 1, VLA_HEAD_C = 2, VLA_HEAD_D = 3 };
@@ -85,8 +92,7 @@ typedef struct {
   int32_t mode;             /* VLA_MODE_* */
   int32_t n_streams;        /* request streams R */
   int32_t ring_depth;       /* frames in flight per request stream, >= 2 */
-  int32_t policy;           /* COSCHED pick: 0 = two-phase resource-aware pick (Algorithm 1), 1 = fixed class order,
-                             * 2 = round robin over the classes */
+  int32_t policy;           /* COSCHED pick: VLA_POLICY_* below */
   uint64_t wait_limit_ns;   /* bound of every device-side wait; 0 = default (5 s) */
   uint32_t trace_capacity;  /* tile records kept by the device trace; 0 = tracing off */
   int32_t workers_per_sm;   /* COSCHED worker groups per SM; 0 = default */
@@ -103,7 +109,8 @@ typedef struct {
   int64_t shape[4];
 } vla_tensor;
 
-/* One executed tile, as recorded by the device trace (all modes). */
+/* One executed tile, as recorded by the device trace (all modes).  In COSCHED mode the admission of a frame into
+ * the persistent kernel is recorded too, as a record with node = 0xFFFFFFFF, cls = 0xFF and t_start = t_end. */
 typedef struct {
   uint32_t inst;            /* request stream * ring_depth + ring slot */
   uint32_t node;            /* node index in the tile program */
@@ -123,6 +130,8 @@ typedef struct {
   int32_t succ_begin, succ_count; /* range in the successor array */
   int32_t smem_bytes, tmem_cols;  /* shared memory and tensor-memory columns one tile of the node occupies */
   char name[48];
+  double flops;             /* algorithmic FLOPs of the node: 2 M N K per matrix product, 4 Tq Tkv Hq hd per attention */
+  double weight_bytes;      /* bf16 weight bytes the node's tiles stream (0 for nodes without a weight matrix) */
 } vla_node_info;
 
 /* Bytes of device arena a context needs (weights, tile program, queues, per-frame buffers). */
@@ -187,6 +196,19 @@ int vla_policy_probe(int32_t n_cls, const int32_t* taus /*[n_cls*3]*/, const int
                      int32_t* cta_count, int32_t* u /*[3]*/, int32_t rr_start, int32_t u_max, int32_t* picked,
                      int32_t* phase);
 
+/* Same probe for the scoring variants of Section 4: policy = VLA_POLICY_TWO_PHASE, _TWO_PHASE_G (needs grid[n_cls],
+ * the G_k) or _TWO_PHASE_R (needs res[n_cls], the R_k); the unused array may be NULL. */
+int vla_policy_probe_ex(int32_t n_cls, const int32_t* taus, const int32_t* pending, const int32_t* feasible,
+                        int32_t* cta_count, int32_t* u, int32_t rr_start, int32_t u_max, int32_t policy, const int32_t* grid,
+                        const int32_t* res, int32_t* picked, int32_t* phase);
+
+/* Test hook for the failure path (no counterpart in the paper; Section 2.1 only states the dependency rule it
+ * breaks on purpose): adds `delta` to the dependency counter of `node` in ring slot `slot` of `stream`, with a host
+ * copy into the arena, while nothing is in flight.  A positive delta means the node never becomes ready: the next
+ * frame through that slot stalls, the idle watchdog runs out after wait_limit_ns, the persistent kernel returns and
+ * every later call reports the sticky VLA_ERR_TIMEOUT. */
+int vla_debug_bump_dependency(vla_ctx* ctx, int32_t stream, int32_t slot, int32_t node, int32_t delta);
+
 /* ---- stand-alone operators: the engine's tile bodies on caller-owned DEVICE tensors ------------------------
  * Both run asynchronously on `stream` (a cudaStream_t; NULL = default stream). */
 
@@ -223,6 +245,19 @@ int vla_op_attention_static(const void* q, const void* k, const void* v, void* o
  * out32 (fp32 [m,n]) and/or out16 (bf16 [m,n]) DEVICE, either may be NULL.  act: 0 none, 1 GeLU (tanh form), 2 SiLU. */
 int vla_op_linear(const void* a, const void* w, float* out32, void* out16, int32_t m, int32_t n, int32_t k, int32_t act,
                   void* stream);
+
+/* Every device-side wait of the operators is bounded (2 s by default); a wait that runs out makes the kernel set
+ * the call's error word and return, leaving garbage in the output.  vla_op_status waits for `stream` to drain and
+ * reads that word back: VLA_OK, or VLA_ERR_TIMEOUT when a wait ran out.  op selects the word: VLA_OP_LINEAR (one
+ * word per device, shared by all vla_op_linear calls on it: query before another call reuses it), VLA_OP_ATTENTION
+ * (the word at the start of `scratch`, DEVICE) or VLA_OP_ATTENTION_STATIC (the library's fixed array). */
+enum { VLA_OP_LINEAR = 0, VLA_OP_ATTENTION = 1, VLA_OP_ATTENTION_STATIC = 2 };
+int vla_op_status(int32_t op, const void* scratch, void* stream);
+
+/* Test hook: while drop_operand_loads is non-zero the operators' TMA producers issue no loads, so their consumers
+ * wait for operands that never come and the bounded waits (wait_limit_ns; 0 = the default 2 s) run out.  Process-wide;
+ * call with (0, 0) to restore normal operation. */
+int vla_debug_op_fault(int32_t drop_operand_loads, uint64_t wait_limit_ns);
 
 const char* vla_last_error(vla_ctx* ctx);
 int vla_destroy(vla_ctx* ctx);

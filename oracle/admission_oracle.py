@@ -20,10 +20,22 @@ of Section 3.4.1 says Phase 1 "picks one by round-robin".  ``rr_start`` lets the
 caller rotate the start of the Phase-1 scan; rr_start = 0 is the listing as
 printed.
 
+Two variants of the Phase-2 score (paper Section 4, "Implementations"):
+
+  -G  s_GRID = s * G_k / (c_k(j) + 1)      G_k = full grid size of kernel k, c_k(j) = its CTAs on SM j
+  -R  s_REG  = s / (c_k(j) * R_k + 1)      R_k = registers per CTA of kernel k
+
+Both are ratios of integers; they are compared exactly (Fraction), so a caller
+that compares them by integer cross-multiplication takes the same decisions.
+Phase 1, the strict '>' and the admit / completion rules are unchanged.
+
 Pins: tests/test_admission_oracle.py (hand-derived decision sequence, the
-paper's arithmetic identities 17 x 15 = 255 and 24 + 12 = 36 bits, invariants).
+paper's arithmetic identities 17 x 15 = 255 and 24 + 12 = 36 bits, invariants,
+hand-derived -G / -R cases).
 """
 from __future__ import annotations
+
+from fractions import Fraction
 
 U_MAX = 255
 TAU_MAX = 15
@@ -58,12 +70,27 @@ def complete(state: SMState, k: int, tau) -> None:
         state.u[x] = max(0, state.u[x] - tau[x])
 
 
-def admission_decision(state: SMState, taus, pending, feasible, rr_start: int = 0, u_max: int = U_MAX):
+def variant_score(state: SMState, k: int, tau, variant: str = "base", grid=None, regs=None, u_max: int = U_MAX):
+    """Phase-2 score of kernel k under the base policy or one of its two variants, as an exact ratio."""
+    s = score(state, tau, u_max)
+    c = state.cta_count[k]
+    if variant == "base":
+        return Fraction(s)
+    if variant == "G":
+        return Fraction(s * grid[k], c + 1)
+    if variant == "R":
+        return Fraction(s, c * regs[k] + 1)
+    raise ValueError(variant)
+
+
+def admission_decision(state: SMState, taus, pending, feasible, rr_start: int = 0, u_max: int = U_MAX,
+                       variant: str = "base", grid=None, regs=None):
     """One invocation: returns (kernel admitted or None, phase 1|2|0) and updates ``state``.
 
     taus[k] = (tau_TC, tau_ALU, tau_MEM); pending[k], feasible[k] booleans.  ``u_max`` is the
     saturation value of the utilisation registers (Section 3.3: 8-bit, 255); a caller whose SM
     holds fewer, larger units of work passes the value its counters reach on a full SM.
+    ``variant`` "G" needs grid[k] (G_k), "R" needs regs[k] (R_k).
     """
     n = len(taus)
     # Phase 1
@@ -81,7 +108,7 @@ def admission_decision(state: SMState, taus, pending, feasible, rr_start: int = 
             continue
         if not feasible[k]:
             continue
-        s = score(state, taus[k], u_max)
+        s = variant_score(state, k, taus[k], variant, grid, regs, u_max)
         if s > best_score:
             best_score, best_kernel = s, k
     if best_kernel is None:

@@ -25,7 +25,8 @@ _SOLVER = {"euler": 0, "ddim": 1}
 
 EXPORTS = ["vla_required_arena_bytes", "vla_init", "vla_load_weights", "vla_submit_frame", "vla_submit_frame_device",
            "vla_poll_actions", "vla_wait_idle", "vla_get_trace", "vla_reset_trace", "vla_program_info", "vla_debug_fetch",
-           "vla_get_counters", "vla_policy_probe", "vla_last_error", "vla_destroy",
+           "vla_get_counters", "vla_policy_probe", "vla_policy_probe_ex", "vla_debug_bump_dependency", "vla_last_error",
+           "vla_destroy", "vla_op_status", "vla_debug_op_fault",
            "vla_op_attention_scratch_bytes", "vla_op_attention", "vla_op_linear",
            "vla_op_attention_static_capacity", "vla_op_attention_static"]
 
@@ -58,7 +59,7 @@ class vla_trace_rec(C.Structure):
 class vla_node_info(C.Structure):
     _fields_ = [("op", C.c_int32), ("cls", C.c_int32), ("n_tiles", C.c_int32), ("n_pred", C.c_int32), ("phase", C.c_int32),
                 ("step", C.c_int32), ("succ_begin", C.c_int32), ("succ_count", C.c_int32), ("smem_bytes", C.c_int32), ("tmem_cols", C.c_int32),
-                ("name", C.c_char * 48)]
+                ("name", C.c_char * 48), ("flops", C.c_double), ("weight_bytes", C.c_double)]
 
 
 TRACE_DTYPE = np.dtype([("inst", "<u4"), ("node", "<u4"), ("tile", "<u4"), ("sm", "<u2"), ("worker", "u1"), ("cls", "u1"),
@@ -91,6 +92,11 @@ def load_library() -> C.CDLL:
     lib.vla_get_counters.argtypes = [C.c_void_p, P(C.c_uint64), P(C.c_uint64), P(C.c_uint64)]
     lib.vla_policy_probe.argtypes = [C.c_int32, P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32),
                                      C.c_int32, C.c_int32, P(C.c_int32), P(C.c_int32)]
+    lib.vla_policy_probe_ex.argtypes = [C.c_int32, P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32),
+                                        C.c_int32, C.c_int32, C.c_int32, P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32)]
+    lib.vla_debug_bump_dependency.argtypes = [C.c_void_p] + [C.c_int32] * 4
+    lib.vla_op_status.argtypes = [C.c_int32, C.c_void_p, C.c_void_p]
+    lib.vla_debug_op_fault.argtypes = [C.c_int32, C.c_uint64]
     lib.vla_op_attention_scratch_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, P(C.c_size_t)]
     lib.vla_op_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 6 + [C.c_void_p, C.c_size_t, C.c_void_p]
     lib.vla_op_linear.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 4 + [C.c_void_p]
@@ -308,7 +314,7 @@ class Engine:
         succ = (C.c_int32 * max(ns.value, 1))()
         self._check(self.lib.vla_program_info(self.ctx, nodes, nn.value, C.byref(nn), succ, ns.value, C.byref(ns)))
         out = [dict(op=n.op, cls=n.cls, n_tiles=n.n_tiles, n_pred=n.n_pred, phase=n.phase, step=n.step,
-                    smem_bytes=n.smem_bytes, tmem_cols=n.tmem_cols,
+                    smem_bytes=n.smem_bytes, tmem_cols=n.tmem_cols, flops=n.flops, weight_bytes=n.weight_bytes,
                     succ=[succ[n.succ_begin + i] for i in range(n.succ_count)], name=n.name.decode()) for n in nodes]
         return out
 
@@ -324,6 +330,10 @@ class Engine:
         self._check(self.lib.vla_get_counters(self.ctx, C.byref(a), C.byref(b), C.byref(c)))
         return dict(tiles=a.value, kernel_launches=b.value, persistent_launches=c.value)
 
+    def bump_dependency(self, stream, slot, node, delta):
+        """Test hook: adds ``delta`` to one node's dependency counter (see vla_debug_bump_dependency)."""
+        self._check(self.lib.vla_debug_bump_dependency(self.ctx, stream, slot, node, delta))
+
     def close(self):
         if self.ctx:
             self.lib.vla_destroy(self.ctx)
@@ -337,7 +347,11 @@ class Engine:
             pass
 
 
-def policy_probe(taus, pending, feasible, cta_count, u, rr_start=0, u_max=0):
+POLICIES = {"two_phase": 0, "class_order": 1, "round_robin": 2, "two_phase_g": 3, "two_phase_r": 4}
+OP_LINEAR, OP_ATTENTION, OP_ATTENTION_STATIC = 0, 1, 2
+
+
+def policy_probe(taus, pending, feasible, cta_count, u, rr_start=0, u_max=0, policy=0, grid=None, res=None):
     """Runs the device pick once on the GPU; returns (picked, phase, cta_count, u)."""
     lib = load_library()
     n = len(taus)
@@ -347,7 +361,13 @@ def policy_probe(taus, pending, feasible, cta_count, u, rr_start=0, u_max=0):
     cc = (C.c_int32 * n)(*[int(x) for x in cta_count])
     uu = (C.c_int32 * 3)(*[int(x) for x in u])
     picked, phase = C.c_int32(-1), C.c_int32(0)
-    rc = lib.vla_policy_probe(n, flat, pend, feas, cc, uu, rr_start, u_max, C.byref(picked), C.byref(phase))
+    gg = None if grid is None else (C.c_int32 * n)(*[int(x) for x in grid])
+    rs = None if res is None else (C.c_int32 * n)(*[int(x) for x in res])
+    if policy == 0 and grid is None and res is None:
+        rc = lib.vla_policy_probe(n, flat, pend, feas, cc, uu, rr_start, u_max, C.byref(picked), C.byref(phase))
+    else:
+        rc = lib.vla_policy_probe_ex(n, flat, pend, feas, cc, uu, rr_start, u_max, policy, gg, rs, C.byref(picked),
+                                     C.byref(phase))
     if rc != VLA_OK:
         raise VlaError(rc, "policy probe failed")
     return picked.value, phase.value, list(cc), list(uu)
@@ -406,3 +426,15 @@ def op_attention_static(q, k, v, out, hq, hkv, hd, causal=False, stream=None):
     if rc != VLA_OK:
         raise VlaError(rc, "vla_op_attention_static failed")
     return out
+
+
+def op_status(op, scratch=None, stream=None) -> int:
+    """Waits for ``stream`` and returns the operator's status word as a VLA_* code (VLA_OK or VLA_ERR_TIMEOUT)."""
+    return load_library().vla_op_status(op, None if scratch is None else scratch.data_ptr(), _stream_ptr(stream))
+
+
+def debug_op_fault(drop_operand_loads, wait_limit_ns=0):
+    """Test hook: make the operators' bounded waits run out (see vla_debug_op_fault)."""
+    rc = load_library().vla_debug_op_fault(int(bool(drop_operand_loads)), int(wait_limit_ns))
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_debug_op_fault failed")

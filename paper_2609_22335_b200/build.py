@@ -35,8 +35,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-fmad=false"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    if os.environ.get("VLA_TILE_TIMING"):
-        cmd += ["-DVLA_TILE_TIMING"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     cmd += ["-lcudart"]
     r = subprocess.run(cmd, capture_output=True, text=True)

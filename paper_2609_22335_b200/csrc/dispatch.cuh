@@ -7,6 +7,7 @@
 namespace vla {
 
 constexpr unsigned CTRL_EXITING = 0x80000000u;
+constexpr uint32_t TRACE_ADMIT_NODE = 0xFFFFFFFFu;   // node id of the trace record that marks a frame's admission
 constexpr int MAX_WORKERS = 3;
 constexpr int SM_CTL_BYTES = 1024;       // per-worker control block (mbarriers, row scales) handed to the tile bodies
 constexpr int SM_STATE_BASE = 2048;      // dispatcher state of the SM
@@ -44,6 +45,28 @@ __device__ __forceinline__ void set_error(const DeviceCtx& ctx, unsigned code, u
   }
 }
 
+// ------------------------------------------------------------------ doorbells inside an SM
+// The service warps and idle workers must not spin: every instruction they issue is taken from the worker warps that
+// share their scheduler (a claim loop polling flat out cost the tile bodies 10-40 % of their speed).  They wait on
+// an mbarrier instead -- suspended by the hardware, no issue slots -- which whoever has news for them rings; the
+// wait is bounded by a time hint, so a lost ring (two rings inside one phase look like none) only delays, never hangs.
+__device__ __forceinline__ void bell_ring(const void* bell) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bell)) : "memory");
+}
+// Returns when the bell was rung since the last successful wait or, at the latest, after about `hint_ns`.
+__device__ __forceinline__ bool bell_wait(const void* bell, uint32_t& parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bell)), "r"(parity), "r"(hint_ns)
+      : "memory");
+  if (ok) parity ^= 1u;
+  return ok != 0;
+}
+
 // ------------------------------------------------------------------ tensor memory (whole-warp calls)
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(cols) : "memory");
@@ -74,6 +97,12 @@ __device__ __forceinline__ unsigned long long queue_word(const DeviceCtx& ctx, u
 __device__ inline unsigned long long queue_reserve(const DeviceCtx& ctx, int cls, int n) {
   return atomicAdd(&ctx.queues[cls].tail, (unsigned long long)n);
 }
+// Ordering: a consumer may pop a ticket before that ticket's own commit (`avail` counts anybody's commits) and then
+// waits for the entry's generation tag with an acquire load.  So the entry store itself must publish everything the
+// producer has observed: every filling thread issues a device-scope fence before its (relaxed) entry stores
+// -- queue_fill_fence() -- and the thread that watched the dependency counter reach zero fences after that atomic.
+// The commit carries no ordering duty of its own.
+__device__ __forceinline__ void queue_fill_fence() { __threadfence(); }
 __device__ inline void queue_fill(const DeviceCtx& ctx, int cls, unsigned long long base, uint32_t inst, uint32_t node,
                                   uint32_t res_units, int first, int count, int stride) {
   const unsigned long long mask = (unsigned long long)ctx.q_capacity - 1;
@@ -82,7 +111,6 @@ __device__ inline void queue_fill(const DeviceCtx& ctx, int cls, unsigned long l
     *reinterpret_cast<volatile unsigned long long*>(ent + ((base + i) & mask)) = queue_word(ctx, base + i, inst, node, (uint32_t)i, res_units);
 }
 __device__ inline void queue_commit(const DeviceCtx& ctx, int cls, int n) {
-  __threadfence();
   atomicAdd(reinterpret_cast<unsigned long long*>(&ctx.queues[cls].avail), (unsigned long long)n);
 }
 // One thread pushes everything (admission of a frame's root tiles).
@@ -92,6 +120,7 @@ __device__ __forceinline__ uint32_t node_res_units(const NodeDesc& nd) {
 }
 __device__ inline void queue_push(const DeviceCtx& ctx, int cls, uint32_t inst, uint32_t node, int n) {
   const unsigned long long base = queue_reserve(ctx, cls, n);
+  queue_fill_fence();
   queue_fill(ctx, cls, base, inst, node, node_res_units(ctx.nodes[node]), 0, n, 1);
   queue_commit(ctx, cls, n);
 }
@@ -126,6 +155,10 @@ constexpr int DISPATCH_THREADS = 64;     // two service warps per SM (claim, ret
 constexpr long long PRIO_WINDOW_NS = 8000;   // an action-head tile may be claimed for a worker this close to the end of its tile
 constexpr int PREFETCH_MIN_AVAIL = 128;   // tiles are claimed ahead of need only from queues at least this deep
 constexpr int HELD_DEPTH = 1;            // claimed tiles a worker may have waiting
+constexpr unsigned CLAIM_NAP_NS = 60, CLAIM_NAP_MAX_NS = 240;   // claim warp, while a worker of its SM has nothing to run
+constexpr unsigned CLAIM_SLEEP_NS = 2000;    // claim warp, every worker busy: longest sleep without a ring
+constexpr unsigned RETIRE_SLEEP_NS = 4000;   // retire warp: longest sleep without a ring
+constexpr unsigned long long HEAD_WAIT_NS = 1500;   // an action-head tile nobody took for this long may go to a running worker
 
 struct ReadyItem {
   unsigned long long base;   // reserved queue range
@@ -162,10 +195,15 @@ struct SmState {
   int n_smem_units, n_tmem_units;
   PickState pick;
   unsigned tmem_base;
-  int waiter;                      // worker whose claimed tile is waiting for room (-1: none); others then admit only memory-free tiles
   volatile int quit;               // claim warp -> retire warp: everyone is leaving
   int smem_promised, tmem_promised;  // units of tiles handed to free workers that have not allocated them yet
+  unsigned room_wait;              // a worker waiting for room right now: smem units | tmem units << 8 | (worker + 1) << 16, else 0
+                                   // (the latest one when two wait); the claim warp keeps that room out of its offers
   volatile int ema_ns[N_CLASSES];  // running mean of tile durations per class on this SM (retire warp)
+  int tau_tab[N_CLASSES * 3];      // the classes' intensity tags (read by the workers when a tile ends)
+  unsigned long long bell_claim;   // rung by a worker that took a claimed tile or ran out of work
+  unsigned long long bell_retire;  // rung by a worker that posted a finished tile
+  unsigned long long bell_worker[MAX_WORKERS];   // rung by the claim warp when it hands worker w a tile or sends it home
   WorkerTile cur[MAX_WORKERS];     // the tile each worker is running (written by its leader)
   WorkerSlot slot[MAX_WORKERS];
 };
@@ -219,6 +257,10 @@ __device__ inline void try_admit(const DeviceCtx& ctx) {
   const uint32_t inst = rec->inst;
   const uint64_t frame = rec->frame;
   *reinterpret_cast<volatile uint64_t*>(ctx.inst_frame + inst) = frame;
+  {   // the frame's admission is a trace record of its own (node = TRACE_ADMIT_NODE): no tile of the frame may start earlier
+    const uint64_t now = gtimer();
+    write_trace(ctx, inst, TRACE_ADMIT_NODE, 0, 0, 0xFF, frame, now, now);
+  }
   __threadfence();
   for (int i = 0; i < ctx.n_roots; ++i) {
     int r = ctx.roots[i];
@@ -265,7 +307,18 @@ __device__ inline void complete_tile(const DeviceCtx& ctx, const WorkerTile& f, 
       }
     }
   }
+  if (slot->n_ready > 0) __threadfence();   // acquire side of the counters just read, before the entries are published
   if (f.op == OP_EMIT) atomicSub(&ctx.control->ctrl, 1u);
+}
+
+// u[x] += sign * tau[cls][x] on the SM's utilisation counters, with `cls` known only at run time: the class is matched
+// against loop-constant positions so that the tag table stays in registers.
+__device__ __forceinline__ void tau_add(int* u, const int* tau, int cls, int sign) {
+  int t0 = 0, t1 = 0, t2 = 0;
+#pragma unroll
+  for (int c = 0; c < N_CLASSES; ++c)
+    if (c == cls) { t0 = tau[c * 3]; t1 = tau[c * 3 + 1]; t2 = tau[c * 3 + 2]; }
+  atomicAdd(u + 0, sign * t0); atomicAdd(u + 1, sign * t1); atomicAdd(u + 2, sign * t2);
 }
 
 // ------------------------------------------------------------------ the two service warps of an SM
@@ -282,10 +335,7 @@ __device__ inline void retire_loop(const DeviceCtx& ctx, SmState* sm, int n_work
   const int lane = threadIdx.x & 31;
   const bool serving = lane < n_workers;
   WorkerSlot* slot = sm->slot + (serving ? lane : 0);
-  int tau[N_CLASSES * 3];
-  for (int c = 0; c < N_CLASSES; ++c)
-    for (int x = 0; x < 3; ++x) tau[c * 3 + x] = ctx.classes[c].tau[x];
-  unsigned nap = 40;
+  uint32_t bell_parity = 0;
   for (;;) {
     bool have_fin = false;
     if (serving && slot->done_state == 1) {
@@ -303,8 +353,10 @@ __device__ inline void retire_loop(const DeviceCtx& ctx, SmState* sm, int n_work
     __syncwarp();
     const bool any = __any_sync(0xffffffffu, have_fin);
     if (any) {
+      bool fenced = false;
       for (int w = 0; w < n_workers; ++w) {
         const int nr = sm->slot[w].n_ready;
+        if (nr > 0 && !fenced) { queue_fill_fence(); fenced = true; }
         for (int i = 0; i < nr; ++i) {
           const ReadyItem it = sm->slot[w].ready[i];
           queue_fill(ctx, it.cls, it.base, sm->slot[w].fin.inst, it.node, it.res_units, lane, it.n_tiles, 32);
@@ -316,11 +368,9 @@ __device__ inline void retire_loop(const DeviceCtx& ctx, SmState* sm, int n_work
         slot->n_ready = 0;
       }
       __syncwarp();
-      nap = 40;
     } else {
       if (sm->quit) break;
-      __nanosleep(nap);
-      if (nap < 120) nap += 40;
+      bell_wait(&sm->bell_retire, bell_parity, RETIRE_SLEEP_NS);
     }
   }
 }
@@ -330,13 +380,38 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
   const bool serving = lane < n_workers;
   Control* ctl = ctx.control;
   WorkerSlot* slot = sm->slot + (serving ? lane : 0);
-  int tau[N_CLASSES * 3], group[N_CLASSES];
-  for (int c = 0; c < N_CLASSES; ++c) {
-    for (int x = 0; x < 3; ++x) tau[c * 3 + x] = ctx.classes[c].tau[x];
-    group[c] = ctx.classes[c].group;
+  // Per-class constants live in registers: the arrays below are only ever read at loop-constant positions, and the
+  // shared/tensor-memory needs are packed one byte per class.  (This loop runs on every tile hand-over of the SM;
+  // arrays in local memory and global loads here cost 5 % of the whole step's throughput.)
+  int tau[N_CLASSES * 3], res_units[N_CLASSES];
+  unsigned group_mask[N_CLASSES];
+  unsigned long long su_pack = 0ull, tu_pack = 0ull;
+  {
+    int group[N_CLASSES];
+#pragma unroll
+    for (int c = 0; c < N_CLASSES; ++c) {
+#pragma unroll
+      for (int x = 0; x < 3; ++x) tau[c * 3 + x] = ctx.classes[c].tau[x];
+      group[c] = ctx.classes[c].group;
+      const int su = ctx.classes[c].smem_units, tu = ctx.classes[c].tmem_units;
+      res_units[c] = su > 0 ? su : 1;                                                 // R_k of the -R score
+      su_pack |= (unsigned long long)(su & 0xFF) << (8 * c);
+      tu_pack |= (unsigned long long)(tu & 0xFF) << (8 * c);
+    }
+#pragma unroll
+    for (int c = 0; c < N_CLASSES; ++c) {
+      unsigned m = 0;
+#pragma unroll
+      for (int j = 0; j < N_CLASSES; ++j)
+        if (group[j] == group[c]) m |= 1u << j;
+      group_mask[c] = m;
+    }
   }
+  const bool variant = ctx.policy == POLICY_TWO_PHASE_G || ctx.policy == POLICY_TWO_PHASE_R;
   uint64_t idle_start = 0, last_progress = gtimer();
-  unsigned iter = 0, nap = 60, lost = 0, prev_pending = 0;
+  unsigned iter = 0, nap = CLAIM_NAP_NS, lost = 0;
+  uint32_t bell_parity = 0;
+  uint64_t pending_since = 0;     // lane c: since when class c has had committed tiles without a break (0: it has none)
   bool leaving = false;
 
   for (;;) {
@@ -345,8 +420,17 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     long long av = lane < N_CLASSES ? ld_volatile_s64(&ctx.queues[lane].avail) : 0;
     const unsigned pending = __ballot_sync(0xffffffffu, av > 0) & ((1u << N_CLASSES) - 1u);
     const unsigned deep = __ballot_sync(0xffffffffu, av >= PREFETCH_MIN_AVAIL) & ((1u << N_CLASSES) - 1u);
-    const unsigned waiting = pending & prev_pending;   // classes that free workers elsewhere did not drain within a round
-    prev_pending = pending;
+    // classes whose tiles free workers elsewhere did not drain within head_wait_ns (by the clock, not by polling
+    // rounds: how fast this loop spins must not change what it decides)
+    if (av > 0) { if (pending_since == 0) pending_since = gtimer(); } else pending_since = 0;
+    const unsigned waiting = __ballot_sync(0xffffffffu, pending_since != 0 && gtimer() - pending_since >= HEAD_WAIT_NS) &
+                             ((1u << N_CLASSES) - 1u);
+    int grid[N_CLASSES];                               // G_k of the -G score: the class's tiles still to place
+    if (variant) {
+      const int depth = (int)(av < 0 ? 0 : (av > (1 << 20) ? (1 << 20) : av));
+#pragma unroll
+      for (int c = 0; c < N_CLASSES; ++c) grid[c] = __shfl_sync(0xffffffffu, depth, c);
+    }
     // ---- choose, lane by lane, which class each worker claims from
     int want = -1, promised_s = 0, promised_t = 0;
     bool to_prio = false;
@@ -363,7 +447,7 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         // short action-head tile is never stuck behind more than the tail of one tile.
         const unsigned act_mask = ((1u << N_KINDS) - 1u) << N_KINDS;
         const bool busy = slot->busy != 0 || queued > 0 || pq > 0;
-        const bool head_pending = ctx.policy == POLICY_TWO_PHASE && (pending & act_mask & ~avoid) != 0u;
+        const bool head_pending = pick_is_two_phase(ctx.policy) && (pending & act_mask & ~avoid) != 0u;
         unsigned cand;
         if (!busy) cand = head_pending ? (pending & act_mask) : pending;
         else if (pq == 0u && head_pending && (waiting & act_mask & ~avoid) != 0u && slot->busy != 0 &&
@@ -377,28 +461,41 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         const unsigned tmask = *reinterpret_cast<volatile unsigned*>(&sm->tmem_mask);
         // room: a free run of units now, and enough units left after what was promised to tiles already handed
         // to free workers of this SM (they allocate a moment later)
-        const int smem_left = sm->n_smem_units - __popcll(smask) - *reinterpret_cast<volatile int*>(&sm->smem_promised);
-        const int tmem_left = sm->n_tmem_units - __popc(tmask) - *reinterpret_cast<volatile int*>(&sm->tmem_promised);
-        unsigned feasible = 0;
-        for (int c = 0; c < N_CLASSES; ++c) {
-          const int su = ctx.classes[c].smem_units, tu = ctx.classes[c].tmem_units;
-          if (busy) { feasible |= 1u << c; continue; }
-          if (su <= smem_left && tu <= tmem_left && find_free(smask, su, sm->n_smem_units) >= 0 &&
-              find_free((unsigned long long)tmask, tu, sm->n_tmem_units) >= 0)
-            feasible |= 1u << c;
+        int smem_left = sm->n_smem_units - __popcll(smask) - *reinterpret_cast<volatile int*>(&sm->smem_promised);
+        int tmem_left = sm->n_tmem_units - __popc(tmask) - *reinterpret_cast<volatile int*>(&sm->tmem_promised);
+        {   // a worker of this SM that waits for room is served first: what it needs is not offered to the others
+          const unsigned rw = *reinterpret_cast<volatile unsigned*>(&sm->room_wait);
+          if (rw != 0u && (int)(rw >> 16) != w + 1) { smem_left -= (int)(rw & 0xFFu); tmem_left -= (int)((rw >> 8) & 0xFFu); }
         }
-        PickState ps;
-        for (int c = 0; c < N_CLASSES; ++c) ps.cta_count[c] = *reinterpret_cast<volatile int*>(&sm->pick.cta_count[c]);
-        for (int x = 0; x < 3; ++x) ps.u[x] = *reinterpret_cast<volatile int*>(&sm->pick.u[x]);
-        int phase;
-        want = pick_choose(N_CLASSES, tau, group, cand, feasible, ps, sm->pick.rr, ctx.policy, ctx.u_max, &phase);
+        unsigned feasible = 0;
+        if (busy) feasible = (1u << N_CLASSES) - 1u;   // a tile claimed ahead waits for room when its worker takes it
+        else
+          for (unsigned m = cand; m != 0u; m &= m - 1u) {                // only the candidate classes are looked at
+            const int c = __ffs((int)m) - 1;
+            const int su = (int)((su_pack >> (8 * c)) & 0xFFull), tu = (int)((tu_pack >> (8 * c)) & 0xFFull);
+            if (su <= smem_left && tu <= tmem_left && find_free(smask, su, sm->n_smem_units) >= 0 &&
+                find_free((unsigned long long)tmask, tu, sm->n_tmem_units) >= 0)
+              feasible |= 1u << c;
+          }
+        if ((cand & feasible) != 0u) {
+          PickState ps;
+#pragma unroll
+          for (int c = 0; c < N_CLASSES; ++c) ps.cta_count[c] = *reinterpret_cast<volatile int*>(&sm->pick.cta_count[c]);
+#pragma unroll
+          for (int x = 0; x < 3; ++x) ps.u[x] = *reinterpret_cast<volatile int*>(&sm->pick.u[x]);
+          int phase;
+          if (variant)
+            want = pick_choose(N_CLASSES, tau, group_mask, cand, feasible, ps, sm->pick.rr, ctx.policy, ctx.u_max, &phase, grid, res_units);
+          else
+            want = pick_choose(N_CLASSES, tau, group_mask, cand, feasible, ps, sm->pick.rr, ctx.policy, ctx.u_max, &phase);
+        }
         if (want >= 0) {
           if (!busy) {                                   // promised until the worker has allocated (or the pop is lost)
-            promised_s = ctx.classes[want].smem_units; promised_t = ctx.classes[want].tmem_units;
+            promised_s = (int)((su_pack >> (8 * want)) & 0xFFull); promised_t = (int)((tu_pack >> (8 * want)) & 0xFFull);
             atomicAdd(&sm->smem_promised, promised_s); atomicAdd(&sm->tmem_promised, promised_t);
           }
           atomicAdd(&sm->pick.cta_count[want], 1);     // counted from the claim on, so the next lane sees it
-          for (int x = 0; x < 3; ++x) atomicAdd(&sm->pick.u[x], tau[want * 3 + x]);
+          tau_add(&sm->pick.u[0], tau, want, 1);
           sm->pick.rr = (want + 1) % N_CLASSES;
         }
       }
@@ -424,10 +521,11 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
         __threadfence_block();
         if (to_prio) slot->prio_tail = slot->prio_tail + 1;
         else slot->held_tail = slot->held_tail + 1;      // the worker takes it as soon as it is free
+        bell_ring(&sm->bell_worker[lane]);
         progressed = true;
       } else {                                         // lost the race: undo the count
         atomicSub(&sm->pick.cta_count[want], 1);
-        for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[want * 3 + x]);
+        tau_add(&sm->pick.u[0], tau, want, -1);
         if (promised_s | promised_t) { atomicSub(&sm->smem_promised, promised_s); atomicSub(&sm->tmem_promised, promised_t); }
         lost = 1u << want;                             // look elsewhere in the next round, which follows at once
       }
@@ -464,13 +562,19 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
       const bool quiet = !serving || (slot->busy == 0 && slot->done_state == 0 && slot->held_tail == slot->held_head &&
                                       slot->prio_tail == slot->prio_head);
       if (__all_sync(0xffffffffu, quiet)) {
-        if (serving) { __threadfence_block(); slot->leave = 1; }
+        if (serving) { __threadfence_block(); slot->leave = 1; bell_ring(&sm->bell_worker[lane]); }
         __syncwarp();
-        if (lane == 0) { __threadfence_block(); sm->quit = 1; }
+        if (lane == 0) { __threadfence_block(); sm->quit = 1; bell_ring(&sm->bell_retire); }
         break;
       }
     }
-    if (!__any_sync(0xffffffffu, progressed || lost != 0u)) { __nanosleep(nap); if (nap < 240) nap += 60; } else nap = 60;
+    if (!__any_sync(0xffffffffu, progressed || lost != 0u)) {
+      // A free worker with nothing to run: poll the queues at short intervals (its scheduler slots are idle anyway).
+      // Every worker busy: sleep until one of them rings (it took its claimed tile, or ran dry) or the hint runs out.
+      const bool hungry = serving && slot->busy == 0 && slot->held_tail == slot->held_head && slot->prio_tail == slot->prio_head;
+      if (__any_sync(0xffffffffu, hungry)) { __nanosleep(nap); if (nap < CLAIM_NAP_MAX_NS) nap += CLAIM_NAP_NS; }
+      else { bell_wait(&sm->bell_claim, bell_parity, CLAIM_SLEEP_NS); nap = CLAIM_NAP_NS; }
+    } else nap = CLAIM_NAP_NS;
   }
 }
 
@@ -496,13 +600,19 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
     sm->pick.u[0] = sm->pick.u[1] = sm->pick.u[2] = 0;
     sm->pick.rr = (int)(blockIdx.x % N_CLASSES);
     sm->tmem_base = 0;
-    sm->waiter = -1;
     sm->quit = 0;
     sm->smem_promised = 0; sm->tmem_promised = 0;
+    sm->room_wait = 0u;
+    mbar_init(smem_u32(&sm->bell_claim), 1); mbar_init(smem_u32(&sm->bell_retire), 1);
+    for (int w = 0; w < MAX_WORKERS; ++w) mbar_init(smem_u32(&sm->bell_worker[w]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     for (int c = 0; c < N_CLASSES; ++c) sm->ema_ns[c] = 30000;
+    for (int c = 0; c < N_CLASSES; ++c)
+      for (int x = 0; x < 3; ++x) sm->tau_tab[c * 3 + x] = ctx.classes[c].tau[x];
     for (int w = 0; w < MAX_WORKERS; ++w) {
       sm->slot[w].held_tail = 0; sm->slot[w].held_head = 0; sm->slot[w].leave = 0; sm->slot[w].done_state = 0;
       sm->slot[w].prio_tail = 0; sm->slot[w].prio_head = 0; sm->slot[w].t_busy = 0;
+
       sm->slot[w].busy = 0;
       sm->slot[w].n_ready = 0;
     }
@@ -521,32 +631,20 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
     const int bar_id = worker + 1;
     WorkerSlot* slot = sm->slot + worker;
     unsigned long long tiles = 0;
-    int tau[N_CLASSES * 3];
-    for (int c = 0; c < N_CLASSES; ++c)
-      for (int x = 0; x < 3; ++x) tau[c * 3 + x] = ctx.classes[c].tau[x];
-#ifdef VLA_TILE_TIMING
-    long long ck_end = 0, ck_posted = 0, ck_seen = 0, ck_alloc = 0;
-#endif
+    uint32_t bell_parity = 0;
     for (;;) {
       if (wt == 0) {
         // take the tile the claim warp holds for this worker, then give it its exact memory need
         int st;
         unsigned naps = 0;
-#ifdef VLA_TILE_TIMING
-        const uint64_t tw0 = gtimer();
-#endif
         for (;;) {
           if (slot->prio_tail != slot->prio_head) { st = 3; break; }
           if (slot->held_tail != slot->held_head) { st = 1; break; }
           if (slot->leave) { st = 2; break; }
-          __nanosleep(naps < 64 ? 20 : 100);
+          if (naps < 8) __nanosleep(20);                               // a claimed tile is usually a moment away
+          else bell_wait(&sm->bell_worker[worker], bell_parity, 2000u);
           ++naps;
         }
-#ifdef VLA_TILE_TIMING
-        const uint64_t tw1 = gtimer();
-        ck_seen = clock64();
-        atomicAdd(ctl->dbg + 5, tw1 - tw0); atomicAdd(ctl->dbg + 6, 1ull);
-#endif
         WorkerTile& cur = sm->cur[worker];
         if (st == 1 || st == 3) {
           cur = st == 3 ? slot->prio : slot->held[slot->held_head % HELD_DEPTH];
@@ -555,6 +653,7 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
           __threadfence_block();
           if (st == 3) slot->prio_head = slot->prio_head + 1;
           else slot->held_head = slot->held_head + 1;   // the claim warp may refill the slot
+          bell_ring(&sm->bell_claim);
           const uint64_t lim = gtimer() + ctx.wait_limit_ns;
           bool ok = false;
           for (unsigned spin = 0;; ++spin) {
@@ -582,13 +681,14 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
                 if (cur.smem_units) atomicAnd(&sm->smem_mask, ~sbits);   // no tensor memory yet: give the shared memory back
               }
             }
+            if (spin == 0)        // waiting for room
+              *reinterpret_cast<volatile unsigned*>(&sm->room_wait) =
+                  (unsigned)cur.smem_units | ((unsigned)cur.tmem_units << 8) | ((unsigned)(worker + 1) << 16);
             __nanosleep(100);
             if ((spin & 255u) == 255u && (gtimer() > lim || ld_volatile_u32(&ctl->error) != 0u)) break;
           }
-#ifdef VLA_TILE_TIMING
-          atomicAdd(ctl->dbg + 7, gtimer() - tw1); atomicAdd(ctl->dbg + 8, 1ull);
-          ck_alloc = clock64();
-#endif
+          if ((*reinterpret_cast<volatile unsigned*>(&sm->room_wait) >> 16) == (unsigned)(worker + 1))
+            *reinterpret_cast<volatile unsigned*>(&sm->room_wait) = 0u;
           if (cur.succ_begin | cur.succ_count) {     // the claim warp's promise of room is settled either way
             atomicSub(&sm->smem_promised, cur.succ_begin); atomicSub(&sm->tmem_promised, cur.succ_count);
           }
@@ -612,19 +712,11 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
       tc.bar_id = bar_id;
       tc.error = &ctl->error;
       tc.tmaps = ctx.tmaps;
-      tc.dbg = ctl->dbg;
       tc.inputs = ctx.input_ptrs + (size_t)cmd.inst * N_FRAME_INPUTS;
       tc.amap_base = ctx.n_weight_tmaps + (int)cmd.inst * ctx.n_act_tmaps;
+      tc.drop_loads = 0;
       const uint64_t t0 = gtimer();
       tc.deadline = t0 + ctx.wait_limit_ns;
-#ifdef VLA_TILE_TIMING
-      if (wt == 0 && ck_end != 0 && cmd.t0 == 1) {     // SM clocks between two tiles of this worker
-        const long long now = clock64();
-        atomicAdd(ctl->dbg + 36, (unsigned long long)(ck_posted - ck_end)); atomicAdd(ctl->dbg + 37, (unsigned long long)(ck_seen - ck_posted));
-        atomicAdd(ctl->dbg + 38, (unsigned long long)(ck_alloc - ck_seen)); atomicAdd(ctl->dbg + 39, (unsigned long long)(now - ck_alloc));
-        atomicAdd(ctl->dbg + 22, 1ull);
-      }
-#endif
       // the frame id is only needed by the emit tile and by the trace
       const int n_op = __ldg(&n.op);
       // the node's successor range travels with the finished tile; read it now, while the description is hot
@@ -645,15 +737,12 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
       // barrier that opens the next tile).
       if (wt == 0) {
         ++tiles;
-#ifdef VLA_TILE_TIMING
-        ck_end = clock64();
-        ck_posted = ck_end;
-#endif
         if (cmd.t0 == 1) {
           if (cmd.smem_units) atomicAnd(&sm->smem_mask, ~(unit_bits(cmd.smem_units) << cmd.smem_unit0));
           if (cmd.tmem_units) atomicAnd(&sm->tmem_mask, ~(unsigned)(unit_bits(cmd.tmem_units) << cmd.tmem_unit0));
         }
         slot->busy = 0;
+        if (slot->held_tail == slot->held_head && slot->prio_tail == slot->prio_head) bell_ring(&sm->bell_claim);   // out of work
       } else if (wt == 32) {
         const uint64_t t1 = gtimer();
         WorkerTile d = cmd;
@@ -664,9 +753,6 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
           __nanosleep(40);
           if ((++naps & 0xFFFFu) == 0 && gtimer() - t0 > 2 * ctx.wait_limit_ns) break;   // retire warp gone: give up posting
         }
-#ifdef VLA_TILE_TIMING
-        atomicAdd(ctl->dbg + 9, gtimer() - t1); atomicAdd(ctl->dbg + 10, 1ull);
-#endif
         slot->done = d;
         // The tile's writes (all threads, ordered by the barrier above) must be visible device-wide before any
         // successor is released.  That fence is the retire warp's (first statement of complete_tile, after it has
@@ -674,8 +760,9 @@ __global__ void __launch_bounds__(MAX_WORKERS* WORKER_THREADS + DISPATCH_THREADS
         // keeps the writes ahead of the counter atomics without a device-scope round trip on the worker's path.
         __threadfence_block();
         slot->done_state = 1;
+        bell_ring(&sm->bell_retire);
         atomicSub(&sm->pick.cta_count[cmd.cls], 1);    // the pick's view of this SM, after the completion is on its way
-        for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], tau[cmd.cls * 3 + x]);
+        for (int x = 0; x < 3; ++x) atomicSub(&sm->pick.u[x], sm->tau_tab[cmd.cls * 3 + x]);
       }
     }
     if (wt == 0) atomicAdd(&ctl->tiles_done, tiles);
@@ -710,9 +797,9 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_node_kernel(DeviceCtx ctx,
   tc.bar_id = 1;
   tc.error = &ctx.control->error;
   tc.tmaps = ctx.tmaps;
-  tc.dbg = ctx.control->dbg;
   tc.inputs = ctx.input_ptrs + (size_t)(inst >= 0 ? inst : 0) * N_FRAME_INPUTS;
   tc.amap_base = ctx.n_weight_tmaps + (inst >= 0 ? inst : 0) * ctx.n_act_tmaps;
+  tc.drop_loads = 0;
   const uint64_t t0 = gtimer();
   tc.deadline = t0 + ctx.wait_limit_ns;
   const uint64_t frame = inst >= 0 ? ctx.inst_frame[inst] : 0;
@@ -730,11 +817,11 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_node_kernel(DeviceCtx ctx,
 
 // ------------------------------------------------------------------ pick probe (tests)
 __global__ void vla_pick_probe_kernel(int n_cls, const int* tau, unsigned pending, unsigned feasible, PickState* st,
-                                      int rr_start, int policy, int u_max, int* out) {
+                                      int rr_start, int policy, int u_max, const int* grid, const int* res, int* out) {
   int phase;
-  int group[PICK_MAX_CLASSES];
-  for (int i = 0; i < PICK_MAX_CLASSES; ++i) group[i] = i;   // one class per group: the paper's listing
-  int k = pick_choose(n_cls, tau, group, pending, feasible, *st, rr_start, policy, u_max, &phase);
+  unsigned group_mask[PICK_MAX_CLASSES];
+  for (int i = 0; i < PICK_MAX_CLASSES; ++i) group_mask[i] = 1u << i;   // one class per group: the paper's listing
+  int k = pick_choose(n_cls, tau, group_mask, pending, feasible, *st, rr_start, policy, u_max, &phase, grid, res);
   if (k >= 0) pick_commit(*st, k, tau);
   out[0] = k;
   out[1] = phase;

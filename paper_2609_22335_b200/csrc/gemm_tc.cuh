@@ -296,9 +296,6 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   const bool fok = gf < g.N;
   const uint32_t tmem_d = c.tmem;                 // accumulator columns [0, bt)
   float* rs_smem = reinterpret_cast<float*>(c.ctl + 256);        // [bt] row scales, in the control block
-#ifdef VLA_TILE_TIMING
-  uint64_t tt0; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt0));
-#endif
   // Whole warps take a role: lanes 1..31 of the producer and MMA warps park at __syncwarp (they must not
   // spin on a barrier, which would stall the issuing lane of the same warp).
   if (warp == 0) {
@@ -309,7 +306,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
     const void* wmap = tm + (size_t)g.wmap * 128;
     const void* w2map = tm + (size_t)g.w2map * 128;
     const void* amap = tm + (size_t)(c.amap_base + g.amap) * 128;
-    for (int kb = 0; kb < nkb; ++kb) {
+    for (int kb = 0; kb < nkb && !c.drop_loads; ++kb) {
       const int s = kb % S;
       const uint32_t ph = (uint32_t)(kb / S) & 1u;
       if (!mbar_wait(c, empty_bar(s), ph ^ 1u)) break;
@@ -331,9 +328,6 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       const uint32_t ph = (uint32_t)(kb / S) & 1u;
       ok = mbar_wait(c, full_bar(s), ph);
       if (!ok) break;
-#ifdef VLA_TILE_TIMING
-      if (kb == 0 && g.M > 512 && c.dbg) { uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); atomicAdd(c.dbg + 0, t - tt0); }
-#endif
       tc_fence_after();
       const uint32_t wsm = stage0 + (uint32_t)(s * stage_bytes);
       const uint32_t asm_ = wsm + GEMM_W_STAGE_BYTES;
@@ -371,12 +365,6 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
   const bool ready = mbar_wait(c, accum_bar, 0u);
   __syncwarp();
   tc_fence_after();
-#ifdef VLA_TILE_TIMING
-  uint64_t tt1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt1));
-#endif
-#ifdef VLA_TILE_TIMING
-  long long ck[6]; ck[0] = clock64();
-#endif
   float* St = reinterpret_cast<float*>(c.smem);   // [bt][128] fp32
   // The residual rows of this tile start their way into the staging area now (asynchronous 16-byte copies
   // through L2, no registers held), so their latency overlaps the accumulator read-out.
@@ -388,9 +376,6 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
     cp_async_wait_all();
   }
   if (g.rs_d > 0 || x_staged) worker_sync(c);     // row scales written by warps 2 and 3; residual rows landed
-#ifdef VLA_TILE_TIMING
-  ck[1] = clock64();
-#endif
   if (ready) {
     Phase1Args p1;
     p1.St = St; p1.rs = g.rs_d > 0 ? rs_smem : nullptr; p1.c_acc = g.c_acc; p1.c_x = g.c_x; p1.x_staged = x_staged;
@@ -403,14 +388,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
     else if (g.act == ACT_SILU) gemm_phase1<ACT_SILU>(p1);
     else gemm_phase1<ACT_NONE>(p1);
   }
-#ifdef VLA_TILE_TIMING
-  ck[2] = clock64();
-#endif
   worker_sync(c);
-#ifdef VLA_TILE_TIMING
-  ck[3] = clock64();
-  uint64_t tt2; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt2));
-#endif
   if (ready) {
     float* ssq_out = resolve<float>(c, g.ss_out);
     if (vec4) {
@@ -438,9 +416,6 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       } else if (!has_tab && !ptrs.out32 && !ssq_out) gemm_phase2_rows<false, false, true, false>(p2);      // bf16 only (q|k|v, MLP up)
       else if (!has_tab) gemm_phase2_rows<false, true, true, true>(p2);                                // residual stream
       else gemm_phase2_rows<true, true, true, true>(p2);
-#ifdef VLA_TILE_TIMING
-      ck[4] = clock64();
-#endif
       if (ssq_out) {
         __syncwarp();
         const int tok = warp + 4 * lane;                 // this lane's row: slot `lane` of this warp
@@ -475,29 +450,8 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
       }
     }
   }
-#ifdef VLA_TILE_TIMING
-  if (c.tid == 64 && g.M > 512 && c.dbg) {
-    uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    const int kind = ptrs.X ? 0 : (g.act != ACT_NONE ? 1 : (ptrs.outT ? 2 : 3));     // residual, w1, qkv, other
-    atomicAdd(c.dbg + 14 + 2 * kind, t - tt1); atomicAdd(c.dbg + 15 + 2 * kind, 1ull);
-    atomicAdd(c.dbg + 11, tt2 - tt1);
-    if (ptrs.X) { atomicAdd(c.dbg + 12, 1ull); }
-    ck[5] = clock64();
-    if (kind == 0 || kind == 2) {
-      const int b = kind == 0 ? 24 : 30;
-      for (int i = 0; i < 5; ++i) atomicAdd(c.dbg + b + i, (unsigned long long)(ck[i + 1] - ck[i]));
-      atomicAdd(c.dbg + b + 5, 1ull);
-    }
-  }
-#endif
   tc_fence_before();
   worker_sync(c);
-#ifdef VLA_TILE_TIMING
-  if (c.tid == 64 && g.M > 512 && c.dbg) {
-    uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    atomicAdd(c.dbg + 1, tt1 - tt0); atomicAdd(c.dbg + 2, t - tt1); atomicAdd(c.dbg + 3, 1ull); atomicAdd(c.dbg + 4, (unsigned long long)nkb);
-  }
-#endif
   if (c.tid == 0) {
     for (int s = 0; s < 2 * S + 1; ++s) mbar_inval(bar0 + 8u * s);
   }

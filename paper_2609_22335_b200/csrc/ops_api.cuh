@@ -6,6 +6,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "../../include/vla.h"
 #include "dispatch.cuh"
 
@@ -44,7 +46,18 @@ inline bool op_encode(CUtensorMap* out, const void* base, int64_t rows, int64_t 
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-__device__ __forceinline__ TileCtx op_tile_ctx(char* smem, char* ctl, uint32_t tmem, const void* maps, unsigned* err) {
+// Bound of the operators' device-side waits, and the test hook that makes one run out (vla_debug_op_fault).
+struct OpFault {
+  unsigned long long wait_limit_ns;
+  int drop_loads;
+};
+inline OpFault& op_fault() {
+  static OpFault f = {2000000000ull, 0};
+  return f;
+}
+
+__device__ __forceinline__ TileCtx op_tile_ctx(char* smem, char* ctl, uint32_t tmem, const void* maps, unsigned* err,
+                                               OpFault fault) {
   TileCtx tc;
   tc.arena = nullptr;          // Refs of the stand-alone operators are absolute device addresses
   tc.slot_base = 0;
@@ -56,14 +69,14 @@ __device__ __forceinline__ TileCtx op_tile_ctx(char* smem, char* ctl, uint32_t t
   tc.error = err;
   tc.tmaps = maps;
   tc.inputs = nullptr;
-  tc.dbg = nullptr;
   tc.amap_base = 0;
-  tc.deadline = gtimer() + 2000000000ull;
+  tc.drop_loads = fault.drop_loads;
+  tc.deadline = gtimer() + fault.wait_limit_ns;
   return tc;
 }
 
 __global__ void __launch_bounds__(WORKER_THREADS) vla_op_attention_kernel(AttnArgs a, const __grid_constant__ OpMaps maps,
-                                                                          int tmem_cols, unsigned* err) {
+                                                                          int tmem_cols, unsigned* err, OpFault fault) {
   extern __shared__ __align__(1024) char smem_raw[];
   __shared__ uint32_t tmem_base_s;
   __shared__ __align__(16) char ctl_block[1024];
@@ -71,7 +84,7 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_op_attention_kernel(AttnAr
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  TileCtx tc = op_tile_ctx(smem_raw, ctl_block, tmem_base_s, &maps, err);
+  TileCtx tc = op_tile_ctx(smem_raw, ctl_block, tmem_base_s, &maps, err, fault);
   tile_attention(tc, a, (int)blockIdx.x);
   tc_fence_before();
   __syncthreads();
@@ -79,7 +92,7 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_op_attention_kernel(AttnAr
 }
 
 __global__ void __launch_bounds__(WORKER_THREADS) vla_op_linear_kernel(GemmArgs g, const __grid_constant__ OpMaps maps,
-                                                                       int tmem_cols, unsigned* err) {
+                                                                       int tmem_cols, unsigned* err, OpFault fault) {
   extern __shared__ __align__(1024) char smem_raw[];
   __shared__ uint32_t tmem_base_s;
   __shared__ __align__(16) char ctl_block[1024];
@@ -87,7 +100,7 @@ __global__ void __launch_bounds__(WORKER_THREADS) vla_op_linear_kernel(GemmArgs 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  TileCtx tc = op_tile_ctx(smem_raw, ctl_block, tmem_base_s, &maps, err);
+  TileCtx tc = op_tile_ctx(smem_raw, ctl_block, tmem_base_s, &maps, err, fault);
   tile_gemm(tc, g, (int)blockIdx.x);
   tc_fence_before();
   __syncthreads();
@@ -110,6 +123,33 @@ __global__ void vla_op_transpose_kernel(const unsigned short* v, unsigned short*
 }
 
 constexpr size_t OP_ATTN_HEADER = 256;   // error word + padding in front of V^T
+
+// Error word of vla_op_linear: one per device, in a fixed device array of the library, looked up on the first call
+// made with that device current.  Calls on one device share it (see the header: check vla_op_status before
+// launching another operator call that could overwrite it).
+static __device__ __align__(256) unsigned g_op_linear_error[64];
+inline unsigned* op_linear_error_word() {
+  constexpr int kMax = 64;
+  static std::atomic<unsigned*> ptr[kMax];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMax) return nullptr;
+  unsigned* p = ptr[dev].load(std::memory_order_acquire);
+  if (!p) {
+    void* a = nullptr;
+    if (cudaGetSymbolAddress(&a, g_op_linear_error) != cudaSuccess || !a) return nullptr;
+    p = static_cast<unsigned*>(a);
+    ptr[dev].store(p, std::memory_order_release);
+  }
+  return p;
+}
+
+// Reads an operator's error word back after the stream has drained.
+inline int op_status_of(const unsigned* dev_word, cudaStream_t s) {
+  if (cudaStreamSynchronize(s) != cudaSuccess) return VLA_ERR_CUDA;
+  unsigned v = 0;
+  if (cudaMemcpy(&v, dev_word, sizeof v, cudaMemcpyDeviceToHost) != cudaSuccess) return VLA_ERR_CUDA;
+  return v == 0 ? VLA_OK : VLA_ERR_TIMEOUT;
+}
 
 inline int64_t op_pad(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 
@@ -147,13 +187,12 @@ inline int op_attention_run(const void* q, const void* k, const void* v, void* o
       !op_encode(&maps.m[1], k, tkv, (int64_t)hkv * hd, (int64_t)hkv * hd, a.bn) ||
       !op_encode(&maps.m[2], vt, (int64_t)hkv * hd, tkv, tpad, hd))
     return VLA_ERR_CUDA;
-  const int nbox = (hd + 63) / 64;
   const int smem = attn_smem_bytes(hd);
   int tmem_cols = 32;
   while (tmem_cols < a.bn + hd) tmem_cols <<= 1;
   if (cudaFuncSetAttribute(vla_op_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
     return VLA_ERR_CUDA;
-  vla_op_attention_kernel<<<hq * a.q_blocks, WORKER_THREADS, smem, s>>>(a, maps, tmem_cols, err);
+  vla_op_attention_kernel<<<hq * a.q_blocks, WORKER_THREADS, smem, s>>>(a, maps, tmem_cols, err, op_fault());
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 
@@ -196,13 +235,19 @@ int vla_op_linear(const void* a, const void* w, float* out32, void* out16, int32
   const int smem = gemm_smem_bytes(g.bt, g.stages);
   int tmem_cols = 32;
   while (tmem_cols < g.bt) tmem_cols <<= 1;
-  static unsigned* err = nullptr;       // one error word per process, allocated on first use
-  if (!err && cudaMalloc(&err, 256) != cudaSuccess) return VLA_ERR_CUDA;
+  unsigned* err = op_linear_error_word();     // this device's word (a fixed device array: nothing is allocated)
+  if (!err) return VLA_ERR_CUDA;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(err, 0, 4, s) != cudaSuccess) return VLA_ERR_CUDA;
   if (cudaFuncSetAttribute(vla_op_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return VLA_ERR_CUDA;
-  vla_op_linear_kernel<<<((n + GEMM_BM - 1) / GEMM_BM) * g.tiles_t, WORKER_THREADS, smem, s>>>(g, maps, tmem_cols, err);
+  vla_op_linear_kernel<<<((n + GEMM_BM - 1) / GEMM_BM) * g.tiles_t, WORKER_THREADS, smem, s>>>(g, maps, tmem_cols, err, op_fault());
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+int vla_debug_op_fault(int32_t drop_operand_loads, uint64_t wait_limit_ns) {
+  vla::op_fault().drop_loads = drop_operand_loads ? 1 : 0;
+  vla::op_fault().wait_limit_ns = wait_limit_ns ? wait_limit_ns : 2000000000ull;
+  return VLA_OK;
 }
 
 }  // extern "C"

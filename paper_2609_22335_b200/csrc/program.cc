@@ -194,6 +194,8 @@ class Builder {
     }
     p.nodes.push_back(n);
     p.node_names.push_back(name);
+    p.node_flops.push_back(0.0);
+    p.node_wbytes.push_back(0.0);
     preds.emplace_back();
     return (int)p.nodes.size() - 1;
   }
@@ -263,6 +265,11 @@ class Builder {
     const int feat_per_tile = g.dual ? GEMM_BM / 2 : GEMM_BM;
     n.n_tiles = (int)((g.N + feat_per_tile - 1) / feat_per_tile) * tiles_t;
     int id = add(n, name, g.dual ? KIND_GEMM2 : KIND_GEMM);
+    if (!init_mode) {
+      const double mats = g.dual ? 2.0 : 1.0;
+      p.node_flops[id] = mats * 2.0 * (double)g.M * (double)g.N * (double)wt.cols;
+      p.node_wbytes[id] = mats * 2.0 * (double)g.N * (double)wt.cols;
+    }
     read(id, A);
     if (o.X.buf >= 0) read(id, o.X);
     if (o.out32.buf >= 0) write(id, o.out32);
@@ -358,6 +365,7 @@ class Builder {
       a.v1map = act_map(all(kv1->vt), kv1->T, hs);
     }
     int id = add(n, name, KIND_ATTN);
+    if (!init_mode) p.node_flops[id] = 4.0 * (double)tq * (double)(a.t0 + a.t1) * (double)hq * (double)hd;
     read(id, q);
     read(id, all(kv0.qk)); read(id, all(kv0.vt));
     if (kv1) { read(id, all(kv1->qk)); read(id, all(kv1->vt)); }
@@ -980,13 +988,13 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   uint64_t want = tiles_per_frame * (uint64_t)p.n_inst + 1024;
   int cap = 1 << 12;
   while ((uint64_t)cap < want && cap < (1 << 24)) cap <<= 1;
+  if ((uint64_t)cap < want) { set_err(p, "tile program x frame slots needs a queue of more than 2^24 entries per class"); return false; }
   p.q_capacity = cap;
   p.off_q_entries = place(sizeof(QueueEntry) * (uint64_t)cap * N_CLASSES);
   p.admit_capacity = 1;
   while (p.admit_capacity < 2 * p.n_inst) p.admit_capacity <<= 1;
   p.off_admit = place(sizeof(AdmitRec) * p.admit_capacity);
   p.off_dep = place(sizeof(int32_t) * (uint64_t)nn * p.n_inst);
-  p.off_tiles_done = place(sizeof(int32_t) * (uint64_t)nn * p.n_inst);
   p.off_inst_frame = place(sizeof(uint64_t) * p.n_inst);
   p.off_slot_base = place(sizeof(uint64_t) * p.n_inst);
   p.off_input_ptrs = place(sizeof(uint64_t) * N_FRAME_INPUTS * p.n_inst);

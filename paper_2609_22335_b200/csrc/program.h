@@ -51,6 +51,7 @@ struct Program {
 
   std::vector<NodeDesc> nodes;
   std::vector<std::string> node_names;
+  std::vector<double> node_flops, node_wbytes;   // algorithmic FLOPs of a node and the weight bytes its tiles stream
   std::vector<int32_t> succ;
   std::vector<int32_t> roots;
   std::vector<int> init_nodes;          // nodes of the one-off constant precomputation (separate program)
@@ -73,7 +74,7 @@ struct Program {
   // arena layout (byte offsets)
   uint64_t off_weights = 0, off_consts = 0, off_nodes = 0, off_succ = 0, off_roots = 0, off_classes = 0,
            off_control = 0, off_queues = 0, off_q_entries = 0, off_admit = 0, off_dep = 0,
-           off_tiles_done = 0, off_inst_frame = 0, off_slot_base = 0, off_input_ptrs = 0, off_trace = 0, off_tmaps = 0,
+           off_inst_frame = 0, off_slot_base = 0, off_input_ptrs = 0, off_trace = 0, off_tmaps = 0,
            off_init_nodes = 0, off_slots = 0;
   uint64_t slot_bytes = 0, arena_bytes = 0, zero_bytes_begin = 0;
   int q_capacity = 0, admit_capacity = 0;

@@ -24,9 +24,10 @@ struct TileCtx {
   uint64_t deadline;    // %globaltimer value after which bounded waits give up
   unsigned int* error;  // sticky device error word
   const uint64_t* inputs;  // this frame slot's input pointer table
-  unsigned long long* dbg; // bring-up counters (VLA_TILE_TIMING builds only)
   const void* tmaps;    // tensor-map table (128 bytes per entry)
   int amap_base;        // index of this frame slot's first activation map
+  int drop_loads;       // test hook of the stand-alone operators: the TMA producer issues nothing, so the consumers'
+                        // bounded waits run out (0 everywhere else)
 };
 
 template <typename T>

@@ -404,7 +404,6 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
   x.q_entries = at<QueueEntry>(c, p.off_q_entries);
   x.admit_ring = at<AdmitRec>(c, p.off_admit);
   x.dep_count = at<int32_t>(c, p.off_dep);
-  x.tiles_done = at<int32_t>(c, p.off_tiles_done);
   x.inst_frame = at<uint64_t>(c, p.off_inst_frame);
   x.slot_base = at<uint64_t>(c, p.off_slot_base);
   x.input_ptrs = at<uint64_t>(c, p.off_input_ptrs);
@@ -621,6 +620,8 @@ int vla_program_info(vla_ctx* c, vla_node_info* nodes, size_t node_cap, size_t* 
       o.smem_bytes = n.smem_bytes; o.tmem_cols = n.tmem_cols;
       std::memset(o.name, 0, sizeof o.name);
       std::strncpy(o.name, p.node_names[i].c_str(), sizeof(o.name) - 1);
+      o.flops = p.node_flops[i];
+      o.weight_bytes = p.node_wbytes[i];
     }
   if (succ)
     for (size_t i = 0; i < std::min(succ_cap, p.succ.size()); ++i) succ[i] = p.succ[i];
@@ -659,66 +660,67 @@ int vla_get_counters(vla_ctx* c, uint64_t* tiles, uint64_t* kernel_launches, uin
     Control ctl;
     CU(cudaMemcpy(&ctl, c->dctx.control, sizeof ctl, cudaMemcpyDeviceToHost));
     *tiles = ctl.tiles_done;
-    if (getenv("VLA_PRINT_DBG"))
-      fprintf(stderr, "dbg: first_full %.2f us  mainloop %.2f us  epilogue %.2f us  tiles %llu  kb/tile %.1f\n",
-              ctl.dbg[3] ? ctl.dbg[0] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3] ? ctl.dbg[1] / 1e3 / ctl.dbg[3] : 0.0,
-              ctl.dbg[3] ? ctl.dbg[2] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3], ctl.dbg[3] ? (double)ctl.dbg[4] / ctl.dbg[3] : 0.0);
-    if (getenv("VLA_PRINT_DBG"))
-      fprintf(stderr, "dbg: epilogue phase 1 %.2f us (sync+ptrs %.2f us), tiles with residual %llu\n", ctl.dbg[3] ? ctl.dbg[11] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[3] ? ctl.dbg[13] / 1e3 / ctl.dbg[3] : 0.0, ctl.dbg[12]);
-    if (getenv("VLA_PRINT_DBG"))
-      fprintf(stderr, "dbg: epilogue (own warp, before the last barrier) by kind: residual %.2f us x %llu  gelu %.2f us x %llu  qkv %.2f us x %llu  other %.2f us x %llu\n",
-              ctl.dbg[15] ? ctl.dbg[14] / 1e3 / ctl.dbg[15] : 0.0, ctl.dbg[15], ctl.dbg[17] ? ctl.dbg[16] / 1e3 / ctl.dbg[17] : 0.0, ctl.dbg[17],
-              ctl.dbg[19] ? ctl.dbg[18] / 1e3 / ctl.dbg[19] : 0.0, ctl.dbg[19], ctl.dbg[21] ? ctl.dbg[20] / 1e3 / ctl.dbg[21] : 0.0, ctl.dbg[21]);
-    if (getenv("VLA_PRINT_DBG"))
-      for (int b = 24; b <= 30; b += 6)
-        if (ctl.dbg[b + 5])
-          fprintf(stderr, "dbg: epilogue clocks (%s): ptrs+stage+sync %.0f  phase1 %.0f  sync %.0f  phase2 rows %.0f  row sums+rest %.0f (x %llu)\n",
-                  b == 24 ? "residual" : "qkv", (double)ctl.dbg[b] / ctl.dbg[b + 5], (double)ctl.dbg[b + 1] / ctl.dbg[b + 5],
-                  (double)ctl.dbg[b + 2] / ctl.dbg[b + 5], (double)ctl.dbg[b + 3] / ctl.dbg[b + 5], (double)ctl.dbg[b + 4] / ctl.dbg[b + 5], ctl.dbg[b + 5]);
-    if (getenv("VLA_PRINT_DBG") && ctl.dbg[22])
-      fprintf(stderr, "dbg: between two tiles of a worker (SM clocks): post %.0f  wait for the next tile %.0f  allocate %.0f  barrier + setup %.0f (x %llu)\n",
-              (double)ctl.dbg[36] / ctl.dbg[22], (double)ctl.dbg[37] / ctl.dbg[22], (double)ctl.dbg[38] / ctl.dbg[22],
-              (double)ctl.dbg[39] / ctl.dbg[22], ctl.dbg[22]);
-    if (getenv("VLA_PRINT_DBG"))
-      fprintf(stderr, "dbg: wait-for-claim %.2f us x %llu  wait-for-room %.2f us x %llu  wait-to-post %.2f us x %llu\n",
-              ctl.dbg[6] ? ctl.dbg[5] / 1e3 / ctl.dbg[6] : 0.0, ctl.dbg[6], ctl.dbg[8] ? ctl.dbg[7] / 1e3 / ctl.dbg[8] : 0.0,
-              ctl.dbg[8], ctl.dbg[10] ? ctl.dbg[9] / 1e3 / ctl.dbg[10] : 0.0, ctl.dbg[10]);
   }
   if (kernel_launches) *kernel_launches = c->n_kernel_launches;
   if (persistent_launches) *persistent_launches = c->n_persistent_launches;
   return VLA_OK;
 }
 
-int vla_policy_probe(int32_t n_cls, const int32_t* taus, const int32_t* pending, const int32_t* feasible, int32_t* cta_count,
-                     int32_t* u, int32_t rr_start, int32_t u_max, int32_t* picked, int32_t* phase) {
+int vla_policy_probe_ex(int32_t n_cls, const int32_t* taus, const int32_t* pending, const int32_t* feasible,
+                        int32_t* cta_count, int32_t* u, int32_t rr_start, int32_t u_max, int32_t policy, const int32_t* grid,
+                        const int32_t* res, int32_t* picked, int32_t* phase) {
   if (n_cls < 1 || n_cls > PICK_MAX_CLASSES || !taus || !pending || !feasible || !cta_count || !u || !picked || !phase)
     return VLA_ERR_INVALID;
-  PickState st;
-  std::memset(&st, 0, sizeof st);
+  if (policy < POLICY_TWO_PHASE || policy > POLICY_TWO_PHASE_R) return VLA_ERR_INVALID;
+  if ((policy == POLICY_TWO_PHASE_G && !grid) || (policy == POLICY_TWO_PHASE_R && !res)) return VLA_ERR_INVALID;
+  // inputs and outputs of the probe in one block: one allocation, one copy each way
+  struct Block { PickState st; int tau[PICK_MAX_CLASSES * 3]; int grid[PICK_MAX_CLASSES]; int res[PICK_MAX_CLASSES]; int out[2]; } h;
+  std::memset(&h, 0, sizeof h);
   unsigned pm = 0, fm = 0;
   for (int k = 0; k < n_cls; ++k) {
-    st.cta_count[k] = cta_count[k];
+    h.st.cta_count[k] = cta_count[k];
     if (pending[k]) pm |= 1u << k;
     if (feasible[k]) fm |= 1u << k;
+    for (int x = 0; x < 3; ++x) h.tau[k * 3 + x] = taus[k * 3 + x];
+    h.grid[k] = grid ? grid[k] : 1;
+    h.res[k] = res ? res[k] : 1;
   }
-  for (int x = 0; x < 3; ++x) st.u[x] = u[x];
-  int* d_tau = nullptr; PickState* d_st = nullptr; int* d_out = nullptr;
-  if (cudaMalloc(&d_tau, sizeof(int) * n_cls * 3) != cudaSuccess || cudaMalloc(&d_st, sizeof st) != cudaSuccess ||
-      cudaMalloc(&d_out, 8) != cudaSuccess)
-    return VLA_ERR_CUDA;
-  int out[2] = {-1, 0};
-  cudaMemcpy(d_tau, taus, sizeof(int) * n_cls * 3, cudaMemcpyHostToDevice);
-  cudaMemcpy(d_st, &st, sizeof st, cudaMemcpyHostToDevice);
-  vla_pick_probe_kernel<<<1, 1>>>(n_cls, d_tau, pm, fm, d_st, rr_start, POLICY_TWO_PHASE, u_max > 0 ? u_max : PICK_U_MAX, d_out);
+  for (int x = 0; x < 3; ++x) h.st.u[x] = u[x];
+  h.out[0] = -1;
+  Block* d = nullptr;
+  if (cudaMalloc(&d, sizeof h) != cudaSuccess) return VLA_ERR_CUDA;
+  cudaMemcpy(d, &h, sizeof h, cudaMemcpyHostToDevice);
+  vla_pick_probe_kernel<<<1, 1>>>(n_cls, d->tau, pm, fm, &d->st, rr_start, policy, u_max > 0 ? u_max : PICK_U_MAX, d->grid,
+                                  d->res, d->out);
   cudaError_t e = cudaDeviceSynchronize();
-  cudaMemcpy(out, d_out, 8, cudaMemcpyDeviceToHost);
-  cudaMemcpy(&st, d_st, sizeof st, cudaMemcpyDeviceToHost);
-  cudaFree(d_tau); cudaFree(d_st); cudaFree(d_out);
+  if (e == cudaSuccess) e = cudaMemcpy(&h, d, sizeof h, cudaMemcpyDeviceToHost);
+  cudaFree(d);
   if (e != cudaSuccess) return VLA_ERR_CUDA;
-  for (int k = 0; k < n_cls; ++k) cta_count[k] = st.cta_count[k];
-  for (int x = 0; x < 3; ++x) u[x] = st.u[x];
-  *picked = out[0];
-  *phase = out[1];
+  for (int k = 0; k < n_cls; ++k) cta_count[k] = h.st.cta_count[k];
+  for (int x = 0; x < 3; ++x) u[x] = h.st.u[x];
+  *picked = h.out[0];
+  *phase = h.out[1];
+  return VLA_OK;
+}
+
+int vla_policy_probe(int32_t n_cls, const int32_t* taus, const int32_t* pending, const int32_t* feasible, int32_t* cta_count,
+                     int32_t* u, int32_t rr_start, int32_t u_max, int32_t* picked, int32_t* phase) {
+  return vla_policy_probe_ex(n_cls, taus, pending, feasible, cta_count, u, rr_start, u_max, POLICY_TWO_PHASE, nullptr, nullptr,
+                             picked, phase);
+}
+
+int vla_debug_bump_dependency(vla_ctx* c, int32_t stream, int32_t slot, int32_t node, int32_t delta) {
+  if (!c) return VLA_ERR_INVALID;
+  const Program& p = c->prog;
+  if (stream < 0 || stream >= p.n_streams || slot < 0 || slot >= p.ring_depth || node < 0 || node >= (int)p.nodes.size())
+    return fail(c, VLA_ERR_INVALID, "bad stream, slot or node");
+  if (c->pending_frames != 0) return fail(c, VLA_ERR_STATE, "frames are in flight");
+  CU(cudaDeviceSynchronize());
+  int32_t* cnt = c->dctx.dep_count + (size_t)(stream * p.ring_depth + slot) * p.nodes.size() + node;
+  int32_t v = 0;
+  CU(cudaMemcpy(&v, cnt, sizeof v, cudaMemcpyDeviceToHost));
+  v += delta;
+  CU(cudaMemcpy(cnt, &v, sizeof v, cudaMemcpyHostToDevice));
   return VLA_OK;
 }
 
@@ -804,6 +806,24 @@ int vla_op_attention_static(const void* q, const void* k, const void* v, void* o
   if (rc != VLA_OK) return rc;
   // op_attention_run clears the error word itself; V^T is fully rewritten for the rows and tokens it reads
   return vla::op_attention_run(q, k, v, out, tq, tkv, hq, hkv, hd, causal, scratch, static_cast<cudaStream_t>(stream));
+}
+
+int vla_op_status(int32_t op, const void* scratch, void* stream) {
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (op == VLA_OP_LINEAR) {
+    unsigned* w = vla::op_linear_error_word();
+    return w ? vla::op_status_of(w, s) : VLA_ERR_CUDA;
+  }
+  if (op == VLA_OP_ATTENTION) {
+    if (!scratch) return VLA_ERR_INVALID;
+    return vla::op_status_of(static_cast<const unsigned*>(scratch), s);
+  }
+  if (op == VLA_OP_ATTENTION_STATIC) {
+    void* p = nullptr;
+    int rc = static_scratch_for_current_device(&p);
+    return rc != VLA_OK ? rc : vla::op_status_of(static_cast<const unsigned*>(p), s);
+  }
+  return VLA_ERR_INVALID;
 }
 
 }  // extern "C"

@@ -213,7 +213,6 @@ struct Control {                 // polled words and hot counters live on separa
   unsigned long long pad2[15];
   unsigned long long tiles_done;
   unsigned long long trace_count;
-  unsigned long long dbg[40];    // scratch counters for kernel bring-up (see VLA_TILE_TIMING)
 };
 
 enum DevError : uint32_t {
@@ -235,7 +234,6 @@ struct DeviceCtx {
   QueueEntry* q_entries;         // [N_CLASSES][q_capacity]
   AdmitRec* admit_ring;
   int32_t* dep_count;            // [n_inst][n_nodes]
-  int32_t* tiles_done;           // [n_inst][n_nodes]
   uint64_t* inst_frame;          // [n_inst] frame id currently owning the slot
   const uint64_t* slot_base;     // [n_inst] arena offset of the instance's buffers
   const uint64_t* input_ptrs;    // [n_inst][N_FRAME_INPUTS] device addresses of the frame's input arrays

@@ -1,7 +1,9 @@
 """Pins of the admission-decision oracle (paper Algorithm 1, Section 3.3) on hand-derived cases."""
 import random
 
-from oracle.admission_oracle import (SMState, admission_decision, admit, complete, score, quantise_tau,
+from fractions import Fraction
+
+from oracle.admission_oracle import (SMState, admission_decision, admit, complete, score, quantise_tau, variant_score,
                                      U_MAX, TAU_MAX)
 
 
@@ -96,3 +98,57 @@ def test_random_invariants():
 
 def test_quantise_tau():
     assert [quantise_tau(x) for x in (0.0, 0.03, 0.374, 1.0, 1.7)] == [0, 0, 6, 15, 15]
+
+
+def test_grid_progress_variant_hand_derived():
+    # the state of test_hand_derived_sequence before its third call: U = (15, 6, 12), one CTA of A and of B resident,
+    # s_A = 4827, s_B = 3183 (the base policy admits A)
+    taus = [(15, 2, 3), (0, 4, 9)]
+
+    def fresh():
+        st = SMState(2)
+        st.cta_count = [1, 1]
+        st.u = [15, 6, 12]
+        return st
+    # -G: s * G_k / (c_k + 1).  A has a 2-CTA grid, B a 30-CTA grid: 4827*2/2 = 4827 < 3183*30/2 = 47745 -> B
+    st = fresh()
+    assert variant_score(st, 0, taus[0], "G", grid=[2, 30]) == 4827
+    assert variant_score(st, 1, taus[1], "G", grid=[2, 30]) == 47745
+    assert admission_decision(st, taus, [True, True], [True, True], variant="G", grid=[2, 30]) == (1, 2)
+    # equal grids: the factor G/(c+1) is common and the base order stands
+    assert admission_decision(fresh(), taus, [True, True], [True, True], variant="G", grid=[8, 8]) == (0, 2)
+    # the score decays as a kernel accumulates CTAs: with 3 CTAs of A resident, 4 * s_B > 2 * s_A flips the order
+    st = fresh()
+    st.cta_count = [3, 1]
+    assert variant_score(st, 0, taus[0], "G", grid=[8, 8]) == Fraction(4827 * 8, 4)
+    assert variant_score(st, 1, taus[1], "G", grid=[8, 8]) == Fraction(3183 * 8, 2)
+    assert admission_decision(st, taus, [True, True], [True, True], variant="G", grid=[8, 8]) == (1, 2)
+    # Phase 1 is untouched by the variants
+    st = SMState(2)
+    assert admission_decision(st, taus, [True, True], [True, True], variant="G", grid=[1, 1000]) == (0, 1)
+
+
+def test_register_variant_hand_derived():
+    taus = [(15, 2, 3), (0, 4, 9)]
+
+    def fresh():
+        st = SMState(2)
+        st.cta_count = [1, 1]
+        st.u = [15, 6, 12]
+        return st
+    # -R: s / (c_k * R_k + 1).  A uses 64 registers per CTA, B 32: 4827/65 = 74.3 < 3183/33 = 96.5 -> B
+    st = fresh()
+    assert variant_score(st, 0, taus[0], "R", regs=[64, 32]) == Fraction(4827, 65)
+    assert variant_score(st, 1, taus[1], "R", regs=[64, 32]) == Fraction(3183, 33)
+    assert admission_decision(st, taus, [True, True], [True, True], variant="R", regs=[64, 32]) == (1, 2)
+    # equal register counts: the base order stands
+    assert admission_decision(fresh(), taus, [True, True], [True, True], variant="R", regs=[48, 48]) == (0, 2)
+    # a kernel with no CTA resident is not penalised at all (denominator 1) -- but then Phase 1 takes it anyway
+    st = fresh()
+    st.cta_count = [1, 0]
+    assert admission_decision(st, taus, [True, True], [True, True], variant="R", regs=[64, 32]) == (1, 1)
+    # exact ties keep the first seen: s_0/(1*1+1) == s_1/(1*3+1) with s_1 = 2 s_0
+    taus2 = [(1, 0, 0), (2, 0, 0)]
+    st = SMState(2)
+    st.cta_count = [1, 1]
+    assert admission_decision(st, taus2, [True, True], [True, True], variant="R", regs=[1, 3]) == (0, 2)

@@ -32,10 +32,13 @@ def test_full_size_sampled_parity(m, frames, check_two_stream):
         ref = O.action_chunk(m, w, fr[r][n], np.float32)
         rel = float(np.linalg.norm(got[r][n] - ref) / np.linalg.norm(ref))
         mx = float(np.max(np.abs(got[r][n] - ref)))
-        # DDIM with untrained weights amplifies the sample ~5-7x: its absolute bound is taken relative to the rms
-        scale = max(1.0, float(np.sqrt(np.mean(ref * ref)))) if m.solver == "ddim" else 1.0
+        rms = float(np.sqrt(np.mean(ref * ref)))
+        print(f"{m.name} stream {r} frame {n}: rel-L2 {rel:.2e}, max-abs {mx:.3e}, chunk rms {rms:.2f}")
+        # DDIM chunks (rms 4-7 with an untrained eps-network): the absolute bound is taken relative to the chunk's
+        # scale, see tests/test_gpu_parity.py::_check_vs_oracle; Euler chunks are held to the plain 3e-2
+        scale = max(1.0, rms) if m.solver == "ddim" else 1.0
         assert rel <= REL_L2_TOL, (m.name, r, n, rel)
-        assert mx <= MAX_ABS_TOL * scale, (m.name, r, n, mx, scale)
+        assert mx <= MAX_ABS_TOL * scale, (m.name, r, n, mx, rms)
     # every chunk of every stream is finite and distinct streams differ
     for r in range(R):
         for n in range(frames):

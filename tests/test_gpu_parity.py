@@ -47,17 +47,25 @@ def _run(m, w, frames, mode, **kw):
 
 
 def _check_vs_oracle(m, w, frames, got, dtype=np.float32):
-    worst = (0.0, 0.0)
+    """Every chunk within rel-L2 <= 1e-2 and max-abs <= 3e-2 of the oracle.
+
+    DDIM chunks: deterministic DDIM with an untrained eps-network multiplies the sample by 1/sqrt(alpha_bar) of the
+    first timestep (4-7x here), so chunks have rms 4-7 and peak values 13-25, where an absolute 3e-2 is finer than
+    the bf16 spacing of the operands (2^-8 relative).  A head whose only deviation from the oracle is rounding its
+    matrix-product inputs to bf16 already shows max-abs 1.7e-2 on the reduced workload (CPU emulation), the GPU
+    path 3.3e-2.  For that solver the absolute bound is therefore taken relative to the chunk's scale,
+    3e-2 x max(1, rms); the measured unscaled value is returned and printed by the callers."""
+    worst = (0.0, 0.0, 1.0)
     for r in range(len(frames)):
         for n in range(len(frames[r])):
             ref = O.action_chunk(m, w, frames[r][n], dtype)
             rel = float(np.linalg.norm(got[r][n] - ref) / np.linalg.norm(ref))
             mx = float(np.max(np.abs(got[r][n] - ref)))
-            worst = (max(worst[0], rel), max(worst[1], mx))
-            # DDIM with untrained weights multiplies the sample by ~1/sqrt(alpha_bar_90) = 7, so for that solver the
-            # absolute bound is taken relative to the chunk's rms (it then is the same relative requirement)
-            scale = max(1.0, float(np.sqrt(np.mean(ref * ref)))) if m.solver == "ddim" else 1.0
-            assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL * scale, (m.name, r, n, rel, mx)
+            rms = float(np.sqrt(np.mean(ref * ref)))
+            if mx >= worst[1]:
+                worst = (max(worst[0], rel), mx, rms)
+            scale = max(1.0, rms) if m.solver == "ddim" else 1.0
+            assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL * scale, (m.name, r, n, rel, mx, rms)
     return worst
 
 
@@ -67,7 +75,8 @@ def test_parity_serial_vs_oracle(key):
     w = make_weights(m, seed=0)
     frames = _frames(m)
     got, _ = _run(m, w, frames, "serial")
-    _check_vs_oracle(m, w, frames, got)
+    worst = _check_vs_oracle(m, w, frames, got)
+    print(f"{key}: worst rel-L2 {worst[0]:.2e}, max-abs {worst[1]:.3e} at chunk rms {worst[2]:.2f}")
 
 
 @pytest.mark.parametrize("key", list(SMALL))
@@ -77,7 +86,7 @@ def test_modes_bit_identical_and_trace_valid(key):
     frames = _frames(m)
     ref, _ = _run(m, w, frames, "serial")
     for mode in ("cosched", "two_stream", "multi_stream"):
-        cap = 1 << 20 if mode == "cosched" else 0
+        cap = 1 << 21 if mode == "cosched" else 0
         got, extra = _run(m, w, frames, mode, trace_capacity=cap)
         for r in range(len(frames)):
             for n in range(len(frames[r])):
@@ -87,33 +96,9 @@ def test_modes_bit_identical_and_trace_valid(key):
 
 
 def _check_trace(trace, total, program, n_streams, n_frames):
-    """Every tile of every (stream, frame) ran exactly once and no tile started before all tiles of
-    each predecessor node had ended."""
-    assert total == len(trace), "trace ring overflowed"
-    tiles_per_frame = sum(n["n_tiles"] for n in program)
-    assert len(trace) == tiles_per_frame * n_streams * n_frames
-    depth = 2
-    by_frame = {}
-    for rec in trace:
-        key = (int(rec["inst"]) // depth, int(rec["frame"]))
-        by_frame.setdefault(key, []).append(rec)
-    assert len(by_frame) == n_streams * n_frames
-    for key, recs in by_frame.items():
-        start = {}
-        end = {}
-        seen = set()
-        for rec in recs:
-            t = (int(rec["node"]), int(rec["tile"]))
-            assert t not in seen, ("tile ran twice", key, t)
-            seen.add(t)
-            nd = t[0]
-            start[nd] = min(start.get(nd, 1 << 62), int(rec["t_start"]))
-            end[nd] = max(end.get(nd, 0), int(rec["t_end"]))
-            assert int(rec["inst"]) % depth == key[1] % depth
-        for i, n in enumerate(program):
-            assert sum(1 for t in seen if t[0] == i) == n["n_tiles"], ("missing tiles", key, n["name"])
-            for s in n["succ"]:
-                assert end[i] <= start[s], ("dependency violated", key, n["name"], program[s]["name"])
+    """Exactly once, DAG edges, admission before the first tile, ring-slot reuse after the emit (tests/trace_check.py)."""
+    from trace_check import check_trace
+    check_trace(trace, total, program, n_streams, n_frames)
 
 
 def test_dependency_rule_on_gpu():
@@ -265,4 +250,5 @@ def test_non_unit_norm_gains(key):
             w.override(name, round_to_bf16(rng.uniform(0.5, 1.5, size=w.shapes[name]).astype(np.float32)))
     frames = [[frame_inputs(m, r, n, seed=0) for n in range(2)] for r in range(2)]
     got, _ = _run(m, w, frames, "cosched")
-    _check_vs_oracle(m, w, frames, got)
+    worst = _check_vs_oracle(m, w, frames, got)
+    print(f"{key}: worst rel-L2 {worst[0]:.2e}, max-abs {worst[1]:.3e} at chunk rms {worst[2]:.2f}")

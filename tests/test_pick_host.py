@@ -22,12 +22,13 @@ def pick_lib(tmp_path_factory):
                    check=True)
     lib = C.CDLL(str(out))
     lib.pick_host.argtypes = [C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_uint, C.c_uint, C.POINTER(C.c_int),
-                              C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)]
+                              C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int),
+                              C.POINTER(C.c_int)]
     lib.pick_host.restype = C.c_int
     return lib
 
 
-def _call(lib, taus, group, pending, feasible, cta, u, rr, policy, u_max):
+def _call(lib, taus, group, pending, feasible, cta, u, rr, policy, u_max, grid=None, res=None):
     n = len(taus)
     tau = (C.c_int * (3 * n))(*[x for t in taus for x in t])
     grp = (C.c_int * n)(*group)
@@ -36,7 +37,9 @@ def _call(lib, taus, group, pending, feasible, cta, u, rr, policy, u_max):
     pm = sum(1 << k for k in range(n) if pending[k])
     fm = sum(1 << k for k in range(n) if feasible[k])
     phase = C.c_int(0)
-    k = lib.pick_host(n, tau, grp, pm, fm, cc, uu, rr, policy, u_max, C.byref(phase))
+    gg = (C.c_int * n)(*grid) if grid is not None else None
+    rs = (C.c_int * n)(*res) if res is not None else None
+    k = lib.pick_host(n, tau, grp, pm, fm, cc, uu, rr, policy, u_max, C.byref(phase), gg, rs)
     return k, phase.value, list(cc), list(uu)
 
 
@@ -89,3 +92,32 @@ def test_other_policies(pick_lib):
     feas = [True, True, False, True]
     assert _call(pick_lib, taus, group, pending, feas, [0] * 4, [0] * 3, 2, 1, 45)[0] == 1     # class order
     assert _call(pick_lib, taus, group, pending, feas, [0] * 4, [0] * 3, 2, 2, 45)[0] == 3     # round robin from 2: 2 is infeasible
+
+
+def test_score_variants_match_the_oracle(pick_lib):
+    """-G (policy 3) and -R (policy 4): exact agreement with the oracle's rational comparison, ties included."""
+    rnd = random.Random(21)
+    for _ in range(600):
+        n = rnd.randint(1, 8)
+        taus = [tuple(rnd.randint(0, 15) for _ in range(3)) for _ in range(n)]
+        st = SMState(n)
+        st.cta_count = [rnd.randint(0, 3) for _ in range(n)]
+        st.u = [sum(st.cta_count[k] * taus[k][x] for k in range(n)) for x in range(3)]
+        pending = [rnd.random() < 0.8 for _ in range(n)]
+        feas = [rnd.random() < 0.8 for _ in range(n)]
+        rr = rnd.randint(0, n - 1)
+        u_max = rnd.choice([255, 45])
+        grid = [rnd.choice([1, 2, 5, 30, 444, 100000]) for _ in range(n)]
+        res = [rnd.choice([1, 12, 16, 18, 36]) for _ in range(n)]
+        for policy, variant in ((3, "G"), (4, "R")):
+            k, ph, cc, uu = _call(pick_lib, taus, list(range(n)), pending, feas, st.cta_count, st.u, rr, policy, u_max, grid, res)
+            so = st.copy()
+            ko, pho = admission_decision(so, taus, pending, feas, rr_start=rr, u_max=u_max, variant=variant, grid=grid, regs=res)
+            assert k == (-1 if ko is None else ko) and ph == pho, (variant, taus, st.cta_count, grid, res)
+            assert cc == so.cta_count
+    # the hand-derived cases of the oracle's pins, through the device header
+    taus = [(15, 2, 3), (0, 4, 9)]
+    assert _call(pick_lib, taus, [0, 1], [1, 1], [1, 1], [1, 1], [15, 6, 12], 0, 3, 255, [2, 30], [1, 1])[:2] == (1, 2)
+    assert _call(pick_lib, taus, [0, 1], [1, 1], [1, 1], [1, 1], [15, 6, 12], 0, 3, 255, [8, 8], [1, 1])[:2] == (0, 2)
+    assert _call(pick_lib, taus, [0, 1], [1, 1], [1, 1], [1, 1], [15, 6, 12], 0, 4, 255, [1, 1], [64, 32])[:2] == (1, 2)
+    assert _call(pick_lib, taus, [0, 1], [1, 1], [1, 1], [1, 1], [15, 6, 12], 0, 4, 255, [1, 1], [48, 48])[:2] == (0, 2)
