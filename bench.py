@@ -36,6 +36,7 @@ if ROOT not in sys.path:
 from vla_synth.configs import get_config  # noqa: E402
 from vla_synth.gen import make_weights, frame_inputs  # noqa: E402
 
+HEAD_PASSES = 1          # action-head passes per VLM pass (--head-passes): asynchronous inference
 METRIC = "action_chunks_per_sec"
 UNIT = "chunks/s"
 # DRAM bytes per action chunk of the persistent kernel, from the ncu capture summarised in
@@ -127,16 +128,17 @@ def traced_pass(m, weights, R, frames, policy, rank):
     """One short co-scheduled pass with the device trace on; returns trace_stats.summary of it."""
     import torch
     from paper_2609_22335_b200 import Engine, trace_stats
-    probe = Engine(m, mode="cosched", n_streams=1, policy=policy, device=f"cuda:{torch.cuda.current_device()}")
+    probe = Engine(m, mode="cosched", n_streams=1, policy=policy, head_passes=HEAD_PASSES,
+                   device=f"cuda:{torch.cuda.current_device()}")
     tiles_per_frame = sum(n["n_tiles"] for n in probe.program_info())
     probe.close()
     cap = (tiles_per_frame + 1) * R * frames + 1024
-    eng = Engine(m, mode="cosched", n_streams=R, policy=policy, trace_capacity=cap,
+    eng = Engine(m, mode="cosched", n_streams=R, policy=policy, trace_capacity=cap, head_passes=HEAD_PASSES,
                  device=f"cuda:{torch.cuda.current_device()}")
     try:
         eng.load_weights(weights)
         pool = min(frames, 2)
-        host = [[frame_inputs(m, gid, n, seed=0) for n in range(pool)] for gid in rank_stream_ids(R, rank)]
+        host = [[frame_inputs(m, gid, n, seed=0, passes=HEAD_PASSES) for n in range(pool)] for gid in rank_stream_ids(R, rank)]
         dev = [[{k: (None if v is None else torch.from_numpy(np.ascontiguousarray(v)).to(eng.device)) for k, v in fr.items()}
                 for fr in st] for st in host]
         torch.cuda.synchronize()
@@ -166,11 +168,12 @@ def run_mode(m, weights, mode, R, F, steps, warmup, e2e_steps, policy, rank, sam
     """Times `steps` passes in one run mode; returns dict with timings."""
     import torch
     from paper_2609_22335_b200 import Engine
-    eng = Engine(m, mode=mode, n_streams=R, policy=policy, device=f"cuda:{torch.cuda.current_device()}")
+    eng = Engine(m, mode=mode, n_streams=R, policy=policy, head_passes=HEAD_PASSES,
+                 device=f"cuda:{torch.cuda.current_device()}")
     eng.load_weights(weights)
     # a small pool of distinct frames per stream, cycled (inputs > L2 in total for the large workloads)
     pool = min(F, 4)
-    host = [[frame_inputs(m, gid, n, seed=0) for n in range(pool)] for gid in rank_stream_ids(R, rank)]
+    host = [[frame_inputs(m, gid, n, seed=0, passes=HEAD_PASSES) for n in range(pool)] for gid in rank_stream_ids(R, rank)]
     dev = [[{k: (None if v is None else torch.from_numpy(np.ascontiguousarray(v)).to(eng.device)) for k, v in fr.items()}
             for fr in s] for s in host]
     pinned = [[{k: (None if v is None else torch.from_numpy(np.ascontiguousarray(v)).pin_memory()) for k, v in fr.items()}
@@ -287,6 +290,8 @@ def main():
     ap.add_argument("--compare", action="store_true", help="time every other mode (serial too) with the full step count")
     ap.add_argument("--no-modes", action="store_true", help="skip the two-stream / multi-stream timings")
     ap.add_argument("--no-trace", action="store_true", help="skip the traced pass")
+    ap.add_argument("--head-passes", type=int, default=1,
+                    help="asynchronous inference: action-head passes (chunks) per VLM pass")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -294,16 +299,23 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    global HEAD_PASSES
+    HEAD_PASSES = max(1, args.head_passes)
     m = get_config(args.config)
     R = args.streams or m.n_streams
     F = args.frames or m.n_frames
     workload = f"{m.name}: {R} request streams x {F} frames, VLM(n+1) overlapping action head(n)"
+    if HEAD_PASSES > 1:
+        workload += f", {HEAD_PASSES} action-head passes per VLM pass"
     config = {"workload": workload, "mode": args.mode, "policy": args.policy, "ring_depth": 2,
               "l2": "distinct per-stream inputs and weights larger than L2 for cfg2-cfg5; no flush needed" if m.name != "cfg1_tiny"
                     else "working set fits L2 (latency-bound workload)"}
 
     from paper_2609_22335_b200.workload_math import chunk_work
     work = chunk_work(m)
+    if HEAD_PASSES > 1:      # per chunk: one head pass plus its share of the VLM pass
+        work = dict(work, flops=work["vlm_flops"] / HEAD_PASSES + work["head_flops"],
+                    weight_bytes=2 * (work["vlm_params"] / HEAD_PASSES + m.n_steps * work["head_params"]))
 
     if args.impl == "reference":
         if rank != 0:
@@ -334,12 +346,13 @@ def main():
     weights = make_weights(m, seed=0)
     sampler = ClockSampler(local) if rank == 0 else None
     res = run_mode(m, weights, args.mode, R, F, args.steps, args.warmup, 0 if args.no_e2e else 1, args.policy, rank, sampler)
-    agg = aggregate_over_ranks(res["device_s"] / args.steps, res.get("e2e_s"), R * F, world, device="cuda")
+    CH = R * F * HEAD_PASSES          # chunks per step and rank
+    agg = aggregate_over_ranks(res["device_s"] / args.steps, res.get("e2e_s"), CH, world, device="cuda")
     step_s, e2e_s, chunks, value = agg["step_s"], agg["e2e_s"], agg["chunks"], agg["value"]
     peaks = measured_peaks()
-    flops_step = work["flops"] * R * F
+    flops_step = work["flops"] * CH
     t_tensor = flops_step / (peaks["tflops_sustained"] * 1e12)
-    t_hbm = work["weight_bytes"] * F / (peaks["hbm_gbs"] * 1e9)      # every weight once per pass, shared by the streams
+    t_hbm = work["weight_bytes"] * F * HEAD_PASSES / (peaks["hbm_gbs"] * 1e9)      # every weight once per pass, shared by the streams
     bound = "tensor" if t_tensor >= t_hbm else "hbm"
     launches_per_step = max(res["launches"] / args.steps, 1)
     if bound == "tensor":
@@ -347,14 +360,14 @@ def main():
         roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops_sustained"], "unit": "TFLOP/s",
                 "frac": achieved / peaks["tflops_sustained"]}
     else:
-        achieved = work["weight_bytes"] * F / (res["device_s"] / args.steps) / 1e9
+        achieved = work["weight_bytes"] * F * HEAD_PASSES / (res["device_s"] / args.steps) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"]}
     per_chunk = MEASURED_DRAM_BYTES_PER_CHUNK.get(m.name)
-    roof.update({"traffic": (per_chunk * R * F) if per_chunk else None,
+    roof.update({"traffic": (per_chunk * CH) if (per_chunk and HEAD_PASSES == 1) else None,
                  "traffic_note": "ncu dram bytes per chunk on a 2x2 case x chunks per step (upper bound)" if per_chunk else None,
                  "peak_source": peaks["source"] + (" (sustained bf16)" if bound == "tensor" else ""),
                  "kernel": "vla_cosched_kernel (whole step)" if args.mode == "cosched" else "all node kernels of the step",
-                 "launches_per_step": launches_per_step, "roof_chunks_per_s": R * F / max(t_tensor, t_hbm)})
+                 "launches_per_step": launches_per_step, "roof_chunks_per_s": CH / max(t_tensor, t_hbm)})
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
@@ -377,7 +390,7 @@ def main():
             if mode == args.mode:
                 continue
             r2 = run_mode(m, weights, mode, R, F, k_steps, k_warm, 0, args.policy, rank, ClockSampler(local))
-            cmp_[mode] = {"value": R * F / (r2["device_s"] / k_steps), "ms_per_step": r2["device_s"] / k_steps * 1e3,
+            cmp_[mode] = {"value": CH / (r2["device_s"] / k_steps), "ms_per_step": r2["device_s"] / k_steps * 1e3,
                           "steps": k_steps, "warmup": k_warm, "gpu_launches": int(r2["launches"]), "clocks": r2["clocks"]}
         out["modes"] = cmp_
         if "two_stream" in cmp_:

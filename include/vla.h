@@ -99,6 +99,11 @@ typedef struct {
   int32_t u_max;            /* saturation value of the per-SM utilisation counters in the pick's Phase-2 score
                              * (Section 3.3); 0 = default: 15 x worker groups per SM (the hardware proposal's
                              * 8-bit registers would be 255) */
+  int32_t head_passes;      /* asynchronous inference (Section 2.1, decoupled update rates of the two phases): the action
+                             * head runs this many times per VLM pass, every pass on the same VLM output with its own
+                             * robot state and noise sample; 0 or 1 = one pass per frame.  With P passes a frame's
+                             * state is [P, state_dim], its noise [P, horizon, act_dim] and its chunk [P, horizon, act_dim] */
+  int32_t reserved_;
 } vla_runtime_opts;
 
 typedef struct {
@@ -152,7 +157,8 @@ int vla_load_weights(vla_ctx* ctx, const vla_tensor* tensors, size_t n, int32_t 
  * an image of 64 KiB or more in page-locked (pinned) memory is read by an asynchronous copy,
  * so that buffer must stay valid and unmodified until this frame's chunk has been polled:
  * image fp32 [n_cam,3,img,img]; text_ids int32 [n_text]; state fp32 [state_dim] or NULL
- * when the model has none; noise fp32 [horizon,act_dim].  Non-blocking with respect to
+ * when the model has none; noise fp32 [horizon,act_dim] (with head_passes = P > 1: state [P,state_dim], noise
+ * [P,horizon,act_dim]).  Non-blocking with respect to
  * the GPU.  Ring full -> VLA_ERR_BUSY.  frame_id (optional) gets the per-stream frame number. */
 int vla_submit_frame(vla_ctx* ctx, int32_t stream, const float* image, const int32_t* text_ids,
                      const float* state, const float* noise, uint64_t* frame_id);
@@ -165,7 +171,8 @@ int vla_submit_frame_device(vla_ctx* ctx, int32_t stream, const float* image, co
                             const float* state, const float* noise, uint64_t* frame_id);
 
 /* Fetches the next finished action chunk of `stream`, in frame order (Section 2.1: the
- * head of frame N consumed frame N's VLM output).  chunk: HOST fp32 [horizon,act_dim].
+ * head of frame N consumed frame N's VLM output).  chunk: HOST fp32 [horizon,act_dim]
+ * ([head_passes,horizon,act_dim] with several head passes per frame: all of a frame's chunks arrive together).
  * Non-blocking; nothing ready -> VLA_ERR_NOT_READY. */
 int vla_poll_actions(vla_ctx* ctx, int32_t stream, float* chunk, uint64_t* frame_id);
 

@@ -372,6 +372,18 @@ def action_chunk(m, w, frame, dtype=np.float32):
     return action_head(m, w, vlm, frame["state"], frame["noise"], dtype)
 
 
+def action_chunks_async(m, w, frame, dtype=np.float32):
+    """Asynchronous inference (paper Section 2.1, decoupled update rates): one VLM pass, then the action head once per
+    (state, noise) pair of the frame, every pass on that same VLM output.  frame["state"] [P, state_dim] or None,
+    frame["noise"] [P, H, A]; returns [P, H, A]."""
+    vlm = vlm_forward(m, w, frame["image"], frame["text"], dtype)
+    out = []
+    for p in range(frame["noise"].shape[0]):
+        state = None if frame["state"] is None else frame["state"][p]
+        out.append(action_head(m, w, vlm, state, frame["noise"][p], dtype))
+    return np.stack(out)
+
+
 def run_streams(m, w, frames, dtype=np.float32):
     """frames[r][n] -> chunks[r][n]; every (stream, frame) is computed from its own inputs alone."""
     return [[action_chunk(m, w, f, dtype) for f in stream] for stream in frames]

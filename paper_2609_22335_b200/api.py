@@ -43,7 +43,7 @@ class vla_runtime_opts(C.Structure):
     _fields_ = [("arena", C.c_void_p), ("arena_bytes", C.c_size_t), ("stream_a", C.c_void_p), ("stream_b", C.c_void_p),
                 ("mode", C.c_int32), ("n_streams", C.c_int32), ("ring_depth", C.c_int32), ("policy", C.c_int32),
                 ("wait_limit_ns", C.c_uint64), ("trace_capacity", C.c_uint32), ("workers_per_sm", C.c_int32),
-                ("u_max", C.c_int32)]
+                ("u_max", C.c_int32), ("head_passes", C.c_int32), ("reserved_", C.c_int32)]
 
 
 class vla_tensor(C.Structure):
@@ -147,7 +147,7 @@ class Engine:
     """One library context plus the torch-owned arena and streams it runs on."""
 
     def __init__(self, model, mode="cosched", n_streams=None, ring_depth=2, policy=0, trace_capacity=0,
-                 wait_limit_ns=0, workers_per_sm=0, u_max=0, device="cuda:0"):
+                 wait_limit_ns=0, workers_per_sm=0, u_max=0, head_passes=1, device="cuda:0"):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU fallback)")
@@ -169,6 +169,7 @@ class Engine:
         self.opts.trace_capacity = trace_capacity
         self.opts.workers_per_sm = workers_per_sm
         self.opts.u_max = u_max
+        self.opts.head_passes = head_passes
         self.arena_bytes = vla_required_arena_bytes(self.desc, self.opts)
         self.arena = torch.empty(self.arena_bytes + 256, dtype=torch.uint8, device=self.device)
         base = self.arena.data_ptr()
@@ -186,7 +187,8 @@ class Engine:
                 self.lib.vla_destroy(self.ctx)
                 self.ctx = C.c_void_p(None)
             raise VlaError(rc, msg)
-        self.chunk_shape = (model.horizon, model.act_dim)
+        self.head_passes = max(1, int(head_passes))
+        self.chunk_shape = (model.horizon, model.act_dim) if self.head_passes == 1 else (self.head_passes, model.horizon, model.act_dim)
 
     # ---- thin wrappers -------------------------------------------------------------
     def last_error(self) -> str:

@@ -40,6 +40,7 @@ class Builder {
   uint64_t slot_cursor = 0, const_cursor = 0, weight_cursor = 0;
   int phase = PHASE_VLM, step = -1;
   bool init_mode = false;                 // nodes go to the constant-precomputation program
+  std::string name_suffix;                // appended to node names (head passes after the first)
 
   Builder(Program& prog) : p(prog), m(prog.desc) {}
 
@@ -193,7 +194,7 @@ class Builder {
       return (int)p.init_program.size() - 1;
     }
     p.nodes.push_back(n);
-    p.node_names.push_back(name);
+    p.node_names.push_back(name + name_suffix);
     p.node_flops.push_back(0.0);
     p.node_wbytes.push_back(0.0);
     preds.emplace_back();
@@ -484,6 +485,9 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   p.n_streams = o.n_streams;
   p.ring_depth = o.ring_depth;
   p.n_inst = o.n_streams * o.ring_depth;
+  p.head_passes = o.head_passes > 1 ? o.head_passes : 1;
+  if (p.head_passes > 64) { set_err(p, "head_passes must be at most 64"); return false; }
+  const int P = p.head_passes;
   if (p.n_inst >= 4096) { set_err(p, "too many frame slots"); return false; }
 
   Builder b(p);
@@ -658,11 +662,11 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   // inputs
   int in_img = b.buf("in.image", d.n_cam, (int64_t)3 * d.img * d.img, 4);
   int in_txt = b.buf("in.text", 1, pad_to(d.n_text, 4), 4);
-  int in_state = has_state ? b.buf("in.state", 1, d.state_dim, 4) : -1;
-  int in_noise = b.buf("in.noise", d.horizon, d.act_dim, 4);
+  int in_state = has_state ? b.buf("in.state", P, d.state_dim, 4) : -1;
+  int in_noise = b.buf("in.noise", (int64_t)P * d.horizon, d.act_dim, 4);
   p.in_image = p.bufs[in_img].offset; p.image_bytes = p.bufs[in_img].bytes;
   p.in_text = p.bufs[in_txt].offset; p.text_bytes = (uint64_t)d.n_text * 4;
-  if (has_state) { p.in_state = p.bufs[in_state].offset; p.state_bytes = (uint64_t)d.state_dim * 4; }
+  if (has_state) { p.in_state = p.bufs[in_state].offset; p.state_bytes = (uint64_t)P * d.state_dim * 4; }
   p.in_noise = p.bufs[in_noise].offset; p.noise_bytes = p.bufs[in_noise].bytes;
 
   // LLM
@@ -816,8 +820,14 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   int tok0 = first ? b.buf("act.tok0", 1, da, 4) : -1;
   int state_bf = has_state ? b.buf("act.state_bf", 1, P64(d.state_dim), 2) : -1;
 
+  // Asynchronous inference: the head runs P times on the same VLM output, pass by pass on the same buffers (the
+  // buffer accesses order the passes), every pass with its own robot state and noise sample and its own chunk.
+  for (int pass = 0; pass < P; ++pass) {
+  if (pass > 0) { std::snprintf(nm, sizeof nm, ".p%d", pass); b.name_suffix = nm; }
+  b.step = -1;
   if (has_state) {
-    b.addrows("act.state_cvt", View(), Builder::in_ref(2), d.state_dim, 1, d.state_dim, 0, 0, 0, View(), b.all(state_bf));
+    b.addrows("act.state_cvt", View(), Builder::in_ref(2, (uint64_t)pass * d.state_dim * 4), d.state_dim, 1, d.state_dim, 0, 0, 0,
+              View(), b.all(state_bf));
     Builder::GemmOpt g;
     if (head_pos) { g.tab = b.wref(w_apos, 0); g.ldtab = da; }
     g.out32 = b.all(tok0);
@@ -828,7 +838,8 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     g.out32 = b.all(tok0);
     b.gemm("act.cond_tok", b.rows(hidden, S - 1, 1), w_acond, da, g);
   }
-  b.addrows("act.x_init", View(), Builder::in_ref(3), d.act_dim, d.horizon, d.act_dim, 0, 0, 0, b.all(xs), b.all(xbf));
+  b.addrows("act.x_init", View(), Builder::in_ref(3, (uint64_t)pass * d.horizon * d.act_dim * 4), d.act_dim, d.horizon, d.act_dim,
+            0, 0, 0, b.all(xs), b.all(xbf));
 
   for (int k = 0; k < ns; ++k) {
     b.step = k;
@@ -907,13 +918,16 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   {
     NodeDesc n;
     std::memset(&n, 0, sizeof n);
-    n.op = OP_EMIT;
+    n.op = pass == P - 1 ? OP_EMIT : OP_EMIT_PART;        // the last pass's emit publishes the frame
     n.u.emit.x = b.ref(b.all(xs));
     n.u.emit.H = d.horizon; n.u.emit.A = d.act_dim; n.u.emit.ldx = d.act_dim;
+    n.u.emit.chunk_off = pass * d.horizon * d.act_dim;
     n.n_tiles = 1;
     int id = b.add(n, "act.emit", KIND_ELEM);
     b.read(id, b.all(xs));
   }
+  }   // head passes
+  b.name_suffix.clear();
   if (!p.error.empty()) return false;
 
   // ================================================================== successors, roots

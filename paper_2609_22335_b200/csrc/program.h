@@ -48,6 +48,7 @@ struct TmapSpec {           // a 2-D bf16 row-major tensor to describe to the TM
 struct Program {
   vla_model_desc desc;
   int n_streams = 0, ring_depth = 0, n_inst = 0;
+  int head_passes = 1;                  // action-head passes per VLM pass
 
   std::vector<NodeDesc> nodes;
   std::vector<std::string> node_names;

@@ -229,15 +229,16 @@ __device__ void tile_timeemb(const TileCtx& c, const TimeEmbArgs& a, int) {
 }
 
 // Copies the chunk to the host-visible ring, then publishes the frame id (system-scope fence between).
-__device__ void tile_emit(const TileCtx& c, const EmitArgs& a, float* chunk_host, DoneRec* done, uint64_t frame) {
+__device__ void tile_emit(const TileCtx& c, const EmitArgs& a, float* chunk_host, DoneRec* done, uint64_t frame, bool last) {
   const float* x = resolve<const float>(c, a.x);
+  chunk_host += a.chunk_off;
   for (int e = c.tid; e < a.H * a.A; e += WORKER_THREADS) {
     int r = e / a.A, col = e % a.A;
     chunk_host[e] = ld_act(x + (size_t)r * a.ldx + col);
   }
   __threadfence_system();
   worker_sync(c);
-  if (c.tid == 0) {
+  if (c.tid == 0 && last) {
     done->frame_plus1 = frame + 1;
     __threadfence_system();
   }
@@ -255,7 +256,8 @@ __device__ __forceinline__ void run_tile(const DeviceCtx& ctx, const TileCtx& c,
     case OP_ADDROWS: tile_addrows(c, n.u.addrows, tile); break;
     case OP_TIMEEMB: tile_timeemb(c, n.u.timeemb, tile); break;
     case OP_EMIT:
-      tile_emit(c, n.u.emit, ctx.chunk_host + (size_t)inst * ctx.chunk_elems, ctx.done_host + inst, frame);
+    case OP_EMIT_PART:
+      tile_emit(c, n.u.emit, ctx.chunk_host + (size_t)inst * ctx.chunk_elems, ctx.done_host + inst, frame, n.op == OP_EMIT);
       break;
     default:
       if (c.tid == 0) atomicCAS(c.error, 0u, (unsigned)DEV_ERR_BAD_OP);

@@ -383,7 +383,7 @@ int vla_init(const vla_model_desc* desc, const vla_runtime_opts* opts, vla_ctx**
   std::memset(c->staging, 0, c->staging_bytes * p.n_inst);
   CU(cudaHostAlloc(&c->done_host, sizeof(DoneRec) * p.n_inst, cudaHostAllocMapped));
   std::memset((void*)c->done_host, 0, sizeof(DoneRec) * p.n_inst);
-  const size_t chunk_elems = (size_t)desc->horizon * desc->act_dim;
+  const size_t chunk_elems = (size_t)p.head_passes * desc->horizon * desc->act_dim;
   CU(cudaHostAlloc(&c->chunk_host, sizeof(float) * chunk_elems * p.n_inst, cudaHostAllocMapped));
   CU(cudaHostAlloc(&c->error_host, 64, cudaHostAllocMapped));
   *c->error_host = 0;

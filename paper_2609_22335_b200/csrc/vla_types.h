@@ -15,7 +15,8 @@ enum Op : int32_t {
   OP_ADDROWS = 6,   // out fp32 [M,N] = in fp32 (+ vec) (+ table)
   OP_TIMEEMB = 7,   // sinusoidal timestep embedding rows -> bf16
   OP_EMIT = 8,      // copy the finished chunk to the host-visible ring and publish its frame id
-  OP_COUNT = 9
+  OP_EMIT_PART = 9, // copy the chunk of one head pass to the host-visible ring (more passes of the frame follow)
+  OP_COUNT = 10
 };
 
 enum Kind : int32_t { KIND_GEMM = 0, KIND_GEMM2 = 1, KIND_ATTN = 2, KIND_ELEM = 3 };   // GEMM2: two accumulators (gated MLP)
@@ -134,6 +135,7 @@ struct TimeEmbArgs {
 struct EmitArgs {
   Ref x;               // fp32 [H,ldx]
   int32_t H, A, ldx;
+  int32_t chunk_off;   // first element of this pass's chunk inside the frame's host-visible chunk block
 };
 
 struct NodeDesc {

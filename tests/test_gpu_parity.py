@@ -252,3 +252,35 @@ def test_non_unit_norm_gains(key):
     got, _ = _run(m, w, frames, "cosched")
     worst = _check_vs_oracle(m, w, frames, got)
     print(f"{key}: worst rel-L2 {worst[0]:.2e}, max-abs {worst[1]:.3e} at chunk rms {worst[2]:.2f}")
+
+
+@pytest.mark.parametrize("key", ["cfg1", "cfg2s", "cfg3s"])
+def test_async_head_passes(key):
+    """Asynchronous inference (Section 2.1): three action-head passes per VLM pass, each on the same VLM output with
+    its own state and noise.  Against the oracle; bit-identical across modes; pass p equals the chunk of a one-pass
+    frame carrying pass p's state and noise; the trace respects the DAG (passes of a frame run in order)."""
+    m = SMALL[key]
+    P, R, F = 3, 2, 2
+    w = make_weights(m, seed=0)
+    frames = [[frame_inputs(m, r, n, seed=0, passes=P) for n in range(F)] for r in range(R)]
+    got, extra = _run(m, w, frames, "cosched", head_passes=P, trace_capacity=1 << 21)
+    _check_trace(extra["trace"], extra["trace_total"], extra["program"], R, F)
+    assert sum(1 for n in extra["program"] if n["op"] == 9) == P - 1          # one partial emit per pass but the last
+    for r in range(R):
+        for n in range(F):
+            assert got[r][n].shape == (P, m.horizon, m.act_dim)
+            ref = O.action_chunks_async(m, w, frames[r][n], np.float32)
+            for p in range(P):
+                rel = float(np.linalg.norm(got[r][n][p] - ref[p]) / np.linalg.norm(ref[p]))
+                mx = float(np.max(np.abs(got[r][n][p] - ref[p])))
+                assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL, (key, r, n, p, rel, mx)
+    ser, _ = _run(m, w, frames, "serial", head_passes=P)
+    for r in range(R):
+        for n in range(F):
+            assert np.array_equal(got[r][n], ser[r][n])
+    # pass 2 as a frame of its own through a one-pass engine: same bits
+    single = [[dict(f, state=None if f["state"] is None else f["state"][2], noise=f["noise"][2]) for f in s] for s in frames]
+    one, _ = _run(m, w, single, "cosched")
+    for r in range(R):
+        for n in range(F):
+            assert np.array_equal(got[r][n][2], one[r][n])

@@ -390,3 +390,24 @@ def test_workload_shapes(m, prefix_len, act_tokens, vlm_mparams):
         if m.head == "C":       # the per-frame cross-attention K/V projections run in the VLM phase
             got += sum(2 * m.act_d * m.d for i in range(m.act_layers) if i % 2 == 1) / 1e6
         assert abs(got - vlm_mparams) / vlm_mparams < 0.02
+
+
+# ------------------------------------------------------------------ asynchronous inference (Section 2.1)
+def test_async_passes_are_the_head_on_one_vlm_output():
+    m = TINY["A"]
+    w = make_weights(m, seed=8)
+    fr = frame_inputs(m, 0, 1, seed=8, passes=3)
+    single = frame_inputs(m, 0, 1, seed=8)
+    assert np.array_equal(fr["state"][0], single["state"]) and np.array_equal(fr["noise"][0], single["noise"])
+    assert fr["noise"].shape == (3, m.horizon, m.act_dim) and not np.array_equal(fr["noise"][1], fr["noise"][2])
+    out = O.action_chunks_async(m, w, fr, np.float32)
+    assert out.shape == (3, m.horizon, m.act_dim)
+    # pass p = the plain chunk of a frame with the same image/text and pass p's state and noise
+    for p in range(3):
+        one = dict(single, state=fr["state"][p], noise=fr["noise"][p])
+        assert np.array_equal(out[p], O.action_chunk(m, w, one, np.float32))
+    # passes do not see one another: another state for pass 1 changes pass 1 only
+    fr2 = dict(fr, state=fr["state"].copy())
+    fr2["state"][1] += 1.0
+    out2 = O.action_chunks_async(m, w, fr2, np.float32)
+    assert np.array_equal(out2[0], out[0]) and np.array_equal(out2[2], out[2]) and not np.array_equal(out2[1], out[1])

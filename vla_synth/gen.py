@@ -90,12 +90,25 @@ def make_weights(desc: ModelDesc, seed: int = 0, cache: bool = True) -> Weights:
     return Weights(desc, seed, cache)
 
 
-def frame_inputs(desc: ModelDesc, stream: int, frame: int, seed: int = 0) -> dict:
+def frame_inputs(desc: ModelDesc, stream: int, frame: int, seed: int = 0, passes: int = 1) -> dict:
     """Inputs of one frame of one request stream.
 
     image [n_cam,3,H,W] fp32 (bf16-representable, U[0,1]); text int32 [n_text];
-    state fp32 [state_dim] or None; noise fp32 [horizon, act_dim].
+    state fp32 [state_dim] or None; noise fp32 [horizon, act_dim].  With ``passes`` > 1
+    (several action-head passes per VLM pass) state is [passes, state_dim] and noise
+    [passes, horizon, act_dim]; pass 0 holds the arrays of the single-pass frame.
     """
+    if passes > 1:
+        base = frame_inputs(desc, stream, frame, seed)
+        states, noises = [base["state"]], [base["noise"]]
+        lo = (stream << 24) | (frame << 4)
+        for p in range(1, passes):
+            if desc.state_dim > 0:
+                states.append(_rng(seed, 0x1A + (p << 8), lo | _KIND_STATE).standard_normal(size=(desc.state_dim,), dtype=np.float32))
+            noises.append(_rng(seed, 0x1A + (p << 8), lo | _KIND_NOISE).standard_normal(size=(desc.horizon, desc.act_dim), dtype=np.float32))
+        base["state"] = np.stack(states) if desc.state_dim > 0 else None
+        base["noise"] = np.stack(noises)
+        return base
     lo = (stream << 24) | (frame << 4)
     g = _rng(seed, 0x1A, lo | _KIND_IMAGE)
     image = g.random(size=(desc.n_cam, 3, desc.img, desc.img), dtype=np.float32)
