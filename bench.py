@@ -36,6 +36,7 @@ if ROOT not in sys.path:
 from vla_synth.configs import get_config  # noqa: E402
 from vla_synth.gen import make_weights, frame_inputs  # noqa: E402
 
+CLASS_TAGS = None        # profiled intensity tags (--tags), else the library's hand-assigned ones
 HEAD_PASSES = 1          # action-head passes per VLM pass (--head-passes): asynchronous inference
 METRIC = "action_chunks_per_sec"
 UNIT = "chunks/s"
@@ -171,6 +172,8 @@ def run_mode(m, weights, mode, R, F, steps, warmup, e2e_steps, policy, rank, sam
     eng = Engine(m, mode=mode, n_streams=R, policy=policy, head_passes=HEAD_PASSES,
                  device=f"cuda:{torch.cuda.current_device()}")
     eng.load_weights(weights)
+    if CLASS_TAGS is not None:
+        eng.set_class_tags(CLASS_TAGS)
     # a small pool of distinct frames per stream, cycled (inputs > L2 in total for the large workloads)
     pool = min(F, 4)
     host = [[frame_inputs(m, gid, n, seed=0, passes=HEAD_PASSES) for n in range(pool)] for gid in rank_stream_ids(R, rank)]
@@ -292,6 +295,7 @@ def main():
     ap.add_argument("--no-trace", action="store_true", help="skip the traced pass")
     ap.add_argument("--head-passes", type=int, default=1,
                     help="asynchronous inference: action-head passes (chunks) per VLM pass")
+    ap.add_argument("--tags", default=None, help="JSON file written by `auto_tags derive`: profiled intensity tags instead of the hand-assigned ones")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -299,8 +303,11 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    global HEAD_PASSES
+    global HEAD_PASSES, CLASS_TAGS
     HEAD_PASSES = max(1, args.head_passes)
+    if args.tags:
+        with open(args.tags) as f:
+            CLASS_TAGS = json.load(f)["tags"]
     m = get_config(args.config)
     R = args.streams or m.n_streams
     F = args.frames or m.n_frames
@@ -308,6 +315,7 @@ def main():
     if HEAD_PASSES > 1:
         workload += f", {HEAD_PASSES} action-head passes per VLM pass"
     config = {"workload": workload, "mode": args.mode, "policy": args.policy, "ring_depth": 2,
+              "tags": ("profiled: " + os.path.basename(args.tags)) if args.tags else "hand-assigned",
               "l2": "distinct per-stream inputs and weights larger than L2 for cfg2-cfg5; no flush needed" if m.name != "cfg1_tiny"
                     else "working set fits L2 (latency-bound workload)"}
 

@@ -195,6 +195,13 @@ int vla_debug_fetch(vla_ctx* ctx, int32_t stream, int32_t slot, const char* buff
 /* Counters since init: tiles executed, kernels launched by the library, persistent-kernel launches. */
 int vla_get_counters(vla_ctx* ctx, uint64_t* tiles, uint64_t* kernel_launches, uint64_t* persistent_launches);
 
+/* Intensity tags of the eight tile classes (class = phase * 4 + kind, see vla_trace_rec): taus[8][3] =
+ * (tau_TC, tau_ALU, tau_MEM), each 0..15 (Section 3.2.1, Table "Intensity Descriptor").  vla_init installs
+ * hand-assigned defaults; vla_set_class_tags replaces them, e.g. by tags derived from a profiling pass (Section
+ * 3.2.2).  Call while no frame is in flight; the persistent kernel reads the table when it is next launched.  HOST arrays. */
+int vla_set_class_tags(vla_ctx* ctx, const int32_t* taus /*[8*3]*/);
+int vla_get_class_tags(vla_ctx* ctx, int32_t* taus /*[8*3]*/);
+
 /* Runs the device pick function (the COSCHED policy) once on the GPU for a given per-SM
  * state, so tests can compare it with Algorithm 1.  All arrays HOST, n_cls <= 8.
  * cta_count/u are updated as the admission would; *picked = class or -1; *phase = 1, 2 or 0.

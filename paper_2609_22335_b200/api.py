@@ -25,7 +25,7 @@ _SOLVER = {"euler": 0, "ddim": 1}
 
 EXPORTS = ["vla_required_arena_bytes", "vla_init", "vla_load_weights", "vla_submit_frame", "vla_submit_frame_device",
            "vla_poll_actions", "vla_wait_idle", "vla_get_trace", "vla_reset_trace", "vla_program_info", "vla_debug_fetch",
-           "vla_get_counters", "vla_policy_probe", "vla_policy_probe_ex", "vla_debug_bump_dependency", "vla_last_error",
+           "vla_get_counters", "vla_set_class_tags", "vla_get_class_tags", "vla_policy_probe", "vla_policy_probe_ex", "vla_debug_bump_dependency", "vla_last_error",
            "vla_destroy", "vla_op_status", "vla_debug_op_fault",
            "vla_op_attention_scratch_bytes", "vla_op_attention", "vla_op_linear",
            "vla_op_attention_static_capacity", "vla_op_attention_static"]
@@ -94,6 +94,8 @@ def load_library() -> C.CDLL:
                                      C.c_int32, C.c_int32, P(C.c_int32), P(C.c_int32)]
     lib.vla_policy_probe_ex.argtypes = [C.c_int32, P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32),
                                         C.c_int32, C.c_int32, C.c_int32, P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32)]
+    lib.vla_set_class_tags.argtypes = [C.c_void_p, P(C.c_int32)]
+    lib.vla_get_class_tags.argtypes = [C.c_void_p, P(C.c_int32)]
     lib.vla_debug_bump_dependency.argtypes = [C.c_void_p] + [C.c_int32] * 4
     lib.vla_op_status.argtypes = [C.c_int32, C.c_void_p, C.c_void_p]
     lib.vla_debug_op_fault.argtypes = [C.c_int32, C.c_uint64]
@@ -331,6 +333,18 @@ class Engine:
         a, b, c = C.c_uint64(0), C.c_uint64(0), C.c_uint64(0)
         self._check(self.lib.vla_get_counters(self.ctx, C.byref(a), C.byref(b), C.byref(c)))
         return dict(tiles=a.value, kernel_launches=b.value, persistent_launches=c.value)
+
+    def class_tags(self):
+        """The eight tile classes' (tau_TC, tau_ALU, tau_MEM) tags."""
+        t = (C.c_int32 * 24)()
+        self._check(self.lib.vla_get_class_tags(self.ctx, t))
+        return [[t[3 * k + x] for x in range(3)] for k in range(8)]
+
+    def set_class_tags(self, tags):
+        """tags[8][3]; entries that are None keep their current value."""
+        cur = self.class_tags()
+        flat = [int((tags[k] or cur[k])[x]) for k in range(8) for x in range(3)]
+        self._check(self.lib.vla_set_class_tags(self.ctx, (C.c_int32 * 24)(*flat)))
 
     def bump_dependency(self, stream, slot, node, delta):
         """Test hook: adds ``delta`` to one node's dependency counter (see vla_debug_bump_dependency)."""

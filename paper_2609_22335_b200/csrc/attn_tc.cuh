@@ -31,6 +31,7 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16_n(int n) { return umma_idesc
 
 constexpr int ATTN_BQ = 128;   // queries per tile (MMA M)
 constexpr int ATTN_BN = 64;    // keys per block (MMA N of S, MMA K of P V; one 128-byte swizzle row of P)
+constexpr float ATTN_RESCALE_LOG2 = 8.0f;   // the running row maximum may lag the true one by this much (log2 units)
 
 // Barrier over the worker's threads that also ANDs a predicate, so every thread takes the same exit.
 __device__ __forceinline__ bool worker_all(const TileCtx& c, bool pred) {
@@ -193,9 +194,16 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a_in, int tile)
       for (int j = 0; j < ATTN_BN; ++j)
         if (j < lim) m4[j & 3] = fmaxf(m4[j & 3], __uint_as_float(sr[j]));
     }
-    const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-    const float alpha = (m_run == -INFINITY) ? 0.f : exp2_fast((m_run - mx) * a.scale_log2e);
+    float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
     const float sl2 = a.scale_log2e;
+    // The running maximum only has to keep the exponentials in range, not to be exact: softmax does not depend on
+    // the shift, and l and O are accumulated with the same one.  It follows the true maximum only when that has
+    // moved by more than 8 in the exponent (p then stays below 2^8), so O is rescaled on few blocks instead of
+    // on nearly every one (with 32 rows per warp some row's maximum moves in almost every block).
+    float alpha;
+    if (m_run == -INFINITY) alpha = 0.f;
+    else if ((mx - m_run) * sl2 <= ATTN_RESCALE_LOG2) { mx = m_run; alpha = 1.0f; }
+    else alpha = exp2_fast((m_run - mx) * sl2);
     const float mb = mx * sl2;
     float s4[4] = {0.f, 0.f, 0.f, 0.f};
     char* prow = Ps_gen + (size_t)r_in * 128;

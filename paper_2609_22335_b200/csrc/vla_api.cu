@@ -709,6 +709,25 @@ int vla_policy_probe(int32_t n_cls, const int32_t* taus, const int32_t* pending,
                              picked, phase);
 }
 
+int vla_set_class_tags(vla_ctx* c, const int32_t* taus) {
+  if (!c || !taus) return VLA_ERR_INVALID;
+  for (int i = 0; i < N_CLASSES * 3; ++i)
+    if (taus[i] < 0 || taus[i] > 15) return fail(c, VLA_ERR_INVALID, "intensity tags are 4-bit values (0..15)");
+  if (c->pending_frames != 0) return fail(c, VLA_ERR_STATE, "frames are in flight");
+  CU(cudaDeviceSynchronize());          // an idle persistent kernel leaves within its idle limit
+  for (int k = 0; k < N_CLASSES; ++k)
+    for (int x = 0; x < 3; ++x) c->prog.classes[k].tau[x] = taus[k * 3 + x];
+  CU(cudaMemcpy(at<char>(c, c->prog.off_classes), c->prog.classes, sizeof(ClassInfo) * N_CLASSES, cudaMemcpyHostToDevice));
+  return VLA_OK;
+}
+
+int vla_get_class_tags(vla_ctx* c, int32_t* taus) {
+  if (!c || !taus) return VLA_ERR_INVALID;
+  for (int k = 0; k < N_CLASSES; ++k)
+    for (int x = 0; x < 3; ++x) taus[k * 3 + x] = c->prog.classes[k].tau[x];
+  return VLA_OK;
+}
+
 int vla_debug_bump_dependency(vla_ctx* c, int32_t stream, int32_t slot, int32_t node, int32_t delta) {
   if (!c) return VLA_ERR_INVALID;
   const Program& p = c->prog;

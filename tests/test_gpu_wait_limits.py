@@ -176,3 +176,30 @@ def test_every_pick_policy_gives_the_same_chunks(policy):
     for r in range(m.n_streams):
         for n in range(m.n_frames):
             assert np.array_equal(out[0][r][n], out[policy][r][n])
+
+
+def test_class_tags_round_trip_and_leave_the_chunks_unchanged():
+    """vla_set_class_tags / vla_get_class_tags: tags steer the pick only -- the chunks stay bit-identical."""
+    from paper_2609_22335_b200 import Engine, api
+    m = CFG1
+    w = make_weights(m, seed=0)
+    frames = [[frame_inputs(m, r, n, seed=0) for n in range(2)] for r in range(2)]
+    eng = Engine(m, mode="cosched", n_streams=2)
+    try:
+        eng.load_weights(w)
+        hand = eng.class_tags()
+        assert len(hand) == 8 and all(0 <= t <= 15 for row in hand for t in row)
+        base = eng.run(frames)
+        new = [[(3 * k + x) % 16 for x in range(3)] for k in range(8)]
+        new[5] = None                                    # keep the current tags of class 5
+        eng.set_class_tags(new)
+        got = eng.class_tags()
+        assert got[5] == hand[5] and all(got[k] == new[k] for k in range(8) if k != 5)
+        again = eng.run(frames)
+        for r in range(2):
+            for n in range(2):
+                assert np.array_equal(again[r][n], base[r][n])
+        bad = (api.C.c_int32 * 24)(*([16] * 24))
+        assert eng.lib.vla_set_class_tags(eng.ctx, bad) == api.VLA_ERR_INVALID
+    finally:
+        eng.close()
