@@ -36,13 +36,15 @@ if ROOT not in sys.path:
 from vla_synth.configs import get_config  # noqa: E402
 from vla_synth.gen import make_weights, frame_inputs  # noqa: E402
 
+HOLD_LAUNCH = False      # --hold-launch: the first wave of frames of a pass is admitted by one launch
 CLASS_TAGS = None        # profiled intensity tags (--tags), else the library's hand-assigned ones
 HEAD_PASSES = 1          # action-head passes per VLM pass (--head-passes): asynchronous inference
 METRIC = "action_chunks_per_sec"
 UNIT = "chunks/s"
-# DRAM bytes per action chunk of the persistent kernel, from the ncu capture summarised in
-# profiles/cosched_kernel_cfg2_small_dram.md (small case, scaled by chunks: an upper bound at full size)
-MEASURED_DRAM_BYTES_PER_CHUNK = {"cfg2_smolvla": 2.655e9 + 0.091e9}
+# DRAM bytes per action chunk of the persistent kernel, from the one-launch ncu capture of 32 request streams x 2 frames
+# summarised in profiles/cosched_kernel_cfg2_dram_and_pipes.md (109.08 GB read + 49.88 GB written for 64 chunks; the
+# 8-stream capture gives 2.41 GB per chunk, so traffic grows in proportion to the chunks and is scaled by them)
+MEASURED_DRAM_BYTES_PER_CHUNK = {"cfg2_smolvla": (109.08e9 + 49.88e9) / 64}
 
 
 def measured_peaks():
@@ -103,6 +105,12 @@ def drive(eng, n_streams, n_frames, submit, poll_buf):
     done = [0] * n_streams
     remaining = n_streams * n_frames
     idle_since = None
+    if HOLD_LAUNCH:      # first wave (up to ring depth per stream) handed over as one launch
+        eng.hold_launches(True)
+        for r in range(n_streams):
+            while nxt[r] < n_frames and submit(r, nxt[r]) == 0:
+                nxt[r] += 1
+        eng.hold_launches(False)
     while remaining:
         progressed = False
         for r in range(n_streams):
@@ -296,6 +304,8 @@ def main():
     ap.add_argument("--head-passes", type=int, default=1,
                     help="asynchronous inference: action-head passes (chunks) per VLM pass")
     ap.add_argument("--tags", default=None, help="JSON file written by `auto_tags derive`: profiled intensity tags instead of the hand-assigned ones")
+    ap.add_argument("--hold-launch", action="store_true",
+                    help="hand the first wave of frames of every pass to one launch of the persistent kernel (profiler captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -303,7 +313,8 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    global HEAD_PASSES, CLASS_TAGS
+    global HEAD_PASSES, CLASS_TAGS, HOLD_LAUNCH
+    HOLD_LAUNCH = args.hold_launch and args.mode == "cosched"
     HEAD_PASSES = max(1, args.head_passes)
     if args.tags:
         with open(args.tags) as f:
@@ -372,7 +383,8 @@ def main():
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"]}
     per_chunk = MEASURED_DRAM_BYTES_PER_CHUNK.get(m.name)
     roof.update({"traffic": (per_chunk * CH) if (per_chunk and HEAD_PASSES == 1) else None,
-                 "traffic_note": "ncu dram bytes per chunk on a 2x2 case x chunks per step (upper bound)" if per_chunk else None,
+                 "traffic_note": ("dram__bytes_read+write of one vla_cosched_kernel launch over 32 streams x 2 frames (64 chunks), "
+                                  "scaled by chunks to this step") if per_chunk else None,
                  "peak_source": peaks["source"] + (" (sustained bf16)" if bound == "tensor" else ""),
                  "kernel": "vla_cosched_kernel (whole step)" if args.mode == "cosched" else "all node kernels of the step",
                  "launches_per_step": launches_per_step, "roof_chunks_per_s": CH / max(t_tensor, t_hbm)})

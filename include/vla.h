@@ -176,6 +176,12 @@ int vla_submit_frame_device(vla_ctx* ctx, int32_t stream, const float* image, co
  * Non-blocking; nothing ready -> VLA_ERR_NOT_READY. */
 int vla_poll_actions(vla_ctx* ctx, int32_t stream, float* chunk, uint64_t* frame_id);
 
+/* COSCHED mode: while the hold is on, submitted frames are queued for admission but the persistent kernel is not
+ * launched; switching it off launches the kernel, which then admits everything queued at once (no counterpart in
+ * the paper).  Lets a caller hand over a batch of frames -- up to ring_depth per stream -- as one launch, which is
+ * also what a one-pass profiler capture of a whole multi-stream step needs. */
+int vla_hold_launches(vla_ctx* ctx, int32_t on);
+
 /* Blocks (host) until every submitted frame has produced its chunk or timeout_ms passed. */
 int vla_wait_idle(vla_ctx* ctx, uint32_t timeout_ms);
 

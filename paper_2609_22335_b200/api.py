@@ -24,7 +24,7 @@ _HEAD = {"A": 0, "B": 1, "C": 2, "D": 3}
 _SOLVER = {"euler": 0, "ddim": 1}
 
 EXPORTS = ["vla_required_arena_bytes", "vla_init", "vla_load_weights", "vla_submit_frame", "vla_submit_frame_device",
-           "vla_poll_actions", "vla_wait_idle", "vla_get_trace", "vla_reset_trace", "vla_program_info", "vla_debug_fetch",
+           "vla_poll_actions", "vla_hold_launches", "vla_wait_idle", "vla_get_trace", "vla_reset_trace", "vla_program_info", "vla_debug_fetch",
            "vla_get_counters", "vla_set_class_tags", "vla_get_class_tags", "vla_policy_probe", "vla_policy_probe_ex", "vla_debug_bump_dependency", "vla_last_error",
            "vla_destroy", "vla_op_status", "vla_debug_op_fault",
            "vla_op_attention_scratch_bytes", "vla_op_attention", "vla_op_linear",
@@ -84,6 +84,7 @@ def load_library() -> C.CDLL:
         fn.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, P(C.c_uint64)]
     lib.vla_poll_actions.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, P(C.c_uint64)]
     lib.vla_wait_idle.argtypes = [C.c_void_p, C.c_uint32]
+    lib.vla_hold_launches.argtypes = [C.c_void_p, C.c_int32]
     lib.vla_get_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, P(C.c_size_t)]
     lib.vla_reset_trace.argtypes = [C.c_void_p]
     lib.vla_program_info.argtypes = [C.c_void_p, P(vla_node_info), C.c_size_t, P(C.c_size_t), P(C.c_int32), C.c_size_t,
@@ -260,6 +261,10 @@ class Engine:
             return None
         self._check(rc)
         return out, fid.value
+
+    def hold_launches(self, on):
+        """While on, submitted frames are queued but the persistent kernel is not launched (see vla_hold_launches)."""
+        self._check(self.lib.vla_hold_launches(self.ctx, int(bool(on))))
 
     def wait_idle(self, timeout_ms=60000):
         self._check(self.lib.vla_wait_idle(self.ctx, timeout_ms))

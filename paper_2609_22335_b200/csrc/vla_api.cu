@@ -54,6 +54,7 @@ struct vla_ctx {
   // persistent kernel
   cudaEvent_t ev_kernel = nullptr;
   bool kernel_launched = false;
+  bool hold_launches = false;       // submits queue their frames but do not launch the persistent kernel
   int sm_count = 0, dyn_smem = 0, workers = MAX_WORKERS;
   uint64_t pending_frames = 0;      // submitted, chunk not yet observed
   uint64_t n_kernel_launches = 0, n_persistent_launches = 0, n_tiles_streams = 0;
@@ -194,7 +195,7 @@ __global__ void vla_fold_gain_kernel(unsigned short* w, int64_t rows, int cols, 
 
 // (Re)launch the persistent kernel if it is not running and frames are waiting.
 int ensure_persistent(vla_ctx* c) {
-  if (c->pending_frames == 0) return VLA_OK;
+  if (c->pending_frames == 0 || c->hold_launches) return VLA_OK;
   if (c->kernel_launched) {
     cudaError_t q = cudaEventQuery(c->ev_kernel);
     if (q == cudaErrorNotReady) return VLA_OK;
@@ -557,6 +558,16 @@ int vla_poll_actions(vla_ctx* c, int32_t stream, float* chunk, uint64_t* frame_i
   c->inst[inst].state = 0;
   c->next_poll[stream] = f + 1;
   c->pending_frames--;
+  return VLA_OK;
+}
+
+int vla_hold_launches(vla_ctx* c, int32_t on) {
+  if (!c) return VLA_ERR_INVALID;
+  c->hold_launches = on != 0;
+  if (!c->hold_launches && c->opts.mode == VLA_MODE_COSCHED) {
+    CU(cudaStreamSynchronize(c->scopy));      // the queued admission records are in device memory before the launch
+    return ensure_persistent(c);
+  }
   return VLA_OK;
 }
 
