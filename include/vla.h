@@ -229,6 +229,12 @@ int vla_policy_probe_ex(int32_t n_cls, const int32_t* taus, const int32_t* pendi
  * every later call reports the sticky VLA_ERR_TIMEOUT. */
 int vla_debug_bump_dependency(vla_ctx* ctx, int32_t stream, int32_t slot, int32_t node, int32_t delta);
 
+/* Stand-in for a memory checker (no counterpart in the paper): every per-frame and constant buffer of the arena is
+ * followed by 64 guard bytes that no tile may write.  fill != 0 writes a pattern into all of them (call when idle,
+ * after vla_load_weights); fill == 0 reads them back and reports in *n_bad how many guards were overwritten (the
+ * first one is named in vla_last_error).  An out-of-bounds store of a tile body shows up here. */
+int vla_debug_guards(vla_ctx* ctx, int32_t fill, size_t* n_bad);
+
 /* ---- stand-alone operators: the engine's tile bodies on caller-owned DEVICE tensors ------------------------
  * Both run asynchronously on `stream` (a cudaStream_t; NULL = default stream). */
 

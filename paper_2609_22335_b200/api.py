@@ -25,7 +25,7 @@ _SOLVER = {"euler": 0, "ddim": 1}
 
 EXPORTS = ["vla_required_arena_bytes", "vla_init", "vla_load_weights", "vla_submit_frame", "vla_submit_frame_device",
            "vla_poll_actions", "vla_hold_launches", "vla_wait_idle", "vla_get_trace", "vla_reset_trace", "vla_program_info", "vla_debug_fetch",
-           "vla_get_counters", "vla_set_class_tags", "vla_get_class_tags", "vla_policy_probe", "vla_policy_probe_ex", "vla_debug_bump_dependency", "vla_last_error",
+           "vla_get_counters", "vla_set_class_tags", "vla_get_class_tags", "vla_policy_probe", "vla_policy_probe_ex", "vla_debug_bump_dependency", "vla_debug_guards", "vla_last_error",
            "vla_destroy", "vla_op_status", "vla_debug_op_fault",
            "vla_op_attention_scratch_bytes", "vla_op_attention", "vla_op_linear",
            "vla_op_attention_static_capacity", "vla_op_attention_static"]
@@ -97,6 +97,7 @@ def load_library() -> C.CDLL:
                                         C.c_int32, C.c_int32, C.c_int32, P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32)]
     lib.vla_set_class_tags.argtypes = [C.c_void_p, P(C.c_int32)]
     lib.vla_get_class_tags.argtypes = [C.c_void_p, P(C.c_int32)]
+    lib.vla_debug_guards.argtypes = [C.c_void_p, C.c_int32, P(C.c_size_t)]
     lib.vla_debug_bump_dependency.argtypes = [C.c_void_p] + [C.c_int32] * 4
     lib.vla_op_status.argtypes = [C.c_int32, C.c_void_p, C.c_void_p]
     lib.vla_debug_op_fault.argtypes = [C.c_int32, C.c_uint64]
@@ -350,6 +351,16 @@ class Engine:
         cur = self.class_tags()
         flat = [int((tags[k] or cur[k])[x]) for k in range(8) for x in range(3)]
         self._check(self.lib.vla_set_class_tags(self.ctx, (C.c_int32 * 24)(*flat)))
+
+    def fill_guards(self):
+        """Writes the guard pattern behind every buffer (see vla_debug_guards)."""
+        self._check(self.lib.vla_debug_guards(self.ctx, 1, None))
+
+    def overwritten_guards(self) -> int:
+        """How many guards no longer hold the pattern (0 = no tile wrote outside its buffers)."""
+        n = C.c_size_t(0)
+        self._check(self.lib.vla_debug_guards(self.ctx, 0, C.byref(n)))
+        return n.value
 
     def bump_dependency(self, stream, slot, node, delta):
         """Test hook: adds ``delta`` to one node's dependency counter (see vla_debug_bump_dependency)."""

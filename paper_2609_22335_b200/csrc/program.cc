@@ -52,7 +52,7 @@ class Builder {
     uint64_t& cur = slot ? slot_cursor : const_cursor;
     cur = align_up(cur, 256);
     b.offset = cur;
-    cur += b.bytes;
+    cur += b.bytes + GUARD_BYTES;         // guard words behind the buffer: nothing may ever write them
     p.bufs.push_back(b);
     p.buf_index[name] = (int)p.bufs.size() - 1;
     acc.emplace_back();

@@ -38,6 +38,8 @@ struct BufInfo {
   int elem;                 // 4 fp32, 2 bf16
 };
 
+constexpr uint64_t GUARD_BYTES = 64;   // guard words behind every buffer (see vla_debug_guards)
+
 struct TmapSpec {           // a 2-D bf16 row-major tensor to describe to the TMA unit
   uint64_t offset;          // arena or slot-relative byte offset
   bool slot;

@@ -739,6 +739,32 @@ int vla_get_class_tags(vla_ctx* c, int32_t* taus) {
   return VLA_OK;
 }
 
+int vla_debug_guards(vla_ctx* c, int32_t fill, size_t* n_bad) {
+  if (!c || (!fill && !n_bad)) return VLA_ERR_INVALID;
+  if (c->pending_frames != 0) return fail(c, VLA_ERR_STATE, "frames are in flight");
+  CU(cudaDeviceSynchronize());
+  const Program& p = c->prog;
+  unsigned char pat[GUARD_BYTES], got[GUARD_BYTES];
+  std::memset(pat, 0xC5, sizeof pat);
+  size_t bad = 0;
+  for (const BufInfo& b : p.bufs) {
+    if (b.name.compare(0, 3, "in.") == 0) continue;      // the staged input copy spans the input buffers, guards included
+    const int copies = b.slot ? p.n_inst : 1;
+    for (int i = 0; i < copies; ++i) {
+      char* g = c->arena + (b.slot ? p.off_slots + (uint64_t)i * p.slot_bytes : p.off_consts) + b.offset + b.bytes;
+      if (fill) {
+        CU(cudaMemcpy(g, pat, GUARD_BYTES, cudaMemcpyHostToDevice));
+      } else {
+        CU(cudaMemcpy(got, g, GUARD_BYTES, cudaMemcpyDeviceToHost));
+        if (std::memcmp(got, pat, GUARD_BYTES) != 0 && bad++ == 0)
+          c->err = "guard behind buffer '" + b.name + "' of frame slot " + std::to_string(i) + " was overwritten";
+      }
+    }
+  }
+  if (n_bad) *n_bad = bad;
+  return VLA_OK;
+}
+
 int vla_debug_bump_dependency(vla_ctx* c, int32_t stream, int32_t slot, int32_t node, int32_t delta) {
   if (!c) return VLA_ERR_INVALID;
   const Program& p = c->prog;

@@ -179,12 +179,39 @@ def smaller_side_of_concurrent_pairs(trace, program) -> dict:
             "eleven_plus": float((sm >= 11).mean()), "median": float(np.median(sm))}
 
 
+def gap_stats(trace) -> dict:
+    """Idle time of the worker groups between two consecutive tiles, by the class of the tile that ended the gap.
+
+    For every (sm, worker) the tiles are ordered by start time; gap = start of the next tile - end of this one.
+    Returns per class: gaps, mean / median / 90th percentile in microseconds, and the class's share of all idle time
+    between tiles (idle time before a worker's first and after its last tile is not counted)."""
+    t = tiles_only(trace)
+    if len(t) < 2:
+        return {}
+    key = t["sm"].astype(np.int64) * 256 + t["worker"]
+    order = np.lexsort((t["t_start"], key))
+    k, s, e, c = key[order], t["t_start"][order].astype(np.int64), t["t_end"][order].astype(np.int64), t["cls"][order]
+    same = k[1:] == k[:-1]
+    gap = (s[1:] - e[:-1])[same].astype(np.float64)
+    nxt = c[1:][same]
+    gap = np.maximum(gap, 0.0)
+    tot = gap.sum()
+    out = {"all": {"gaps": int(len(gap)), "mean_us": float(gap.mean() * 1e-3), "median_us": float(np.median(gap) * 1e-3),
+                   "p90_us": float(np.percentile(gap, 90) * 1e-3)}}
+    for ci, name in enumerate(CLASS_NAMES):
+        g = gap[nxt == ci]
+        if len(g):
+            out[name] = {"gaps": int(len(g)), "mean_us": float(g.mean() * 1e-3), "median_us": float(np.median(g) * 1e-3),
+                         "p90_us": float(np.percentile(g, 90) * 1e-3), "share_of_idle": float(g.sum() / tot) if tot > 0 else 0.0}
+    return out
+
+
 def summary(trace, program=None, n_sms: int | None = None, workers_per_sm: int = 3) -> dict:
     """Everything the benchmark line reports from one traced pass."""
     n_workers = (n_sms * workers_per_sm) if n_sms else None
     out = {"tiles": int(len(tiles_only(trace))), "wall_ms": wall_ns(trace) * 1e-6,
            "sm_busy_frac": busy_fraction(trace, n_workers), "class_share_of_busy_time": class_shares(trace),
-           "concurrency": concurrency_fraction(trace, n_sms)}
+           "concurrency": concurrency_fraction(trace, n_sms), "gaps_between_tiles": gap_stats(trace)}
     if program is not None and n_workers:
         out["per_class"] = per_class_rates(trace, program, n_workers)
         out["smaller_side_of_concurrent_node_pairs"] = smaller_side_of_concurrent_pairs(trace, program)

@@ -1,6 +1,7 @@
 """Full-size parity: the five workloads at their stated shapes and request-stream counts, in the
 co-scheduled launch configuration the benchmark times, against the CPU oracle on sampled chunks
-(first stream / last stream, first / second frame), plus bit-identity with the two-stream mode."""
+(first, middle and last stream; first and last frame), bit-identity with a stream mode, and the
+device trace of the full-size SmolVLA-shaped run checked against the tile DAG."""
 import numpy as np
 import pytest
 
@@ -27,7 +28,7 @@ def test_full_size_sampled_parity(m, frames, check_two_stream):
         got = eng.run(fr, timeout_s=900)
     finally:
         eng.close()
-    samples = [(0, 0), (R - 1, frames - 1)] if m is not CFG5 else [(R - 1, frames - 1)]
+    samples = [(0, 0), (R // 2, 0), (R - 1, frames - 1)] if m is not CFG5 else [(R - 1, frames - 1)]
     for (r, n) in samples:
         ref = O.action_chunk(m, w, fr[r][n], np.float32)
         rel = float(np.linalg.norm(got[r][n] - ref) / np.linalg.norm(ref))
@@ -44,8 +45,8 @@ def test_full_size_sampled_parity(m, frames, check_two_stream):
         for n in range(frames):
             assert np.isfinite(got[r][n]).all()
     assert not np.array_equal(got[0][0], got[R - 1][0])
-    if check_two_stream:
-        eng = Engine(m, mode="two_stream", n_streams=R)
+    if check_two_stream or m is CFG3:
+        eng = Engine(m, mode="two_stream" if check_two_stream else "multi_stream", n_streams=R)
         try:
             eng.load_weights(w)
             got2 = eng.run(fr, timeout_s=900)
@@ -54,3 +55,28 @@ def test_full_size_sampled_parity(m, frames, check_two_stream):
         for r in range(R):
             for n in range(frames):
                 assert np.array_equal(got[r][n], got2[r][n]), (m.name, r, n)
+
+
+def test_full_size_trace_respects_the_dag():
+    """32 request streams x 3 frames of the SmolVLA-shaped workload, co-scheduled, with the device trace on: every
+    one of the 2.6 million tiles ran exactly once, after its frame's admission and after all tiles of its
+    predecessors; the third frame of a stream did not start before the first one's chunk was emitted."""
+    from paper_2609_22335_b200 import Engine
+    from trace_check import check_trace
+    m, F = CFG2, 3
+    w = make_weights(m, seed=0)
+    R = m.n_streams
+    probe = Engine(m, mode="cosched", n_streams=1)
+    tiles_per_frame = sum(n["n_tiles"] for n in probe.program_info())
+    probe.close()
+    fr = [[frame_inputs(m, r, n % 2, seed=0) for n in range(F)] for r in range(R)]
+    eng = Engine(m, mode="cosched", n_streams=R, trace_capacity=(tiles_per_frame + 1) * R * F + 1024)
+    try:
+        eng.load_weights(w)
+        eng.run(fr, timeout_s=900)
+        eng.wait_idle()
+        trace, total = eng.trace()
+        stats = check_trace(trace, total, eng.program_info(), R, F)
+    finally:
+        eng.close()
+    assert stats["tiles"] == tiles_per_frame * R * F and stats["admissions"] == R * F

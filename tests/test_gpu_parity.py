@@ -284,3 +284,23 @@ def test_async_head_passes(key):
     for r in range(R):
         for n in range(F):
             assert np.array_equal(got[r][n][2], one[r][n])
+
+
+@pytest.mark.parametrize("key", ["cfg2s", "cfg3s", "cfg4s", "cfg5s"])
+def test_no_tile_writes_outside_its_buffers(key):
+    """Guard words behind every buffer of every frame slot survive a co-scheduled run (ragged tiles, padded heads,
+    transposed V, pixel-shuffle scatter, odd output widths): the stand-in for a memory checker."""
+    from paper_2609_22335_b200 import Engine
+    m = SMALL[key]
+    w = make_weights(m, seed=0)
+    frames = _frames(m)
+    eng = Engine(m, mode="cosched", n_streams=len(frames))
+    try:
+        eng.load_weights(w)
+        eng.fill_guards()
+        assert eng.overwritten_guards() == 0
+        eng.run(frames)
+        eng.wait_idle()
+        assert eng.overwritten_guards() == 0, eng.last_error()
+    finally:
+        eng.close()

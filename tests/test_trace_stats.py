@@ -70,3 +70,13 @@ def test_per_class_rates_and_pairs():
     assert p["pairs"] == 1 and p["one_tile"] == 1.0 and p["median"] == 1.0
     s = TS.summary(tr, program, n_sms=2, workers_per_sm=2)
     assert s["tiles"] == 3 and abs(s["sm_busy_frac"] - 2500 / (4 * 1000)) < 1e-12
+
+
+def test_gap_stats():
+    # worker (0,0): VLM GEMM [0,10), head GEMM [14,20), VLM GEMM [20,30): gaps 4 (before a head tile) and 0 (before a VLM tile)
+    # worker (1,0): head GEMM [0,5), head GEMM [11,12): gap 6
+    tr = _trace([(0, 0, 0, 0, 0, 10), (0, 0, 4, 1, 14, 20), (0, 0, 0, 0, 20, 30), (1, 0, 4, 1, 0, 5), (1, 0, 4, 1, 11, 12)])
+    g = TS.gap_stats(tr)
+    assert g["all"]["gaps"] == 3 and abs(g["all"]["mean_us"] - 10 / 3 * 1e-3) < 1e-12
+    assert g["head_gemm"]["gaps"] == 2 and abs(g["head_gemm"]["mean_us"] - 5e-3) < 1e-12 and g["head_gemm"]["share_of_idle"] == 1.0
+    assert g["vlm_gemm"]["gaps"] == 1 and g["vlm_gemm"]["mean_us"] == 0.0
