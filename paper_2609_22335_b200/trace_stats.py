@@ -195,6 +195,8 @@ def gap_stats(trace) -> dict:
     gap = (s[1:] - e[:-1])[same].astype(np.float64)
     nxt = c[1:][same]
     gap = np.maximum(gap, 0.0)
+    if len(gap) == 0:
+        return {}
     tot = gap.sum()
     out = {"all": {"gaps": int(len(gap)), "mean_us": float(gap.mean() * 1e-3), "median_us": float(np.median(gap) * 1e-3),
                    "p90_us": float(np.percentile(gap, 90) * 1e-3)}}
