@@ -133,14 +133,18 @@ def drive(eng, n_streams, n_frames, submit, poll_buf):
     return n_streams * n_frames
 
 
-def traced_pass(m, weights, R, frames, policy, rank):
-    """One short co-scheduled pass with the device trace on; returns trace_stats.summary of it."""
+def traced_pass(m, weights, R, frames, policy, rank, max_records=8_000_000):
+    """One co-scheduled pass with the device trace on; returns trace_stats.summary of it.
+
+    As many frames per stream as fit `max_records` trace records (at least 2, at most `frames`): the longer the
+    pass, the less its pipeline fill and drain weigh in the statistics."""
     import torch
     from paper_2609_22335_b200 import Engine, trace_stats
     probe = Engine(m, mode="cosched", n_streams=1, policy=policy, head_passes=HEAD_PASSES,
                    device=f"cuda:{torch.cuda.current_device()}")
     tiles_per_frame = sum(n["n_tiles"] for n in probe.program_info())
     probe.close()
+    frames = max(2, min(frames, max_records // ((tiles_per_frame + 1) * R)))
     cap = (tiles_per_frame + 1) * R * frames + 1024
     eng = Engine(m, mode="cosched", n_streams=R, policy=policy, trace_capacity=cap, head_passes=HEAD_PASSES,
                  device=f"cuda:{torch.cuda.current_device()}")
@@ -418,7 +422,7 @@ def main():
         if "multi_stream" in cmp_:
             out["speedup_vs_multi_stream"] = value / cmp_["multi_stream"]["value"]
     if rank == 0 and world == 1 and not args.no_trace and args.mode == "cosched":
-        tr = traced_pass(m, weights, R, min(F, 2 if m.name != "cfg1_tiny" else F), args.policy, rank)
+        tr = traced_pass(m, weights, R, F, args.policy, rank)
         out["trace"] = tr
         out["sm_busy_frac"] = tr["sm_busy_frac"]
         out["concurrency_frac"] = tr["concurrency"]["mean"]

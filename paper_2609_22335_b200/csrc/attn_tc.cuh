@@ -1,6 +1,7 @@
 // Fused attention tile on tcgen05 / tensor memory.
 //
-// One tile = one query head x 128 queries.  Per block of bn keys:
+// One tile = one query head x 128 queries -- or, where few queries meet grouped KV heads (the action head's 9..51
+// tokens), several query heads of one KV head side by side in the 128 rows.  Per block of bn keys:
 //   S = Q K^T          tcgen05.mma, Q and K tiles K-major (head dim contiguous), S in TMEM
 //   online softmax     one thread per query row reads its S row from TMEM (no shuffles),
 //                      writes P as bf16 into 128-byte-swizzled shared memory
@@ -82,12 +83,19 @@ __device__ __forceinline__ KvBlock kv_next(const A& a, KvBlock b, int q_last) {
 __device__ void tile_attention(const TileCtx& c, const AttnArgs& a_in, int tile) {
   // The node's arguments live in global memory; the shared-memory stores and the asm statements of the block loop
   // would make the compiler fetch them again and again, so the ones the loop uses are copied into registers.
-  struct { int32_t k0map, v0map, k1map, v1map, t0, t1, causal, hq, hkv, hs, hd, q_blocks, qmap, tq, ldo; float scale_log2e; Ref out; } a;
+  struct { int32_t k0map, v0map, k1map, v1map, t0, t1, causal, hq, hkv, hs, hd, q_blocks, qmap, tq, ldo, hpt, rph; float scale_log2e; Ref out; } a;
   a.k0map = a_in.k0map; a.v0map = a_in.v0map; a.k1map = a_in.k1map; a.v1map = a_in.v1map; a.t0 = a_in.t0; a.t1 = a_in.t1;
   a.causal = a_in.causal; a.hq = a_in.hq; a.hkv = a_in.hkv; a.hs = a_in.hs; a.hd = a_in.hd; a.q_blocks = a_in.q_blocks;
   a.qmap = a_in.qmap; a.tq = a_in.tq; a.ldo = a_in.ldo; a.scale_log2e = a_in.scale_log2e; a.out = a_in.out;
+  a.hpt = a_in.hpt > 1 ? a_in.hpt : 1; a.rph = a_in.rph;
   const int warp = c.tid >> 5, lane = c.tid & 31;
-  const int head = tile / a.q_blocks, qb = tile % a.q_blocks;
+  // folded: tile -> (KV head g, first query head, heads in this tile); else tile -> (head, query block)
+  const bool folded = a.hpt > 1;
+  const int group = a.hq / a.hkv;
+  const int tiles_per_group = folded ? (group + a.hpt - 1) / a.hpt : 1;
+  const int head = folded ? (tile / tiles_per_group) * group + (tile % tiles_per_group) * a.hpt : tile / a.q_blocks;
+  const int qb = folded ? 0 : tile % a.q_blocks;
+  const int nh = folded ? min(a.hpt, group - (tile % tiles_per_group) * a.hpt) : 1;
   const int g = (head * a.hkv) / a.hq;
   const int q0 = qb * ATTN_BQ;
   const int hs = a.hs;
@@ -131,13 +139,25 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a_in, int tile)
   const bool loads_on = !c.drop_loads;          // (test hook: with the loads off, the waits below run out)
   if (issuer && loads_on) {
     asm volatile("fence.proxy.async;" ::: "memory");
-    mbar_expect_tx(bar_q, (uint32_t)nbox * (ATTN_BQ * 128));
-    for (int b = 0; b < nbox; ++b) tma_load_2d(Qs + (uint32_t)b * (ATTN_BQ * 128), map_ptr(a.qmap), bar_q, head * hs + b * 64, q0);
+    if (!folded) {
+      mbar_expect_tx(bar_q, (uint32_t)nbox * (ATTN_BQ * 128));
+      for (int b = 0; b < nbox; ++b) tma_load_2d(Qs + (uint32_t)b * (ATTN_BQ * 128), map_ptr(a.qmap), bar_q, head * hs + b * 64, q0);
+    } else {
+      // head i of the tile: a box of rph rows (rows past tq are outside the tensor and arrive as zeros) at row i * rph
+      // (a multiple of 8 rows = of one 1024-byte swizzle group); rows past the last head keep whatever the slab held --
+      // every output row depends on its own query row only, and those rows are never stored
+      mbar_expect_tx(bar_q, (uint32_t)(nh * nbox * a.rph * 128));
+      for (int i = 0; i < nh; ++i)
+        for (int b = 0; b < nbox; ++b)
+          tma_load_2d(Qs + (uint32_t)b * (ATTN_BQ * 128) + (uint32_t)(i * a.rph * 128), map_ptr(a.qmap), bar_q, (head + i) * hs + b * 64, 0);
+    }
     if (cur.valid) load_k(cur);
   }
 
-  const int row = q0 + warp * 32 + lane;                // this thread's query
-  const int r_in = warp * 32 + lane;
+  const int r_in = warp * 32 + lane;                    // this thread's row of the tile
+  const int fold_h = folded ? r_in / a.rph : 0;         // which of the tile's heads the row belongs to
+  const int row = folded ? r_in - fold_h * a.rph : q0 + r_in;   // this thread's query
+  const bool row_ok = row < a.tq && fold_h < nh;
   float m_run = -INFINITY, l_run = 0.f;
   int blk = 0;
   bool ok = true;
@@ -266,14 +286,14 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a_in, int tile)
     for (int c0 = 0; c0 < hs; c0 += 16) {
       float o[16];
       tmem_ld16(tmem_o + lane_off + (uint32_t)c0, o);
-      if (row < a.tq) {
+      if (row_ok) {
         uint32_t pk[8];
 #pragma unroll
         for (int j = 0; j < 16; j += 2) {
           __nv_bfloat162 v = __floats2bfloat162_rn(o[j] * inv, o[j + 1] * inv);
           pk[j >> 1] = *reinterpret_cast<uint32_t*>(&v);
         }
-        unsigned short* dst = O + (size_t)row * a.ldo + head * a.hd + c0;
+        unsigned short* dst = O + (size_t)row * a.ldo + (head + fold_h) * a.hd + c0;
         if (c0 + 16 <= a.hd) {
           *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           *reinterpret_cast<uint4*>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);

@@ -153,7 +153,8 @@ __device__ inline bool queue_try_pop(const DeviceCtx& ctx, int cls, QueueEntry& 
 constexpr int MAX_READY = 6;
 constexpr int DISPATCH_THREADS = 64;     // two service warps per SM (claim, retire), after the worker groups
 constexpr long long PRIO_WINDOW_NS = 8000;   // an action-head tile may be claimed for a worker this close to the end of its tile
-constexpr int PREFETCH_MIN_AVAIL = 128;   // tiles are claimed ahead of need only from queues at least this deep
+constexpr int PREFETCH_MIN_TOTAL = 600;   // tiles are claimed ahead of need only while this many VLM tiles are queued in all
+constexpr int PREFETCH_MIN_AVAIL = 8;     // ... and only from queues at least this deep
 constexpr int HELD_DEPTH = 1;            // claimed tiles a worker may have waiting
 constexpr unsigned CLAIM_NAP_NS = 60, CLAIM_NAP_MAX_NS = 240;   // claim warp, while a worker of its SM has nothing to run
 constexpr unsigned CLAIM_SLEEP_NS = 2000;    // claim warp, every worker busy: longest sleep without a ring
@@ -419,7 +420,14 @@ __device__ inline void claim_loop(const DeviceCtx& ctx, SmState* sm, int n_worke
     bool progressed = false;
     long long av = lane < N_CLASSES ? ld_volatile_s64(&ctx.queues[lane].avail) : 0;
     const unsigned pending = __ballot_sync(0xffffffffu, av > 0) & ((1u << N_CLASSES) - 1u);
-    const unsigned deep = __ballot_sync(0xffffffffu, av >= PREFETCH_MIN_AVAIL) & ((1u << N_CLASSES) - 1u);
+    // Tiles are claimed ahead of need only while the VLM backlog as a whole exceeds what the GPU's workers can hold
+    // (a held tile is a tile no idle worker elsewhere can take), and then from every VLM queue that is not nearly empty.
+    long long vlm_total = (lane < N_KINDS && av > 0) ? av : 0;
+    vlm_total += __shfl_xor_sync(0xffffffffu, vlm_total, 1);
+    vlm_total += __shfl_xor_sync(0xffffffffu, vlm_total, 2);
+    vlm_total = __shfl_sync(0xffffffffu, vlm_total, 0);
+    const unsigned deep = __ballot_sync(0xffffffffu, vlm_total >= PREFETCH_MIN_TOTAL && av >= PREFETCH_MIN_AVAIL) &
+                          ((1u << N_CLASSES) - 1u);
     // classes whose tiles free workers elsewhere did not drain within head_wait_ns (by the clock, not by polling
     // rounds: how fast this loop spins must not change what it decides)
     if (av > 0) { if (pending_since == 0) pending_since = gtimer(); } else pending_since = 0;

@@ -179,11 +179,13 @@ inline int op_attention_run(const void* q, const void* k, const void* v, void* o
   a.hq = hq; a.hkv = hkv; a.hd = hd; a.hs = hd; a.causal = causal ? 1 : 0;
   a.bn = 64;
   a.q_blocks = (tq + 127) / 128;
+  a.hpt = attn_fold(tq, hq, hkv, &a.rph);
+  const int n_tiles = a.hpt > 1 ? hkv * (((hq / hkv) + a.hpt - 1) / a.hpt) : hq * a.q_blocks;
   a.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
   a.qmap = 0; a.k0map = 1; a.v0map = 2; a.k1map = 1; a.v1map = 2;
   OpMaps maps;
   memset(&maps, 0, sizeof maps);
-  if (!op_encode(&maps.m[0], q, tq, (int64_t)hq * hd, (int64_t)hq * hd, 128) ||
+  if (!op_encode(&maps.m[0], q, tq, (int64_t)hq * hd, (int64_t)hq * hd, a.hpt > 1 ? a.rph : 128) ||
       !op_encode(&maps.m[1], k, tkv, (int64_t)hkv * hd, (int64_t)hkv * hd, a.bn) ||
       !op_encode(&maps.m[2], vt, (int64_t)hkv * hd, tkv, tpad, hd))
     return VLA_ERR_CUDA;
@@ -192,7 +194,7 @@ inline int op_attention_run(const void* q, const void* k, const void* v, void* o
   while (tmem_cols < a.bn + hd) tmem_cols <<= 1;
   if (cudaFuncSetAttribute(vla_op_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
     return VLA_ERR_CUDA;
-  vla_op_attention_kernel<<<hq * a.q_blocks, WORKER_THREADS, smem, s>>>(a, maps, tmem_cols, err, op_fault());
+  vla_op_attention_kernel<<<n_tiles, WORKER_THREADS, smem, s>>>(a, maps, tmem_cols, err, op_fault());
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 

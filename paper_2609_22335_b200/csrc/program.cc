@@ -355,9 +355,12 @@ class Builder {
     n.smem_bytes = attn_smem_bytes(hs);
     n.tmem_cols = (int)pad_to(a.bn + hs, TMEM_UNIT);
     n.n_tiles = hq * a.q_blocks;
-    // tensor maps: Q rows in 128-row boxes, K rows in bn-row boxes, V^T in hs-row boxes of 64 tokens
+    a.hpt = attn_fold(tq, hq, hkv, &a.rph);
+    if (a.hpt > 1) n.n_tiles = hkv * (((hq / hkv) + a.hpt - 1) / a.hpt);
+    // tensor maps: Q rows in 128-row boxes (rph-row boxes when heads are folded), K rows in bn-row boxes, V^T in
+    // hs-row boxes of 64 tokens
     const int64_t qcols = ld(q) - q.col0;
-    a.qmap = act_map(q, qcols, 128);
+    a.qmap = act_map(q, qcols, a.hpt > 1 ? a.rph : 128);
     auto kview = [&](const QKV& s_) { return rows(s_.qk, 0, s_.T, (int64_t)s_.hq * s_.hs); };
     a.k0map = act_map(kview(kv0), (int64_t)kv0.hkv * kv0.hs, a.bn);
     a.v0map = act_map(all(kv0.vt), kv0.T, hs);

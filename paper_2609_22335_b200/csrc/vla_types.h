@@ -64,6 +64,16 @@ inline int attn_smem_bytes(int hs) {
   return nbox * 128 * 128 + nbox * 64 * 128 + hs * 128 + 128 * 128;
 }
 
+// Query heads that share a KV head (grouped or multi-query attention) and have few queries are folded into the 128
+// rows of one attention tile: the tile streams K and V^T once for all of them.  Returns heads per tile, sets rows per head.
+inline int attn_fold(int tq, int hq, int hkv, int* rph) {
+  const int group = hkv > 0 ? hq / hkv : 1;
+  *rph = (tq + 7) / 8 * 8;
+  if (tq > 64 || group < 2) return 1;
+  const int fit = 128 / *rph;
+  return fit < group ? fit : group;
+}
+
 struct GemmArgs {
   Ref A, W, W2;        // A bf16 [M,lda]; W (and W2 when dual) bf16 [N,Kp]
   Ref X;               // optional fp32 addend [M,ldx], scaled by c_x
@@ -100,6 +110,8 @@ struct AttnArgs {
   int32_t hq, hkv, hd, hs;     // hs = head stride (hd padded to a multiple of 16)
   int32_t causal;
   int32_t bn, q_blocks;        // keys per block; 128-query blocks
+  int32_t hpt, rph;            // query heads folded into one tile (they share a KV head; 1 = none) and the rows each
+                               // takes in the tile (tq rounded up to a multiple of 8); folding needs q_blocks == 1
   float scale_log2e;           // log2(e) / sqrt(hd)
 };
 

@@ -53,7 +53,10 @@ def test_linear_bf16_output_rounding():
 @pytest.mark.parametrize("tq,tkv,hq,hkv,hd,causal", [
     (9, 80, 4, 4, 64, False), (50, 226, 15, 5, 64, False), (1024, 1024, 12, 12, 64, False), (17, 17, 16, 16, 64, False),
     (96, 96, 16, 8, 128, False), (300, 300, 8, 1, 256, False), (288, 288, 4, 4, 128, True), (130, 130, 2, 2, 32, True),
-    (1, 1, 1, 1, 16, False), (256, 193, 3, 3, 80, False), (200, 200, 2, 2, 64, True)])
+    (1, 1, 1, 1, 16, False), (256, 193, 3, 3, 80, False), (200, 200, 2, 2, 64, True),
+    # few queries and grouped KV heads: query heads of one KV head are folded into one tile (2, 2, 5+1 and 2 per tile)
+    (51, 867, 8, 1, 256, False), (9, 80, 4, 2, 64, False), (17, 40, 6, 1, 64, False), (30, 30, 4, 2, 32, True),
+    (64, 100, 6, 3, 128, False)])
 def test_attention_matches_oracle(tq, tkv, hq, hkv, hd, causal):
     import torch
     from paper_2609_22335_b200 import api
