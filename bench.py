@@ -36,6 +36,7 @@ if ROOT not in sys.path:
 from vla_synth.configs import get_config  # noqa: E402
 from vla_synth.gen import make_weights, frame_inputs  # noqa: E402
 
+RING_DEPTH = 2           # frames in flight per request stream (--ring-depth)
 HOLD_LAUNCH = False      # --hold-launch: the first wave of frames of a pass is admitted by one launch
 CLASS_TAGS = None        # profiled intensity tags (--tags), else the library's hand-assigned ones
 HEAD_PASSES = 1          # action-head passes per VLM pass (--head-passes): asynchronous inference
@@ -147,7 +148,7 @@ def traced_pass(m, weights, R, frames, policy, rank, max_records=8_000_000):
     frames = max(2, min(frames, max_records // ((tiles_per_frame + 1) * R)))
     cap = (tiles_per_frame + 1) * R * frames + 1024
     eng = Engine(m, mode="cosched", n_streams=R, policy=policy, trace_capacity=cap, head_passes=HEAD_PASSES,
-                 device=f"cuda:{torch.cuda.current_device()}")
+                 ring_depth=RING_DEPTH, device=f"cuda:{torch.cuda.current_device()}")
     try:
         eng.load_weights(weights)
         pool = min(frames, 2)
@@ -181,7 +182,7 @@ def run_mode(m, weights, mode, R, F, steps, warmup, e2e_steps, policy, rank, sam
     """Times `steps` passes in one run mode; returns dict with timings."""
     import torch
     from paper_2609_22335_b200 import Engine
-    eng = Engine(m, mode=mode, n_streams=R, policy=policy, head_passes=HEAD_PASSES,
+    eng = Engine(m, mode=mode, n_streams=R, policy=policy, head_passes=HEAD_PASSES, ring_depth=RING_DEPTH,
                  device=f"cuda:{torch.cuda.current_device()}")
     eng.load_weights(weights)
     if CLASS_TAGS is not None:
@@ -308,6 +309,7 @@ def main():
     ap.add_argument("--head-passes", type=int, default=1,
                     help="asynchronous inference: action-head passes (chunks) per VLM pass")
     ap.add_argument("--tags", default=None, help="JSON file written by `auto_tags derive`: profiled intensity tags instead of the hand-assigned ones")
+    ap.add_argument("--ring-depth", type=int, default=2, help="frames in flight per request stream (>= 2)")
     ap.add_argument("--hold-launch", action="store_true",
                     help="hand the first wave of frames of every pass to one launch of the persistent kernel (profiler captures)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -317,7 +319,8 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    global HEAD_PASSES, CLASS_TAGS, HOLD_LAUNCH
+    global HEAD_PASSES, CLASS_TAGS, HOLD_LAUNCH, RING_DEPTH
+    RING_DEPTH = max(2, args.ring_depth)
     HOLD_LAUNCH = args.hold_launch and args.mode == "cosched"
     HEAD_PASSES = max(1, args.head_passes)
     if args.tags:
@@ -329,7 +332,7 @@ def main():
     workload = f"{m.name}: {R} request streams x {F} frames, VLM(n+1) overlapping action head(n)"
     if HEAD_PASSES > 1:
         workload += f", {HEAD_PASSES} action-head passes per VLM pass"
-    config = {"workload": workload, "mode": args.mode, "policy": args.policy, "ring_depth": 2,
+    config = {"workload": workload, "mode": args.mode, "policy": args.policy, "ring_depth": RING_DEPTH,
               "tags": ("profiled: " + os.path.basename(args.tags)) if args.tags else "hand-assigned",
               "l2": "distinct per-stream inputs and weights larger than L2 for cfg2-cfg5; no flush needed" if m.name != "cfg1_tiny"
                     else "working set fits L2 (latency-bound workload)"}
@@ -421,6 +424,14 @@ def main():
             out["speedup_vs_two_stream"] = value / cmp_["two_stream"]["value"]
         if "multi_stream" in cmp_:
             out["speedup_vs_multi_stream"] = value / cmp_["multi_stream"]["value"]
+    if rank == 0 and world == 1 and not args.no_modes and args.mode == "cosched" and RING_DEPTH == 2:
+        # One more data point, not the headline: three frames in flight per request stream instead of two (VLM(n+2) may
+        # then start while head(n) still runs).  With two, a stream whose VLM pass ends before its previous head pass
+        # has no VLM work to offer until that chunk is polled, and the VLM backlog runs dry at times.
+        RING_DEPTH = 3
+        r3 = run_mode(m, weights, "cosched", R, F, 2, 2, 0, args.policy, rank)
+        RING_DEPTH = 2
+        out["ring_depth_3"] = {"value": CH / (r3["device_s"] / 2), "ms_per_step": r3["device_s"] / 2 * 1e3, "steps": 2, "warmup": 2}
     if rank == 0 and world == 1 and not args.no_trace and args.mode == "cosched":
         tr = traced_pass(m, weights, R, F, args.policy, rank)
         out["trace"] = tr

@@ -205,6 +205,13 @@ def gap_stats(trace) -> dict:
         if len(g):
             out[name] = {"gaps": int(len(g)), "mean_us": float(g.mean() * 1e-3), "median_us": float(np.median(g) * 1e-3),
                          "p90_us": float(np.percentile(g, 90) * 1e-3), "share_of_idle": float(g.sum() / tot) if tot > 0 else 0.0}
+    prv = c[:-1][same]
+    for a_, an in ((0, "vlm"), (1, "head")):          # by the phases of the tile before and the tile after the gap
+        for b_, bn in ((0, "vlm"), (1, "head")):
+            g = gap[(prv // N_KINDS == a_) & (nxt // N_KINDS == b_)]
+            if len(g):
+                out[f"{an}->{bn}"] = {"gaps": int(len(g)), "mean_us": float(g.mean() * 1e-3), "median_us": float(np.median(g) * 1e-3),
+                                      "share_of_idle": float(g.sum() / tot) if tot > 0 else 0.0}
     return out
 
 
