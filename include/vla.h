@@ -82,6 +82,11 @@ typedef struct {
   int32_t handoff;
   int32_t head, act_layers, act_d, act_heads, act_mlp, act_mlp_kind;
   int32_t state_dim, horizon, act_dim, n_steps, solver;
+  float guidance;           /* head D variant: classifier-free guidance scale s (0 = off).  Every denoising step evaluates the
+                             * head twice -- with the condition token of a zero cognition feature, then with the real
+                             * one -- and the solver takes eps_u + s (eps_c - eps_u) */
+  int32_t suffix_mask;      /* head B variant: 1 = blocked suffix mask (the leading state token attends the prefix and itself,
+                             * not the action tokens; the action tokens attend everything); 0 = unmasked joint attention */
 } vla_model_desc;
 
 typedef struct {

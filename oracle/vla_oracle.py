@@ -82,11 +82,12 @@ def softmax_rows(s):
     return e / np.sum(e, axis=-1, keepdims=True)
 
 
-def attention(q, k, v, causal=False):
+def attention(q, k, v, causal=False, visible=None):
     """softmax(Q K^T / sqrt(hd) + mask) V per head.
 
     q [Tq,Hq,hd]; k, v [Tkv,Hkv,hd]; query head h reads KV head floor(h*Hkv/Hq).
     causal: key j visible to query i iff j <= i (needs Tq == Tkv).
+    visible: optional boolean [Tq,Tkv]; False entries are masked out (every row must keep one key).
     Returns [Tq,Hq,hd].
     """
     tq, hq, hd = q.shape
@@ -99,6 +100,8 @@ def attention(q, k, v, causal=False):
         if causal:
             assert tq == tkv
             s = np.where(np.tril(np.ones((tq, tkv), dtype=bool)), s, -np.inf)
+        if visible is not None:
+            s = np.where(visible, s, -np.inf)
         out[:, h, :] = softmax_rows(s) @ v[:, g, :]
     return out
 
@@ -225,8 +228,10 @@ def time_condition(m, w, t_arg, dtype):
     return linear(silu(linear(e, w["act.t1"].astype(dtype))), w["act.t2"].astype(dtype))
 
 
-def head_tokens(m, w, vlm, state, x, c_t, dtype):
-    """Token sequence entering the head: [state or condition token ; W_a x_k[i]] plus positions / c_t."""
+def head_tokens(m, w, vlm, state, x, c_t, dtype, uncond=False):
+    """Token sequence entering the head: [state or condition token ; W_a x_k[i]] plus positions / c_t.
+
+    uncond (head D, classifier-free guidance): the condition token is built from a zero cognition feature."""
     tok = linear(x, w["act.in"].astype(dtype))                        # [H, d_a]
     if m.head in ("A", "B"):
         tok = tok + c_t                                               # time enters the action tokens
@@ -235,6 +240,8 @@ def head_tokens(m, w, vlm, state, x, c_t, dtype):
         first = linear(state.astype(dtype), w["act.state"].astype(dtype))
     elif m.head == "D":
         cog = vlm["hidden"][-1]                                       # last position = cognition feature
+        if uncond:
+            cog = np.zeros_like(cog)
         first = linear(cog, w["act.cond"].astype(dtype)) + c_t
     if first is not None:
         tok = np.concatenate([first[None, :], tok], axis=0)
@@ -253,10 +260,10 @@ def _self_attention_block(h, w, p, heads, dtype):
     return linear(a, w[p + "wo"].astype(dtype))
 
 
-def head_velocity(m, w, vlm, state, x, t_arg, dtype=np.float32):
+def head_velocity(m, w, vlm, state, x, t_arg, dtype=np.float32, uncond=False):
     """One evaluation of the head network: v (or eps) [H, A] at sample x and time argument t_arg."""
     c_t = time_condition(m, w, t_arg, dtype)
-    z = head_tokens(m, w, vlm, state, x, c_t, dtype)
+    z = head_tokens(m, w, vlm, state, x, c_t, dtype, uncond)
     ta = z.shape[0]
     s = m.prefix_len
     for i in range(m.act_layers):
@@ -279,7 +286,11 @@ def head_velocity(m, w, vlm, state, x, t_arg, dtype=np.float32):
                 pos = np.arange(s, s + ta)                            # positions continue after the prefix
                 q, k = rope(q, pos), rope(k, pos)
             kp, vp = vlm["kv"][i]                                     # prefix K,V of the same layer index
-            a = attention(q, np.concatenate([kp, k], 0), np.concatenate([vp, v], 0)).reshape(ta, m.hq * m.hd)
+            visible = None
+            if getattr(m, "suffix_mask", 0):                          # blocked suffix mask: the leading state token(s)
+                visible = np.ones((ta, s + ta), dtype=bool)           # see the prefix and themselves, not the actions
+                visible[: m.act_first, s + m.act_first:] = False
+            a = attention(q, np.concatenate([kp, k], 0), np.concatenate([vp, v], 0), visible=visible).reshape(ta, m.hq * m.hd)
             z = z + linear(a, w[p + "wo"].astype(dtype))
             h = rmsnorm(z, w[p + "n2"].astype(dtype))
             z = z + mlp(h, w, p, m.act_mlp_kind, dtype)
@@ -362,6 +373,13 @@ def action_head(m, w, vlm, state, noise, dtype=np.float32):
     if m.solver == "euler":
         return euler_solve(lambda x, t: head_velocity(m, w, vlm, state, x, 1000.0 * t, dtype), x0, m.n_steps)
     if m.solver == "ddim":
+        s_g = float(getattr(m, "guidance", 0.0))
+        if s_g != 0.0:                                                # classifier-free guidance (head D)
+            def guided(x, tau):
+                e_u = head_velocity(m, w, vlm, state, x, float(tau), dtype, uncond=True)
+                e_c = head_velocity(m, w, vlm, state, x, float(tau), dtype)
+                return e_u + dtype(s_g) * (e_c - e_u)
+            return ddim_solve(guided, x0, m.n_steps)
         return ddim_solve(lambda x, tau: head_velocity(m, w, vlm, state, x, float(tau), dtype), x0, m.n_steps)
     raise ValueError(m.solver)
 

@@ -36,7 +36,7 @@ class vla_model_desc(C.Structure):
         "n_cam", "img", "patch", "vis_layers", "vis_d", "vis_heads", "vis_hd", "vis_mlp", "shuffle", "connector",
         "n_text", "vocab", "llm_layers", "d", "hq", "hkv", "hd", "mlp", "mlp_kind", "rope", "causal", "handoff",
         "head", "act_layers", "act_d", "act_heads", "act_mlp", "act_mlp_kind", "state_dim", "horizon", "act_dim",
-        "n_steps", "solver")]
+        "n_steps", "solver")] + [("guidance", C.c_float), ("suffix_mask", C.c_int32)]
 
 
 class vla_runtime_opts(C.Structure):
@@ -120,7 +120,7 @@ def make_desc(m) -> vla_model_desc:
     """vla_synth ModelDesc (or any object with the same fields) -> C struct."""
     d = vla_model_desc()
     for name, _ in vla_model_desc._fields_:
-        v = getattr(m, name)
+        v = getattr(m, name, 0)
         if name in ("mlp_kind", "act_mlp_kind"):
             v = _MLP[v]
         elif name == "handoff":
@@ -129,7 +129,7 @@ def make_desc(m) -> vla_model_desc:
             v = _HEAD[v]
         elif name == "solver":
             v = _SOLVER[v]
-        setattr(d, name, int(v))
+        setattr(d, name, float(v) if name == "guidance" else int(v))
     return d
 
 

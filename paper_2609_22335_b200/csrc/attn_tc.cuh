@@ -83,11 +83,11 @@ __device__ __forceinline__ KvBlock kv_next(const A& a, KvBlock b, int q_last) {
 __device__ void tile_attention(const TileCtx& c, const AttnArgs& a_in, int tile) {
   // The node's arguments live in global memory; the shared-memory stores and the asm statements of the block loop
   // would make the compiler fetch them again and again, so the ones the loop uses are copied into registers.
-  struct { int32_t k0map, v0map, k1map, v1map, t0, t1, causal, hq, hkv, hs, hd, q_blocks, qmap, tq, ldo, hpt, rph; float scale_log2e; Ref out; } a;
+  struct { int32_t k0map, v0map, k1map, v1map, t0, t1, causal, hq, hkv, hs, hd, q_blocks, qmap, tq, ldo, hpt, rph, sfx; float scale_log2e; Ref out; } a;
   a.k0map = a_in.k0map; a.v0map = a_in.v0map; a.k1map = a_in.k1map; a.v1map = a_in.v1map; a.t0 = a_in.t0; a.t1 = a_in.t1;
   a.causal = a_in.causal; a.hq = a_in.hq; a.hkv = a_in.hkv; a.hs = a_in.hs; a.hd = a_in.hd; a.q_blocks = a_in.q_blocks;
   a.qmap = a_in.qmap; a.tq = a_in.tq; a.ldo = a_in.ldo; a.scale_log2e = a_in.scale_log2e; a.out = a_in.out;
-  a.hpt = a_in.hpt > 1 ? a_in.hpt : 1; a.rph = a_in.rph;
+  a.hpt = a_in.hpt > 1 ? a_in.hpt : 1; a.rph = a_in.rph; a.sfx = a_in.sfx;
   const int warp = c.tid >> 5, lane = c.tid & 31;
   // folded: tile -> (KV head g, first query head, heads in this tile); else tile -> (head, query block)
   const bool folded = a.hpt > 1;
@@ -195,7 +195,9 @@ __device__ void tile_attention(const TileCtx& c, const AttnArgs& a_in, int tile)
     // ---- softmax of this block: one thread per query row, the 64 scores held in registers
     const int L = cur.seg == 0 ? a.t0 : a.t1;
     const int valid = min(ATTN_BN, L - cur.kv0);
-    const int lim = a.causal ? min(valid, row - cur.kv0 + 1) : valid;   // keys [0, lim) of the block are visible to this row
+    int lim = a.causal ? min(valid, row - cur.kv0 + 1) : valid;   // keys [0, lim) of the block are visible to this row
+    if (a.sfx > 0 && cur.seg == 1 && row < a.sfx) lim = min(lim, a.sfx - cur.kv0);   // blocked suffix: the leading own tokens
+                                                                                    // see only one another in segment 1
     uint32_t sr[ATTN_BN];
     tmem_ld16_nowait(tmem_s + lane_off + 0u, sr + 0);
     tmem_ld16_nowait(tmem_s + lane_off + 16u, sr + 16);

@@ -209,6 +209,7 @@ class Builder {
     Ref tab = 0; int ldtab = 0;
     Ref tab2 = 0; int ldtab2 = 0;
     View out32, out16, outT;
+    View tabv;               // an fp32 [M, ld] addend that is one of the frame's buffers (read dependency tracked)
     int t_col0 = 0;
     int act = ACT_NONE;
     int W2 = -1;
@@ -230,6 +231,7 @@ class Builder {
     g.X = ref(o.X); g.ldx = o.X.buf >= 0 ? (int)ld(o.X) : 0;
     g.c_x = o.c_x; g.c_acc = o.c_acc;
     g.vec = o.vec; g.tab = o.tab; g.ldtab = o.ldtab; g.tab2 = o.tab2; g.ldtab2 = o.ldtab2;
+    if (o.tabv.buf >= 0) { g.tab = ref(o.tabv); g.ldtab = (int)ld(o.tabv); }
     g.out32 = ref(o.out32); g.ldo32 = o.out32.buf >= 0 ? (int)ld(o.out32) : 0;
     g.out16 = ref(o.out16); g.ldo16 = o.out16.buf >= 0 ? (int)ld(o.out16) : 0;
     g.outT = ref(o.outT); g.ldoT = o.outT.buf >= 0 ? (int)ld(o.outT) : 0; g.t_col0 = o.t_col0;
@@ -273,6 +275,7 @@ class Builder {
     }
     read(id, A);
     if (o.X.buf >= 0) read(id, o.X);
+    if (o.tabv.buf >= 0) read(id, o.tabv);
     if (o.out32.buf >= 0) write(id, o.out32);
     if (o.out16.buf >= 0) write(id, o.out16);
     if (o.outT.buf >= 0) write(id, o.outT);
@@ -341,14 +344,14 @@ class Builder {
   // Fused attention of the queries in `q` (rows [0,tq), head h at column h*hs) over the keys/values of
   // kv0 (all its T tokens) and then, optionally, kv1.
   int attention(const std::string& name, const View& q, int tq, const QKV& kv0, const QKV* kv1, const View& out, int hq,
-                int hkv, int hd, int hs, bool causal) {
+                int hkv, int hd, int hs, bool causal, int sfx = 0) {
     NodeDesc n;
     std::memset(&n, 0, sizeof(n));
     n.op = OP_ATTN;
     AttnArgs& a = n.u.attn;
     a.out = ref(out); a.ldo = (int)ld(out);
     a.tq = tq; a.t0 = kv0.T; a.t1 = kv1 ? kv1->T : 0;
-    a.hq = hq; a.hkv = hkv; a.hd = hd; a.hs = hs; a.causal = causal;
+    a.hq = hq; a.hkv = hkv; a.hd = hd; a.hs = hs; a.causal = causal; a.sfx = sfx;
     a.bn = 64;
     a.q_blocks = (tq + 127) / 128;
     a.scale_log2e = 1.4426950408889634f / std::sqrt((float)hd);
@@ -460,6 +463,10 @@ bool validate(const vla_model_desc& d, Program& p) {
   if (d.head == VLA_HEAD_C && d.handoff != VLA_HANDOFF_FEATURES) return bad("head C needs the features handoff");
   if (d.head == VLA_HEAD_D && (d.handoff != VLA_HANDOFF_COG || d.state_dim != 0)) return bad("head D needs the cog handoff and no state");
   if (d.head == VLA_HEAD_A && d.state_dim == 0) return bad("head A needs a state token");
+  if (d.guidance != 0.0f && (d.head != VLA_HEAD_D || d.solver != VLA_SOLVER_DDIM))
+    return bad("classifier-free guidance needs head D with the DDIM solver");
+  if (d.suffix_mask != 0 && (d.suffix_mask != 1 || d.head != VLA_HEAD_B || d.state_dim == 0))
+    return bad("the blocked suffix mask needs head B with a state token");
   return true;
 }
 
@@ -821,6 +828,8 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   int aqc = (d.head == VLA_HEAD_A || d.head == VLA_HEAD_C) ? b.buf("act.qc", Ta, d.head == VLA_HEAD_A ? nq : da, 2) : -1;
   int amid = b.buf("act.mid", Ta, P64(d.act_mlp), 2);
   int tok0 = first ? b.buf("act.tok0", 1, da, 4) : -1;
+  const bool guided = d.guidance != 0.0f;
+  int vu = guided ? b.buf("act.vu", d.horizon, d.act_dim, 4) : -1;   // the unconditional branch's share of the update
   int state_bf = has_state ? b.buf("act.state_bf", 1, P64(d.state_dim), 2) : -1;
 
   // Asynchronous inference: the head runs P times on the same VLM output, pass by pass on the same buffers (the
@@ -847,9 +856,18 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   for (int k = 0; k < ns; ++k) {
     b.step = k;
     Ref ct_k = b.ref(b.rows(c_ct, k, 1));
+    // classifier-free guidance: the head runs twice per step on the same buffers, first with the condition token of a
+    // zero cognition feature (its epsilon, scaled, parked in act.vu), then with the real one
+    for (int branch = guided ? 0 : 1; branch < 2; ++branch) {
+    const bool uncond = branch == 0;
+    const std::string saved_suffix = b.name_suffix;
+    if (uncond) b.name_suffix += ".u";
     if (first) {
-      b.addrows(N_("act.s%d.tok0", k), b.all(tok0), 0, 0, 1, da, d.head == VLA_HEAD_D ? ct_k : 0, 0, 0, b.rows(z, 0, 1),
-                b.rows(zb, 0, 1));
+      if (uncond)     // W_c . 0 + pos_0 + c_t
+        b.addrows(N_("act.s%d.tok0", k), View(), b.wref(w_apos, 0), da, 1, da, ct_k, 0, 0, b.rows(z, 0, 1), b.rows(zb, 0, 1));
+      else
+        b.addrows(N_("act.s%d.tok0", k), b.all(tok0), 0, 0, 1, da, d.head == VLA_HEAD_D ? ct_k : 0, 0, 0, b.rows(z, 0, 1),
+                  b.rows(zb, 0, 1));
     }
     {
       Builder::GemmOpt g;
@@ -875,7 +893,8 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
         b.qkv_project(NN(""), nin, a.wqkv, aq, ahd, aqkv32, S, fold ? a.n1 : -1, da);
         View att_out = b.rows(aatt, 0, Ta);
         if (d.head == VLA_HEAD_B)
-          b.attention(NN("attn"), b.rows(aq.qk, 0, Ta, 0), Ta, lq[i], &aq, att_out, d.hq, d.hkv, d.hd, lhs, false);
+          b.attention(NN("attn"), b.rows(aq.qk, 0, Ta, 0), Ta, lq[i], &aq, att_out, d.hq, d.hkv, d.hd, lhs, false,
+                      d.suffix_mask ? first : 0);
         else
           b.attention(NN("attn"), b.rows(aq.qk, 0, Ta, 0), Ta, aq, nullptr, att_out, d.act_heads, d.act_heads, ahd, ahs, false);
         b.gemm(NN("wo"), b.all(aatt), a.wo, da, resid());
@@ -911,11 +930,19 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     {
       // final RMSNorm folded into the output projection; the solver update is its epilogue
       Builder::GemmOpt g;
-      g.X = b.all(xs); g.c_x = p.step_c_x[k]; g.c_acc = p.step_c_acc[k];
-      g.out32 = b.all(xs); g.out16 = b.all(xbf);
       g.norm_gain = w_anorm; g.norm_d = da;
+      if (uncond) {          // vu = c_acc (1 - s) eps_u
+        g.c_acc = p.step_c_acc[k] * (1.0f - d.guidance);
+        g.out32 = b.all(vu);
+      } else {               // x <- c_x x + c_acc s eps_c + vu   (s = 1 and vu = 0 without guidance)
+        g.X = b.all(xs); g.c_x = p.step_c_x[k]; g.c_acc = guided ? p.step_c_acc[k] * d.guidance : p.step_c_acc[k];
+        if (guided) g.tabv = b.all(vu);
+        g.out32 = b.all(xs); g.out16 = b.all(xbf);
+      }
       b.gemm(N_("act.s%d.out", k), b.rows(zb, first, d.horizon), w_aout, d.act_dim, g);
     }
+    b.name_suffix = saved_suffix;
+    }   // guidance branches
   }
   b.step = -1;
   {

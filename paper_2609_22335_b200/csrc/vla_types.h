@@ -110,6 +110,7 @@ struct AttnArgs {
   int32_t hq, hkv, hd, hs;     // hs = head stride (hd padded to a multiple of 16)
   int32_t causal;
   int32_t bn, q_blocks;        // keys per block; 128-query blocks
+  int32_t sfx, pad_;           // blocked suffix mask: queries [0, sfx) see only keys [0, sfx) of segment 1 (0 = no mask)
   int32_t hpt, rph;            // query heads folded into one tile (they share a KV head; 1 = none) and the rows each
                                // takes in the tile (tq rounded up to a multiple of 8); folding needs q_blocks == 1
   float scale_log2e;           // log2(e) / sqrt(hd)

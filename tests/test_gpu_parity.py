@@ -304,3 +304,43 @@ def test_no_tile_writes_outside_its_buffers(key):
         assert eng.overwritten_guards() == 0, eng.last_error()
     finally:
         eng.close()
+
+
+def test_blocked_suffix_mask():
+    """Workload variant of the joint-attention expert (head B with a state token): the state token does not attend the
+    action tokens.  Against the oracle, across modes, and different from the unmasked workload."""
+    base = SMALL["cfg4s"]
+    m = mini(base, suffix_mask=1)
+    w = make_weights(m, seed=0)
+    frames = [[frame_inputs(m, r, n, seed=0) for n in range(2)] for r in range(2)]
+    got, _ = _run(m, w, frames, "cosched")
+    worst = _check_vs_oracle(m, w, frames, got)
+    print(f"blocked suffix: worst rel-L2 {worst[0]:.2e}, max-abs {worst[1]:.3e}")
+    ser, _ = _run(m, w, frames, "serial")
+    plain, _ = _run(base, w, frames, "cosched")
+    for r in range(2):
+        for n in range(2):
+            assert np.array_equal(got[r][n], ser[r][n])
+            assert not np.array_equal(got[r][n], plain[r][n])
+
+
+def test_classifier_free_guidance():
+    """Workload variant of the in-context DiT head (head D, DDIM): two head evaluations per step, unconditional then
+    conditional, combined in the solver epilogue.  Against the oracle, across modes; scale 1 reproduces the unguided
+    chunk up to rounding, scale 3 does not."""
+    base = SMALL["cfg5s"]
+    frames = [[frame_inputs(base, r, n, seed=0) for n in range(2)] for r in range(2)]
+    w = make_weights(base, seed=0)
+    plain, _ = _run(base, w, frames, "cosched")
+    for scale in (1.0, 3.0):
+        m = mini(base, guidance=scale)
+        got, extra = _run(m, w, frames, "cosched", trace_capacity=1 << 20)
+        _check_trace(extra["trace"], extra["trace_total"], extra["program"], 2, 2)
+        worst = _check_vs_oracle(m, w, frames, got)
+        print(f"guidance {scale}: worst rel-L2 {worst[0]:.2e}, max-abs {worst[1]:.3e} at chunk rms {worst[2]:.2f}")
+        ser, _ = _run(m, w, frames, "serial")
+        for r in range(2):
+            for n in range(2):
+                assert np.array_equal(got[r][n], ser[r][n])
+                d = float(np.max(np.abs(got[r][n] - plain[r][n])))
+                assert (d < 5e-2) if scale == 1.0 else (d > 5e-2), (scale, d)

@@ -282,8 +282,19 @@ def restated_head(m, w, vlm, state, x, t_arg):
                 q = [[rotate(q[t][hh], S + t) for hh in range(m.hq)] for t in range(Ta)]
                 k = [[rotate(k[t][hh], S + t) for hh in range(m.hkv)] for t in range(Ta)]
             Kp, Vp = vlm["kv"][i]                                              # prefix cache of the SAME layer index
-            keys, vals = L(Kp) + k, L(Vp) + v                                  # [prefix ; own], no mask
-            a = mha(q, keys, vals, m.hq, m.hkv, m.hd)
+            first = Ta - H
+            if getattr(m, "suffix_mask", 0):
+                # blocked suffix mask: the leading state token sees the prefix and the state token(s) only; an action
+                # token sees the prefix, the state token(s) and every action token
+                a = []
+                for t in range(Ta):
+                    own = range(first) if t < first else range(Ta)
+                    keys = L(Kp) + [k[j] for j in own]
+                    vals = L(Vp) + [v[j] for j in own]
+                    a += mha([q[t]], keys, vals, m.hq, m.hkv, m.hd)
+            else:
+                keys, vals = L(Kp) + k, L(Vp) + v                              # [prefix ; own], no mask
+                a = mha(q, keys, vals, m.hq, m.hkv, m.hd)
             z = [add(z[t], matvec(W[p + "wo"], a[t])) for t in range(Ta)]
             h = [rms(r, W[p + "n2"]) for r in z]
             z = [add(z[t], head_mlp(m, W, p, h[t])) for t in range(Ta)]
@@ -324,6 +335,8 @@ HEAD_CASES = {
                    horizon=4, act_dim=3),
     "B_rope": mini(CFG4, **_VLM, llm_layers=2, d=24, hq=4, hkv=1, hd=8, mlp=20, act_layers=2, act_d=12, act_mlp=20,
                    state_dim=5, horizon=4, act_dim=3),
+    "B_rope_blocked_suffix": mini(CFG4, **_VLM, llm_layers=2, d=24, hq=4, hkv=1, hd=8, mlp=20, act_layers=2, act_d=12, act_mlp=20,
+                                  state_dim=5, horizon=4, act_dim=3, suffix_mask=1),
     "C": mini(CFG3, **_VLM, shuffle=1, llm_layers=1, d=24, hq=2, hkv=2, hd=8, mlp=20, act_layers=2, act_d=12, act_heads=2,
               act_mlp=20, state_dim=5, horizon=4, act_dim=3),
     "D": mini(CFG5, **_VLM, llm_layers=1, d=24, hq=2, hkv=2, hd=8, mlp=20, act_layers=2, act_d=12, act_heads=2, act_mlp=20,
@@ -358,6 +371,23 @@ def test_head_velocity_composition(key):
     assert np.max(np.abs(a - c)) > 1e-3
 
 
+def test_blocked_suffix_mask_changes_the_state_token_only_at_layer_one():
+    """With one head layer the mask can only change what the state token computes; the action tokens' outputs
+    (the only rows the head returns) then depend on it through nothing -- so a one-layer head is unchanged, a
+    two-layer head is not."""
+    rng = np.random.default_rng(77)
+    for layers, same in ((1, True), (2, False)):
+        base = mini(HEAD_CASES["B_rope"], act_layers=layers, llm_layers=max(layers, 2))
+        w = random_weights(base, rng, only="act.")
+        S = base.prefix_len
+        vlm = {"kv": [(rng.standard_normal((S, base.hkv, base.hd)), rng.standard_normal((S, base.hkv, base.hd)))
+                      for _ in range(base.llm_layers)], "hidden": rng.standard_normal((S, base.d))}
+        state, x = rng.standard_normal(base.state_dim), rng.standard_normal((base.horizon, base.act_dim))
+        a = O.head_velocity(base, w, vlm, state, x, 100.0, F64)
+        b = O.head_velocity(mini(base, suffix_mask=1), w, vlm, state, x, 100.0, F64)
+        assert (np.max(np.abs(a - b)) < 1e-12) == same
+
+
 def test_action_chunk_is_solver_of_head_on_vlm_output():
     """action_chunk feeds frame n's own VLM output, state and noise to the solver (Euler: x += v/n, t_k = k/n,
     time argument 1000 t_k)."""
@@ -373,3 +403,38 @@ def test_action_chunk_is_solver_of_head_on_vlm_output():
         v = restated_head(m2, w, vlm, fr["state"], np.array(x), 1000.0 * k / m2.n_steps)
         x = [[x[i][j] + v[i][j] / m2.n_steps for j in range(m2.act_dim)] for i in range(m2.horizon)]
     close(O.action_chunk(m2, w, fr, F64), x)
+
+
+def test_classifier_free_guidance_composition():
+    """Head D with guidance: the unconditional branch is the head on a zero cognition feature (restated with loops),
+    and the guided epsilon is e_u + s (e_c - e_u) fed to DDIM."""
+    m = HEAD_CASES["D"]
+    rng = np.random.default_rng(909)
+    w = random_weights(m, rng, only="act.")
+    S = m.prefix_len
+    vlm = {"kv": [], "hidden": rng.standard_normal((S, m.d))}
+    x = rng.standard_normal((m.horizon, m.act_dim))
+    zero = {"kv": [], "hidden": vlm["hidden"].copy()}
+    zero["hidden"][S - 1] = 0.0
+    e_u = O.head_velocity(m, w, vlm, None, x, 40.0, F64, uncond=True)
+    close(e_u, restated_head(m, w, zero, None, x, 40.0))
+    e_c = O.head_velocity(m, w, vlm, None, x, 40.0, F64)
+    assert np.max(np.abs(e_u - e_c)) > 1e-3
+    # the guided chunk: DDIM driven by e_u + s (e_c - e_u), written out here with the restated head
+    s_g = 2.5
+    mg = mini(m, guidance=s_g, n_steps=2)
+    noise = rng.standard_normal((m.horizon, m.act_dim))
+    got = O.action_head(mg, w, vlm, None, noise, F64)
+    ab = O.ddim_alpha_bar()
+    xs = noise.copy()
+    for tau in (50, 0):
+        eu = np.array(restated_head(mg, w, zero, None, xs, float(tau)))
+        ec = np.array(restated_head(mg, w, vlm, None, xs, float(tau)))
+        eps = eu + s_g * (ec - eu)
+        a_t, a_prev = ab[tau], (ab[tau - 50] if tau - 50 >= 0 else 1.0)
+        x0 = (xs - math.sqrt(1 - a_t) * eps) / math.sqrt(a_t)
+        xs = math.sqrt(a_prev) * x0 + math.sqrt(1 - a_prev) * eps
+    close(got, xs)
+    # s = 1 is the conditional head alone; s = 0 switches guidance off
+    close(O.action_head(mini(m, guidance=1.0, n_steps=2), w, vlm, None, noise, F64),
+          O.action_head(mini(m, guidance=0.0, n_steps=2), w, vlm, None, noise, F64))

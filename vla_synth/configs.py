@@ -61,6 +61,11 @@ class ModelDesc:
     # ---- workload
     n_streams: int
     n_frames: int
+    # ---- workload variants (defaults: the five stated workloads)
+    guidance: float = 0.0   # head D: classifier-free guidance scale s (0 = off): eps = eps_u + s (eps_c - eps_u), the
+                            # unconditional branch built from a zero cognition feature
+    suffix_mask: int = 0    # head B: 1 = blocked suffix mask -- the leading state token attends the prefix and itself
+                            # but not the action tokens (the action tokens still attend everything)
 
     # -------- derived sizes
     @property
