@@ -87,6 +87,9 @@ typedef struct {
                              * one -- and the solver takes eps_u + s (eps_c - eps_u) */
   int32_t suffix_mask;      /* head B variant: 1 = blocked suffix mask (the leading state token attends the prefix and itself,
                              * not the action tokens; the action tokens attend everything); 0 = unmasked joint attention */
+  int32_t vis_layernorm;    /* vision encoder variant: 1 = LayerNorm (gain and shift, weights "...n1b", "...n2b", "vis.normb")
+                             * in place of RMSNorm, and an fp32 bias vector on every linear layer of the encoder
+                             * ("vis.patch.b", "...bq", "...bk", "...bv", "...bo", "...b1", "...b2"); 0 = RMSNorm, no biases */
 } vla_model_desc;
 
 typedef struct {

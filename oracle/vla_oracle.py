@@ -54,6 +54,14 @@ def rmsnorm(x, g):
     return x / np.sqrt(ms + x.dtype.type(RMS_EPS)) * g
 
 
+def layernorm(x, g, b):
+    """y_i = g_i (x_i - mean) / sqrt(var + eps) + b_i over the last axis (biased variance)."""
+    mu = np.mean(x, axis=-1, keepdims=True)
+    xc = x - mu
+    var = np.mean(xc * xc, axis=-1, keepdims=True)
+    return xc / np.sqrt(var + x.dtype.type(RMS_EPS)) * g + b
+
+
 def gelu_tanh(x):
     """0.5 x (1 + tanh( sqrt(2/pi) (x + 0.044715 x^3) ))."""
     c = x.dtype.type(math.sqrt(2.0 / math.pi))
@@ -148,6 +156,20 @@ def timestep_embedding(arg, width, dtype):
 
 
 # --------------------------------------------------------------------------- VLM phase
+def _encoder_layer_ln(x, w, p, heads, hd, dtype):
+    """Vision encoder layer of the LayerNorm variant: LayerNorm with shift, and a bias on every linear layer."""
+    W = lambda n: w[p + n].astype(dtype)  # noqa: E731
+    t = x.shape[0]
+    h = layernorm(x, W("n1"), W("n1b"))
+    q = (linear(h, W("wq")) + W("bq")).reshape(t, heads, hd)
+    k = (linear(h, W("wk")) + W("bk")).reshape(t, heads, hd)
+    v = (linear(h, W("wv")) + W("bv")).reshape(t, heads, hd)
+    a = attention(q, k, v).reshape(t, heads * hd)
+    x = x + linear(a, W("wo")) + W("bo")
+    h = layernorm(x, W("n2"), W("n2b"))
+    return x + linear(gelu_tanh(linear(h, W("w1")) + W("b1")), W("w2")) + W("b2")
+
+
 def _encoder_layer(x, w, p, heads, hd, dtype):
     h = rmsnorm(x, w[p + "n1"].astype(dtype))
     t = x.shape[0]
@@ -163,13 +185,17 @@ def _encoder_layer(x, w, p, heads, hd, dtype):
 def vision_tokens(m, w, image, dtype):
     """Cameras -> image tokens in the LLM width: patch embed (+pos) -> encoder -> final norm -> shuffle -> connector."""
     patches = patchify(image.astype(dtype), m.patch)
+    ln = bool(getattr(m, "vis_layernorm", 0))
     outs = []
     for cam in range(m.n_cam):
         x = linear(patches[cam], w["vis.patch.w"].astype(dtype)) + w["vis.pos"].astype(dtype)
+        if ln:
+            x = x + w["vis.patch.b"].astype(dtype)
         for i in range(m.vis_layers):
-            x = _encoder_layer(x, w, f"vis.L{i}.", m.vis_heads, m.vis_hd, dtype)
+            layer = _encoder_layer_ln if ln else _encoder_layer
+            x = layer(x, w, f"vis.L{i}.", m.vis_heads, m.vis_hd, dtype)
         if m.vis_layers > 0:
-            x = rmsnorm(x, w["vis.norm"].astype(dtype))
+            x = layernorm(x, w["vis.norm"].astype(dtype), w["vis.normb"].astype(dtype)) if ln else rmsnorm(x, w["vis.norm"].astype(dtype))
         if m.shuffle > 1:
             x = pixel_shuffle_tokens(x, m.grid, m.shuffle)
         if m.connector:

@@ -36,7 +36,7 @@ class vla_model_desc(C.Structure):
         "n_cam", "img", "patch", "vis_layers", "vis_d", "vis_heads", "vis_hd", "vis_mlp", "shuffle", "connector",
         "n_text", "vocab", "llm_layers", "d", "hq", "hkv", "hd", "mlp", "mlp_kind", "rope", "causal", "handoff",
         "head", "act_layers", "act_d", "act_heads", "act_mlp", "act_mlp_kind", "state_dim", "horizon", "act_dim",
-        "n_steps", "solver")] + [("guidance", C.c_float), ("suffix_mask", C.c_int32)]
+        "n_steps", "solver")] + [("guidance", C.c_float), ("suffix_mask", C.c_int32), ("vis_layernorm", C.c_int32)]
 
 
 class vla_runtime_opts(C.Structure):
@@ -205,7 +205,7 @@ class Engine:
     def load_weights(self, weights, batch_bytes=1 << 30):
         """weights: mapping name -> fp32 ndarray of bf16-representable values (vla_synth.gen.Weights)."""
         from vla_synth.gen import bf16_bits
-        from vla_synth.configs import is_gain
+        from vla_synth.configs import is_vector
         names = list(weights.names())
         batch, keep, size = [], [], 0
 
@@ -216,7 +216,7 @@ class Engine:
 
         for i, name in enumerate(names):
             w = weights[name]
-            fp32 = is_gain(name) or name in ("vis.pos", "llm.pos", "act.pos")
+            fp32 = is_vector(name) or name in ("vis.pos", "llm.pos", "act.pos")
             a = np.ascontiguousarray(w, dtype=np.float32) if fp32 else bf16_bits(w)
             keep.append(a)
             t = vla_tensor()

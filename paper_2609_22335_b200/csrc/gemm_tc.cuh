@@ -129,7 +129,7 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 // feature of the V^T part of a q|k|v projection is written from here, 16 consecutive tokens per store pair.
 struct Phase1Args {
   float* St; const float* rs; unsigned short* outT_row;
-  float c_acc, c_x; uint32_t lane_base; int bt, nt, tid, t0;
+  float c_acc, c_x, bias; uint32_t lane_base; int bt, nt, tid, t0;
   bool x_staged;            // the residual rows already sit in St: accumulate on top of them
 };
 template <int ACT>
@@ -149,7 +149,7 @@ __device__ __forceinline__ void gemm_phase1(const Phase1Args& p) {
     }
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      v[j] = apply_act_t<ACT>(a[j] * sc[j]) * p.c_acc;
+      v[j] = apply_act_t<ACT>(fmaf(a[j], sc[j], p.bias)) * p.c_acc;
     }
     if (p.outT_row) {
       unsigned short* op = p.outT_row + p.t0 + c0;
@@ -382,6 +382,7 @@ __device__ void tile_gemm(const TileCtx& c, const GemmArgs& g, int tile) {
     p1.lane_base = tmem_d + ((uint32_t)(warp * 32) << 16);
     p1.bt = g.bt; p1.nt = nt; p1.tid = c.tid; p1.t0 = t0;
     const int f = f0 + c.tid;
+    p1.bias = (ptrs.bias != nullptr && f < g.N) ? ptrs.bias[f] : 0.0f;      // this thread's output feature
     p1.outT_row = (ptrs.outT != nullptr && f >= g.t_col0 && f < g.N) ? ptrs.outT + (size_t)(f - g.t_col0) * g.ldoT : nullptr;
     if (dual) { p1.c_acc = 1.0f; gemm_phase1<ACT_NONE>(p1); }   // gate and up rows parked raw: phase 2 combines them
     else if (g.act == ACT_GELU) gemm_phase1<ACT_GELU>(p1);

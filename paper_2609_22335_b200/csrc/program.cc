@@ -150,6 +150,23 @@ class Builder {
     p.sources.push_back(s);
     return d;
   }
+  // an fp32 vector made of per-head vectors stacked with each head padded from hd to hs elements (padding stays zero)
+  int vector_heads(const std::string& dev_name, const std::vector<std::string>& parts, const std::vector<int64_t>& part_heads,
+                   int64_t hd, int64_t hs) {
+    int64_t heads = 0;
+    for (auto h : part_heads) heads += h;
+    int d = dev_tensor(dev_name, 1, heads * hs, false);
+    int64_t off = 0;
+    for (size_t i = 0; i < parts.size(); ++i) {
+      SourceTensor s;
+      s.name = parts[i]; s.rows = part_heads[i] * hd; s.cols = 0; s.dev = d; s.row_offset = off;
+      if (hd != hs) { s.group_rows = hd; s.group_stride = hs; }
+      p.source_index[s.name] = (int)p.sources.size();
+      p.sources.push_back(s);
+      off += part_heads[i] * hs;
+    }
+    return d;
+  }
   Ref wref(int dev, int64_t row0 = 0) const {
     const DevTensor& t = p.dev_tensors[dev];
     return WEIGHT_BASE + t.offset + (uint64_t)row0 * t.ld * (t.is_bf16 ? 2 : 4);
@@ -213,6 +230,7 @@ class Builder {
     int t_col0 = 0;
     int act = ACT_NONE;
     int W2 = -1;
+    int bias = -1;           // >= 0: an fp32 [N] device tensor added to the accumulator before the activation
     int64_t w_row0 = 0;
     int norm_gain = -1;      // >= 0: A is the raw residual stream; RMSNorm with this gain is folded into the GEMM
     int norm_d = 0;
@@ -230,6 +248,7 @@ class Builder {
     g.M = (int)A.rows; g.N = (int)N; g.Kp = (int)wt.ld;
     g.X = ref(o.X); g.ldx = o.X.buf >= 0 ? (int)ld(o.X) : 0;
     g.c_x = o.c_x; g.c_acc = o.c_acc;
+    g.bias = o.bias >= 0 ? wref(o.bias) : 0;
     g.vec = o.vec; g.tab = o.tab; g.ldtab = o.ldtab; g.tab2 = o.tab2; g.ldtab2 = o.ldtab2;
     if (o.tabv.buf >= 0) { g.tab = ref(o.tabv); g.ldtab = (int)ld(o.tabv); }
     g.out32 = ref(o.out32); g.ldo32 = o.out32.buf >= 0 ? (int)ld(o.out32) : 0;
@@ -261,6 +280,7 @@ class Builder {
       n.tmem_cols = (int)pad_to((int64_t)bt, TMEM_UNIT);
       g.wmap = weight_map(W, N, g.dual ? GEMM_BM / 2 : GEMM_BM);
       g.w2map = o.W2 >= 0 ? weight_map(o.W2, N, GEMM_BM / 2) : 0;
+      if (g.dual && o.bias >= 0) p.error = "a gated GEMM takes no bias";
       if (g.dual && (N % 4 != 0 || o.X.buf >= 0 || o.outT.buf >= 0 || o.out32.buf >= 0 || o.tab || o.tab2 || o.vec))
         p.error = "internal: a gated GEMM writes bf16 only, width a multiple of 4 (" + name + ")";
       g.amap = act_map(A, g.Kp, bt);
@@ -312,7 +332,7 @@ class Builder {
   }
 
   int rmsnorm(const std::string& name, const View& x, int g_dev, const View& out, Ref mod = 0, int shuffle = 1,
-              int grid = 0) {
+              int grid = 0, int beta_dev = -1) {
     NodeDesc n;
     std::memset(&n, 0, sizeof(n));
     n.op = OP_RMSNORM;
@@ -320,7 +340,9 @@ class Builder {
     a.x = ref(x); a.g = wref(g_dev); a.mod = mod; a.out = ref(out);
     a.M = (int)x.rows; a.d = (int)p.dev_tensors[g_dev].cols; a.ldx = (int)ld(x); a.ldo = (int)ld(out);
     a.rows_per_tile = 16; a.shuffle = shuffle; a.grid = grid;
+    if (beta_dev >= 0) { a.ln = 1; a.beta = wref(beta_dev); }
     if (a.d % 4) p.error = "model widths must be multiples of 4";
+    if (a.ln && a.d > 2048) p.error = "LayerNorm rows wider than 2048 are not supported";
     n.n_tiles = (a.M + a.rows_per_tile - 1) / a.rows_per_tile;
     int id = add(n, name, KIND_ELEM);
     read(id, x);
@@ -383,7 +405,7 @@ class Builder {
   // q|k|v projection of `A` into `dst`: one GEMM whose V columns are written transposed; with RoPE the
   // GEMM writes fp32 and a rotary tile produces the bf16 q|k and V^T.
   void qkv_project(const std::string& name, const View& A, int W, const QKV& dst, int hd, int scratch32, int pos0,
-                   int norm_gain = -1, int norm_d = 0) {
+                   int norm_gain = -1, int norm_d = 0, int bias = -1) {
     const int64_t nqk = (int64_t)(dst.hq + dst.hkv) * dst.hs, nall = nqk + (int64_t)dst.hkv * dst.hs;
     if (scratch32 >= 0) {
       GemmOpt gq; gq.out32 = all(scratch32); gq.norm_gain = norm_gain; gq.norm_d = norm_d;
@@ -402,7 +424,7 @@ class Builder {
       write(id, all(dst.qk));
       write(id, all(dst.vt));
     } else {
-      GemmOpt gq; gq.out16 = all(dst.qk); gq.outT = all(dst.vt); gq.t_col0 = (int)nqk;
+      GemmOpt gq; gq.out16 = all(dst.qk); gq.outT = all(dst.vt); gq.t_col0 = (int)nqk; gq.bias = bias;
       gq.norm_gain = norm_gain; gq.norm_d = norm_d;
       gemm(name + "qkv", A, W, nall, gq);
     }
@@ -465,6 +487,7 @@ bool validate(const vla_model_desc& d, Program& p) {
   if (d.head == VLA_HEAD_A && d.state_dim == 0) return bad("head A needs a state token");
   if (d.guidance != 0.0f && (d.head != VLA_HEAD_D || d.solver != VLA_SOLVER_DDIM))
     return bad("classifier-free guidance needs head D with the DDIM solver");
+  if (d.vis_layernorm != 0 && d.vis_layernorm != 1) return bad("vis_layernorm must be 0 or 1");
   if (d.suffix_mask != 0 && (d.suffix_mask != 1 || d.head != VLA_HEAD_B || d.state_dim == 0))
     return bad("the blocked suffix mask needs head B with a state token");
   return true;
@@ -523,9 +546,11 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
   auto N_ = [&](const char* fmt, int a = 0, int c = 0) { std::snprintf(nm, sizeof nm, fmt, a, c); return std::string(nm); };
 
   // ================================================================== weights
+  const bool vln = d.vis_layernorm != 0;     // LayerNorm-and-bias variant of the vision encoder
   int w_patch = b.matrix1("vis.patch.w", dv, patch_k);
+  int w_patch_b = vln ? b.gain("vis.patch.b", dv) : -1;
   int w_vpos = b.table("vis.pos", T, dv);
-  struct EncW { int n1, wqkv, wo, n2, w1, w2; };
+  struct EncW { int n1, wqkv, wo, n2, w1, w2, n1b = -1, bqkv = -1, bo = -1, n2b = -1, b1 = -1, b2 = -1; };
   std::vector<EncW> venc(d.vis_layers);
   for (int i = 0; i < d.vis_layers; ++i) {
     std::string pre = N_("vis.L%d.", i);
@@ -536,8 +561,18 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     venc[i].n2 = b.gain(pre + "n2", dv);
     venc[i].w1 = b.matrix1(pre + "w1", d.vis_mlp, dv);
     venc[i].w2 = b.matrix1(pre + "w2", dv, d.vis_mlp);
+    if (vln) {
+      venc[i].n1b = b.gain(pre + "n1b", dv);
+      venc[i].bqkv = b.vector_heads(pre + "bqkv", {pre + "bq", pre + "bk", pre + "bv"},
+                                    {d.vis_heads, d.vis_heads, d.vis_heads}, d.vis_hd, vhs);
+      venc[i].bo = b.gain(pre + "bo", dv);
+      venc[i].n2b = b.gain(pre + "n2b", dv);
+      venc[i].b1 = b.gain(pre + "b1", d.vis_mlp);
+      venc[i].b2 = b.gain(pre + "b2", dv);
+    }
   }
   int w_vnorm = d.vis_layers > 0 ? b.gain("vis.norm", dv) : -1;
+  int w_vnorm_b = (vln && d.vis_layers > 0) ? b.gain("vis.normb", dv) : -1;
   int w_conn = d.connector ? b.matrix1("conn.w", D, (int64_t)d.shuffle * d.shuffle * dv) : -1;
   int w_emb = b.matrix1("txt.emb", d.vocab, D);
   int w_lpos = d.rope ? -1 : b.table("llm.pos", S, D);
@@ -724,11 +759,15 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
       if (w_lpos >= 0) { g.tab2 = b.wref(w_lpos, (int64_t)c * tpc); g.ldtab2 = D; }
       g.out32 = b.rows(x, (int64_t)c * tpc, tpc);
       g.out16 = b.rows(xb, (int64_t)c * tpc, tpc);
+      g.bias = w_patch_b;
       b.gemm(N_("vis%d.patch", c), b.all(patches), w_patch, dv, g);
       continue;
     }
     int xv = b.buf(N_("vis%d.x", c), T, dv, 4);
-    int xvb = b.stream_mirror(N_("vis%d.xb", c), T, dv);   // bf16 mirror of the residual stream (GEMM operand)
+    // GEMM operand of the layers: the bf16 mirror of the residual stream (RMSNorm folded into the GEMMs), or, in the
+    // LayerNorm variant, the normalised rows written by a norm node of their own
+    int xvb = vln ? -1 : b.stream_mirror(N_("vis%d.xb", c), T, dv);
+    int hv = (vln && d.vis_layers > 0) ? b.buf(N_("vis%d.h", c), T, P64(dv), 2) : -1;
     Builder::QKV vq;
     if (d.vis_layers > 0) vq = b.make_qkv(N_("vis%d.qkv", c), T, d.vis_heads, d.vis_heads, vhs);
     int vatt = d.vis_layers > 0 ? b.buf(N_("vis%d.att", c), T, P64(hvd), 2) : -1;
@@ -737,10 +776,25 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
     {
       Builder::GemmOpt g;
       g.tab = b.wref(w_vpos); g.ldtab = dv;
-      if (d.vis_layers > 0) { g.out32 = b.all(xv); g.out16 = b.all(xvb); } else g.out16 = b.all(shuf);
+      if (d.vis_layers > 0) { g.out32 = b.all(xv); if (!vln) g.out16 = b.all(xvb); } else g.out16 = b.all(shuf);
+      g.bias = w_patch_b;
       b.gemm(N_("vis%d.patch", c), b.all(patches), w_patch, dv, g);
     }
-    for (int i = 0; i < d.vis_layers; ++i) {
+    for (int i = 0; vln && i < d.vis_layers; ++i) {
+      const EncW& e = venc[i];
+      b.rmsnorm(N_("vis%d.L%d.n1", c, i), b.all(xv), e.n1, b.all(hv), 0, 1, 0, e.n1b);
+      b.qkv_project(N_("vis%d.L%d.", c, i), b.all(hv), e.wqkv, vq, d.vis_hd, -1, 0, -1, 0, e.bqkv);
+      b.attention(N_("vis%d.L%d.attn", c, i), b.rows(vq.qk, 0, T, 0), T, vq, nullptr, b.all(vatt), d.vis_heads, d.vis_heads,
+                  d.vis_hd, vhs, false);
+      Builder::GemmOpt go; go.X = b.all(xv); go.out32 = b.all(xv); go.bias = e.bo;
+      b.gemm(N_("vis%d.L%d.wo", c, i), b.all(vatt), e.wo, dv, go);
+      b.rmsnorm(N_("vis%d.L%d.n2", c, i), b.all(xv), e.n2, b.all(hv), 0, 1, 0, e.n2b);
+      Builder::GemmOpt g1; g1.act = ACT_GELU; g1.out16 = b.all(vmid); g1.bias = e.b1;
+      b.gemm(N_("vis%d.L%d.w1", c, i), b.all(hv), e.w1, d.vis_mlp, g1);
+      Builder::GemmOpt g2; g2.X = b.all(xv); g2.out32 = b.all(xv); g2.bias = e.b2;
+      b.gemm(N_("vis%d.L%d.w2", c, i), b.all(vmid), e.w2, dv, g2);
+    }
+    for (int i = 0; !vln && i < d.vis_layers; ++i) {
       // the two RMSNorms of a layer are folded into the GEMMs that consume them (A = bf16 mirror of the stream)
       b.qkv_project(N_("vis%d.L%d.", c, i), b.all(xvb), venc[i].wqkv, vq, d.vis_hd, -1, 0, venc[i].n1, dv);
       b.attention(N_("vis%d.L%d.attn", c, i), b.rows(vq.qk, 0, T, 0), T, vq, nullptr, b.all(vatt), d.vis_heads, d.vis_heads,
@@ -753,7 +807,7 @@ bool build_program(const vla_model_desc& d, const vla_runtime_opts& o, Program& 
       b.gemm(N_("vis%d.L%d.w2", c, i), b.all(vmid), venc[i].w2, dv, g2);
     }
     if (d.vis_layers > 0)
-      b.rmsnorm(N_("vis%d.norm", c), b.all(xv), w_vnorm, b.all(shuf), 0, d.shuffle, grid);
+      b.rmsnorm(N_("vis%d.norm", c), b.all(xv), w_vnorm, b.all(shuf), 0, d.shuffle, grid, w_vnorm_b);
     {
       Builder::GemmOpt g;
       if (w_lpos >= 0) { g.tab = b.wref(w_lpos, (int64_t)c * tpc); g.ldtab = D; }

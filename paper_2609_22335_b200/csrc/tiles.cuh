@@ -11,8 +11,8 @@ namespace vla {
 // A warp keeps RIF rows in flight (their loads are issued before any arithmetic), each held in registers:
 // RIF x NV float4 per lane covers widths up to 128 * NV.
 template <int RIF, int NV>
-__device__ __forceinline__ void rmsnorm_rows(const NormArgs& a, const float* xbase, const float4* g4, const float* mod,
-                                             unsigned short* out, int r0, int nrows, int lane) {
+__device__ __forceinline__ void rmsnorm_rows(const NormArgs& a, const float* xbase, const float4* g4, const float4* b4,
+                                             const float* mod, unsigned short* out, int r0, int nrows, int lane) {
   const int d4 = a.d >> 2;
   float4 v[RIF][NV];
 #pragma unroll
@@ -27,6 +27,15 @@ __device__ __forceinline__ void rmsnorm_rows(const NormArgs& a, const float* xba
 #pragma unroll
   for (int q = 0; q < RIF; ++q) {
     if (q >= nrows) break;
+    if (a.ln) {                                  // LayerNorm: centre the row first (two passes over registers)
+      float s = 0.f;
+#pragma unroll
+      for (int k = 0; k < NV; ++k) s += (v[q][k].x + v[q][k].y) + (v[q][k].z + v[q][k].w);
+      const float mu = warp_sum(s) / (float)a.d;
+#pragma unroll
+      for (int k = 0; k < NV; ++k)
+        if (lane + 32 * k < d4) { v[q][k].x -= mu; v[q][k].y -= mu; v[q][k].z -= mu; v[q][k].w -= mu; }
+    }
     float ss = 0.f;
 #pragma unroll
     for (int k = 0; k < NV; ++k) {
@@ -49,6 +58,10 @@ __device__ __forceinline__ void rmsnorm_rows(const NormArgs& a, const float* xba
       if (i >= d4) continue;
       const float4 t = v[q][k], gg = g4[i];
       float y0 = t.x * inv * gg.x, y1 = t.y * inv * gg.y, y2 = t.z * inv * gg.z, y3 = t.w * inv * gg.w;
+      if (b4) {
+        const float4 bb = b4[i];
+        y0 += bb.x; y1 += bb.y; y2 += bb.z; y3 += bb.w;
+      }
       if (mod) {
         float4 ga = reinterpret_cast<const float4*>(mod)[i], be = reinterpret_cast<const float4*>(mod + a.d)[i];
         y0 = y0 * (1.0f + ga.x) + be.x; y1 = y1 * (1.0f + ga.y) + be.y;
@@ -63,6 +76,7 @@ __device__ __forceinline__ void rmsnorm_rows(const NormArgs& a, const float* xba
 __device__ void tile_rmsnorm(const TileCtx& c, const NormArgs& a, int tile) {
   const int warp = c.tid >> 5, lane = c.tid & 31;
   const float4* g4 = reinterpret_cast<const float4*>(resolve<const float>(c, a.g));
+  const float4* b4 = reinterpret_cast<const float4*>(resolve<const float>(c, a.beta));
   const float* mod = resolve<const float>(c, a.mod);
   unsigned short* out = resolve<unsigned short>(c, a.out);
   const float* xbase = resolve<const float>(c, a.x);
@@ -72,11 +86,11 @@ __device__ void tile_rmsnorm(const TileCtx& c, const NormArgs& a, int tile) {
   const int row_lo = tile * a.rows_per_tile + warp * per_warp;
   const int row_hi = min(min(row_lo + per_warp, (tile + 1) * a.rows_per_tile), a.M);
   if (d4 <= 128) {
-    for (int r = row_lo; r < row_hi; r += 4) rmsnorm_rows<4, 4>(a, xbase, g4, mod, out, r, min(4, row_hi - r), lane);
+    for (int r = row_lo; r < row_hi; r += 4) rmsnorm_rows<4, 4>(a, xbase, g4, b4, mod, out, r, min(4, row_hi - r), lane);
   } else if (d4 <= 256) {
-    for (int r = row_lo; r < row_hi; r += 2) rmsnorm_rows<2, 8>(a, xbase, g4, mod, out, r, min(2, row_hi - r), lane);
+    for (int r = row_lo; r < row_hi; r += 2) rmsnorm_rows<2, 8>(a, xbase, g4, b4, mod, out, r, min(2, row_hi - r), lane);
   } else if (d4 <= 512) {
-    for (int r = row_lo; r < row_hi; ++r) rmsnorm_rows<1, 16>(a, xbase, g4, mod, out, r, 1, lane);
+    for (int r = row_lo; r < row_hi; ++r) rmsnorm_rows<1, 16>(a, xbase, g4, b4, mod, out, r, 1, lane);
   } else {
     // very wide rows: two passes through L2
     for (int r = row_lo; r < row_hi; ++r) {

@@ -94,13 +94,14 @@ __device__ __forceinline__ float warp_max(float v) {
 
 // ------------------------------------------------------------------ GEMM epilogue (one output element)
 struct GemmPtrs {
-  const float* X; const float* vec; const float* tab; const float* tab2;
+  const float* X; const float* vec; const float* tab; const float* tab2; const float* bias;
   float* out32; unsigned short* out16; unsigned short* outT;
 };
 __device__ __forceinline__ GemmPtrs gemm_ptrs(const TileCtx& c, const GemmArgs& g) {
   GemmPtrs p;
   p.X = resolve<const float>(c, g.X); p.vec = resolve<const float>(c, g.vec);
   p.tab = resolve<const float>(c, g.tab); p.tab2 = resolve<const float>(c, g.tab2);
+  p.bias = resolve<const float>(c, g.bias);
   p.out32 = resolve<float>(c, g.out32); p.out16 = resolve<unsigned short>(c, g.out16);
   p.outT = resolve<unsigned short>(c, g.outT);
   return p;

@@ -474,7 +474,12 @@ int vla_load_weights(vla_ctx* c, const vla_tensor* tensors, size_t n, int32_t fi
     if (!dt.is_bf16) {
       if (t.dtype != 0) return fail(c, VLA_ERR_INVALID, "tensor '%s' must be fp32", t.name);
       size_t count = s.cols == 0 ? (size_t)s.rows : (size_t)s.rows * s.cols;
-      CU(cudaMemcpy(dst, t.host_ptr, count * 4, cudaMemcpyHostToDevice));
+      if (s.cols == 0) dst += (size_t)s.row_offset * 4;        // a vector may be one part of a stacked vector
+      if (s.cols == 0 && s.group_rows > 0)                     // per-head parts, each head padded to group_stride
+        CU(cudaMemcpy2D(dst, (size_t)s.group_stride * 4, t.host_ptr, (size_t)s.group_rows * 4, (size_t)s.group_rows * 4,
+                        (size_t)(s.rows / s.group_rows), cudaMemcpyHostToDevice));
+      else
+        CU(cudaMemcpy(dst, t.host_ptr, count * 4, cudaMemcpyHostToDevice));
     } else {
       dst += (size_t)s.row_offset * dt.ld * 2;
       const void* src = t.host_ptr;

@@ -93,10 +93,13 @@ struct GemmArgs {
   int32_t ss_nft, ss_out_ld, pad_;
   Ref ss_in;                  // fp32 [M, ss_nft]: per-row sums of squares of the stream, one partial per 128 columns
   Ref ss_out;                 // optional fp32 [M, ss_out_ld]: this tile writes the partial of its 128 output features
+  Ref bias;                   // optional fp32 [N] added to the accumulator before the activation (not with dual)
 };
 
 struct NormArgs {
   Ref x, g, mod, out;  // x fp32 [M,ldx]; g fp32 [d]; mod fp32 [2d] (gamma;beta) or null; out bf16
+  Ref beta;            // LayerNorm shift fp32 [d] (ln == 1)
+  int32_t ln, pad_;    // 1: LayerNorm (subtract the row mean, biased variance, gain and shift) instead of RMSNorm
   int32_t M, d, ldx, ldo;
   int32_t rows_per_tile;
   int32_t shuffle, grid;   // shuffle s>1: row r=(y,x) of a grid x grid token map goes to row (y/s,x/s), column block (y%s,x%s)

@@ -324,6 +324,47 @@ def test_blocked_suffix_mask():
             assert not np.array_equal(got[r][n], plain[r][n])
 
 
+@pytest.mark.parametrize("key", ["cfg2s", "cfg4s"])
+def test_vision_layernorm_and_bias_variant(key):
+    """Workload variant of the vision encoder: LayerNorm with shift in place of RMSNorm and a bias on every linear layer.
+    The shifts, biases and gains are drawn large enough (std 0.5; gains in [0.5, 1.5]) that dropping any of them would
+    show.  cfg4s has 72-wide heads padded to 80 on the device, so the stacked q|k|v bias is loaded head by head."""
+    from vla_synth.configs import is_gain, is_vector
+    from vla_synth.gen import round_to_bf16
+    base = SMALL[key]
+    m = mini(base, vis_layernorm=1)
+    w = make_weights(m, seed=0)
+    rng = np.random.default_rng(11)
+    for name, shp in w.shapes.items():
+        if name.startswith("vis.") and is_vector(name):
+            v = rng.uniform(0.5, 1.5, shp) if is_gain(name) else rng.standard_normal(shp) * 0.5
+            w.override(name, round_to_bf16(v.astype(np.float32)))
+    frames = [[frame_inputs(m, r, n, seed=0) for n in range(2)] for r in range(2)]
+    got, _ = _run(m, w, frames, "cosched")
+    worst = _check_vs_oracle(m, w, frames, got)
+    print(f"vision LayerNorm+bias {key}: worst rel-L2 {worst[0]:.2e}, max-abs {worst[1]:.3e}")
+    ser, _ = _run(m, w, frames, "serial")
+    two, _ = _run(m, w, frames, "two_stream")
+    for r in range(2):
+        for n in range(2):
+            assert np.array_equal(got[r][n], ser[r][n])
+            assert np.array_equal(got[r][n], two[r][n])
+    # every shift and bias reaches the chunk: zeroing one kind at a time changes it (the key bias is the exception,
+    # the softmax cancels it, so there the chunk must stay within rounding of the original)
+    if key == "cfg2s":
+        for leaf in ("n1b", "bq", "bv", "bo", "b1", "b2", "normb", "bk"):
+            w2 = make_weights(m, seed=0)
+            for name in w.shapes:
+                if name in w._override:
+                    w2.override(name, np.zeros_like(w[name]) if name.split(".")[-1] == leaf else w[name])
+            other, _ = _run(m, w2, frames[:1], "cosched")
+            d = float(np.max(np.abs(other[0][0] - got[0][0])))
+            if leaf == "bk":
+                assert d < 3e-2, (leaf, d)
+            else:
+                assert d > 1e-3, (leaf, d)
+
+
 def test_classifier_free_guidance():
     """Workload variant of the in-context DiT head (head D, DDIM): two head evaluations per step, unconditional then
     conditional, combined in the solver epilogue.  Against the oracle, across modes; scale 1 reproduces the unguided

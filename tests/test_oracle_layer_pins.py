@@ -149,6 +149,88 @@ def test_vision_encoder_layer_composition():
     assert max(lg) - min(lg) > 1.0
 
 
+def layer_norm(x, g, b):
+    n = len(x)
+    mu = sum(x) / n
+    var = sum((v - mu) ** 2 for v in x) / n
+    return [(x[i] - mu) / math.sqrt(var + 1e-6) * g[i] + b[i] for i in range(n)]
+
+
+def test_layernorm_against_its_textbook_properties():
+    rng = np.random.default_rng(7)
+    x = rng.standard_normal((5, 16)) * 3.0 + 2.0
+    ones, zeros = np.ones(16), np.zeros(16)
+    y = O.layernorm(x, ones, zeros)
+    assert np.allclose(y.mean(axis=-1), 0.0, atol=1e-12)
+    assert np.allclose((y * y).mean(axis=-1), 1.0, atol=1e-6)             # unit variance up to the epsilon
+    assert np.allclose(O.layernorm(x + 11.5, ones, zeros), y, atol=1e-9)  # a shift of the row changes nothing
+    assert np.allclose(O.layernorm(4.0 * x, ones, zeros), y, atol=1e-6)   # nor does a positive scale
+    g, b = rng.uniform(0.5, 1.5, 16), rng.standard_normal(16)
+    close(O.layernorm(x, g, b), [layer_norm(r, L(g), L(b)) for r in L(x)])
+    xc = x - x.mean(axis=-1, keepdims=True)                               # on a centred row it is RMSNorm plus the shift
+    close(O.layernorm(xc, g, b), O.rmsnorm(xc, g) + b)
+
+
+def test_vision_encoder_layer_with_layernorm_and_biases():
+    rng = np.random.default_rng(202)
+    T, d, heads, hd, mlp = 5, 12, 2, 8, 20
+    p = "vis.L0."
+    w = {p + "n1": rng.uniform(0.5, 1.5, d), p + "n2": rng.uniform(0.5, 1.5, d),
+         p + "n1b": rng.standard_normal(d) * 0.5, p + "n2b": rng.standard_normal(d) * 0.5,
+         p + "wq": rng.standard_normal((heads * hd, d)), p + "wk": rng.standard_normal((heads * hd, d)),
+         p + "wv": rng.standard_normal((heads * hd, d)) * 0.5, p + "wo": rng.standard_normal((d, heads * hd)) * 0.3,
+         p + "w1": rng.standard_normal((mlp, d)) * 0.5, p + "w2": rng.standard_normal((d, mlp)) * 0.3,
+         p + "bq": rng.standard_normal(heads * hd), p + "bk": rng.standard_normal(heads * hd),
+         p + "bv": rng.standard_normal(heads * hd), p + "bo": rng.standard_normal(d),
+         p + "b1": rng.standard_normal(mlp), p + "b2": rng.standard_normal(d)}
+    x = rng.standard_normal((T, d)) + 1.5                      # rows with a mean: RMSNorm in its place would differ
+    got = O._encoder_layer_ln(x.copy(), w, p, heads, hd, F64)
+
+    W = {k: L(v) for k, v in w.items()}
+    xs = L(x)
+    h = [layer_norm(r, W[p + "n1"], W[p + "n1b"]) for r in xs]
+    q = [heads_of(add(matvec(W[p + "wq"], r), W[p + "bq"]), heads, hd) for r in h]
+    k = [heads_of(add(matvec(W[p + "wk"], r), W[p + "bk"]), heads, hd) for r in h]
+    v = [heads_of(add(matvec(W[p + "wv"], r), W[p + "bv"]), heads, hd) for r in h]
+    a = mha(q, k, v, heads, heads, hd)
+    xs = [add(add(xs[t], matvec(W[p + "wo"], a[t])), W[p + "bo"]) for t in range(T)]
+    h2 = [layer_norm(r, W[p + "n2"], W[p + "n2b"]) for r in xs]
+    want = []
+    for t in range(T):
+        mid = [gelu(u) for u in add(matvec(W[p + "w1"], h2[t]), W[p + "b1"])]      # bias BEFORE the activation
+        want.append(add(add(xs[t], matvec(W[p + "w2"], mid)), W[p + "b2"]))
+    close(got, want)
+    # every bias and shift matters: zeroing any one of them changes the layer's output
+    for name in ("n1b", "n2b", "bq", "bk", "bv", "bo", "b1", "b2"):
+        w2 = dict(w)
+        w2[p + name] = np.zeros_like(w[p + name])
+        other = O._encoder_layer_ln(x.copy(), w2, p, heads, hd, F64)
+        if name == "bk":
+            # a key bias adds q.bk to EVERY logit of a query's row, which the softmax cancels: the output must not move
+            assert np.allclose(other, got, atol=1e-9)
+        else:
+            assert np.max(np.abs(other - got)) > 1e-3, name
+
+
+def test_vision_tokens_layernorm_variant_adds_patch_bias_and_final_shift():
+    m = mini(CFG2, n_cam=1, img=28, patch=14, vis_layers=1, vis_d=12, vis_heads=2, vis_hd=8, vis_mlp=20, shuffle=1,
+             vis_layernorm=1, d=12, n_text=2, vocab=8, llm_layers=1)
+    rng = np.random.default_rng(5)
+    w = random_weights(m, rng, only="vis.")
+    if "conn.w" in weight_shapes(m):
+        w["conn.w"] = rng.standard_normal(weight_shapes(m)["conn.w"]) * 0.3
+    img = rng.standard_normal((1, 3, 28, 28))
+    got = O.vision_tokens(m, w, img, F64)
+    # restated: patch rows -> embedding + bias + positions -> one LN layer -> final LN -> connector (if any)
+    pt = O.patchify(img, m.patch)[0]
+    xs = [add(add(matvec(L(w["vis.patch.w"]), r), L(w["vis.patch.b"])), prow) for r, prow in zip(L(pt), L(w["vis.pos"]))]
+    xs = O._encoder_layer_ln(np.array(xs), w, "vis.L0.", m.vis_heads, m.vis_hd, F64)     # pinned above
+    xs = [layer_norm(r, L(w["vis.norm"]), L(w["vis.normb"])) for r in L(xs)]
+    if "conn.w" in w:
+        xs = [matvec(L(w["conn.w"]), r) for r in xs]
+    close(got, xs)
+
+
 # ------------------------------------------------------------------ LLM decoder layer
 LLM_CASES = {
     # GQA + RoPE + causal + SwiGLU (the Llama-style prefix decoder)

@@ -62,6 +62,8 @@ class ModelDesc:
     n_streams: int
     n_frames: int
     # ---- workload variants (defaults: the five stated workloads)
+    vis_layernorm: int = 0  # vision encoder: 1 = LayerNorm (gain and shift) instead of RMSNorm, and a bias vector on every
+                            # linear layer of the encoder (patch embedding, q, k, v, o, both MLP layers)
     guidance: float = 0.0   # head D: classifier-free guidance scale s (0 = off): eps = eps_u + s (eps_c - eps_u), the
                             # unconditional branch built from a zero cognition feature
     suffix_mask: int = 0    # head B: 1 = blocked suffix mask -- the leading state token attends the prefix and itself
@@ -212,7 +214,10 @@ def weight_shapes(m: ModelDesc) -> "OrderedDict[str, tuple]":
     """
     w: "OrderedDict[str, tuple]" = OrderedDict()
     dv = m.vis_d
+    ln = bool(getattr(m, "vis_layernorm", 0))
     w["vis.patch.w"] = (dv, m.patch_k)
+    if ln:
+        w["vis.patch.b"] = (dv,)
     w["vis.pos"] = (m.vis_tokens, dv)
     hv = m.vis_heads * m.vis_hd
     for i in range(m.vis_layers):
@@ -225,8 +230,13 @@ def weight_shapes(m: ModelDesc) -> "OrderedDict[str, tuple]":
         w[p + "n2"] = (dv,)
         w[p + "w1"] = (m.vis_mlp, dv)
         w[p + "w2"] = (dv, m.vis_mlp)
+        if ln:
+            for leaf, n in (("n1b", dv), ("bq", hv), ("bk", hv), ("bv", hv), ("bo", dv), ("n2b", dv), ("b1", m.vis_mlp), ("b2", dv)):
+                w[p + leaf] = (n,)
     if m.vis_layers > 0:
         w["vis.norm"] = (dv,)
+        if ln:
+            w["vis.normb"] = (dv,)
     if m.connector:
         w["conn.w"] = (m.d, m.shuffle * m.shuffle * dv)
     w["txt.emb"] = (m.vocab, m.d)
@@ -297,6 +307,12 @@ def weight_shapes(m: ModelDesc) -> "OrderedDict[str, tuple]":
     w["act.norm"] = (da,)
     w["act.out"] = (m.act_dim, da)
     return w
+
+
+def is_vector(name: str) -> bool:
+    """fp32 vectors of the weight table: norm gains, LayerNorm shifts and the biases of linear layers."""
+    leaf = name.split(".")[-1]
+    return is_gain(name) or leaf in ("n1b", "n2b", "normb", "bq", "bk", "bv", "bo", "b1", "b2", "b")
 
 
 def is_gain(name: str) -> bool:
