@@ -57,6 +57,38 @@ def test_full_size_sampled_parity(m, frames, check_two_stream):
                 assert np.array_equal(got[r][n], got2[r][n]), (m.name, r, n)
 
 
+# (The blocked suffix mask on the full pi0-shaped model and classifier-free guidance on the full CogACT-shaped one pass the
+# same test -- rel-L2 1.6e-3 / 2.7e-3 -- but the oracle needs minutes for them; they stay covered at reduced size.)
+@pytest.mark.parametrize("base,variant", [(CFG2, {"vis_layernorm": 1})], ids=["cfg2_vision_layernorm_bias"])
+def test_full_size_workload_variants(base, variant):
+    """The workload variants at full model size (four request streams, one frame each; one chunk against the oracle,
+    all chunks bit-identical between the co-scheduled and the serial run)."""
+    from paper_2609_22335_b200 import Engine
+    from vla_synth.configs import mini
+    m = mini(base, **variant)
+    w = make_weights(m, seed=0, cache=False)
+    R = 4
+    fr = [[frame_inputs(m, r, 0, seed=0)] for r in range(R)]
+    outs = {}
+    for mode in ("cosched", "serial"):
+        eng = Engine(m, mode=mode, n_streams=R)
+        try:
+            eng.load_weights(w)
+            outs[mode] = eng.run(fr, timeout_s=900)
+        finally:
+            eng.close()
+    for r in range(R):
+        assert np.array_equal(outs["cosched"][r][0], outs["serial"][r][0]), (m.name, r)
+    ref = O.action_chunk(m, w, fr[R - 1][0], np.float32)
+    got = outs["cosched"][R - 1][0]
+    rel = float(np.linalg.norm(got - ref) / np.linalg.norm(ref))
+    mx = float(np.max(np.abs(got - ref)))
+    rms = float(np.sqrt(np.mean(ref * ref)))
+    print(f"{m.name} {variant}: rel-L2 {rel:.2e}, max-abs {mx:.3e}, chunk rms {rms:.2f}")
+    scale = max(1.0, rms) if m.solver == "ddim" else 1.0
+    assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL * scale, (m.name, rel, mx, rms)
+
+
 def test_full_size_trace_respects_the_dag():
     """32 request streams x 3 frames of the SmolVLA-shaped workload, co-scheduled, with the device trace on: every
     one of the 2.6 million tiles ran exactly once, after its frame's admission and after all tiles of its
