@@ -215,6 +215,95 @@ def gap_stats(trace) -> dict:
     return out
 
 
+def _node_instance_spans(t):
+    """Per executed node instance (request-stream slot, frame, node): key, first start, last end, tiles seen."""
+    key = t["inst"].astype(np.int64) << 40 | t["frame"].astype(np.int64) % (1 << 19) << 21 | t["node"].astype(np.int64)
+    order = np.argsort(key, kind="stable")
+    k, s, e = key[order], t["t_start"][order].astype(np.int64), t["t_end"][order].astype(np.int64)
+    first = np.flatnonzero(np.r_[True, k[1:] != k[:-1]])
+    return k[first], np.minimum.reduceat(s, first), np.maximum.reduceat(e, first), np.diff(np.r_[first, len(k)])
+
+
+def backlog_stats(trace, program, n_workers: int) -> dict:
+    """Was there work for the idle workers?  (Starvation against dispatch latency.)
+
+    A tile is READY from the moment the last tile of the last predecessor node of its frame has ended (for a node
+    without predecessors: from the frame's admission) and WAITS until it starts.  The backlog at time t is the number of
+    ready tiles that have not started.  Reported: how long a tile waits once ready (by phase), the time-weighted mean
+    backlog, and -- the figure that tells the two causes of idle workers apart -- the share of the worker-idle time
+    (between a worker's tiles) during which the backlog was empty (nothing to run anywhere: the dependency chains are
+    the limit) against non-empty (tiles were ready, but claim, hand-over and room had not caught up)."""
+    t = tiles_only(trace)
+    if len(t) == 0:
+        return {}
+    adm = trace[trace["node"] == ADMIT_NODE]
+    key, span_s, span_e, seen = _node_instance_spans(t)
+    node = (key & ((1 << 21) - 1)).astype(np.int64)
+    inst_frame = key >> 21
+    n_nodes = len(program)
+    # ready time of every executed node instance: admission of its frame, then the ends of its predecessors
+    ready = np.zeros(len(key), dtype=np.int64)
+    if len(adm):
+        akey = adm["inst"].astype(np.int64) << 19 | adm["frame"].astype(np.int64) % (1 << 19)
+        ao = np.argsort(akey, kind="stable")
+        pos = np.clip(np.searchsorted(akey[ao], inst_frame), 0, len(ao) - 1)
+        hit = akey[ao][pos] == inst_frame
+        ready = np.where(hit, adm["t_start"][ao][pos].astype(np.int64), span_s)     # (no marker: never earlier than its start)
+    else:
+        ready = span_s.copy()
+    index = {int(k): i for i, k in enumerate(key)}
+    preds = [[] for _ in range(n_nodes)]
+    for u, n in enumerate(program):
+        for v in n["succ"]:
+            preds[v].append(u)
+    for i in range(len(key)):
+        base = int(inst_frame[i]) << 21
+        for u in preds[int(node[i])]:
+            j = index.get(base | u)
+            if j is not None and span_e[j] > ready[i]:
+                ready[i] = span_e[j]
+    # per tile: the wait between ready and start
+    tkey = t["inst"].astype(np.int64) << 40 | t["frame"].astype(np.int64) % (1 << 19) << 21 | t["node"].astype(np.int64)
+    pos = np.searchsorted(key, tkey)
+    t_ready = ready[pos]
+    ts = t["t_start"].astype(np.int64)
+    wait = np.maximum(ts - t_ready, 0).astype(np.float64)
+    ph = t["cls"] // N_KINDS
+    out = {"wait_ready_to_start_us": {nm: {"mean": float(wait[ph == q].mean() * 1e-3), "median": float(np.median(wait[ph == q]) * 1e-3),
+                                             "p90": float(np.percentile(wait[ph == q], 90) * 1e-3)}
+                                      for q, nm in ((0, "vlm"), (1, "head")) if (ph == q).any()}}
+    # backlog(t): +1 per tile at its ready time, -1 at its start
+    ev_t = np.concatenate([t_ready, ts])
+    ev_d = np.concatenate([np.ones(len(ts), dtype=np.int64), -np.ones(len(ts), dtype=np.int64)])
+    o = np.lexsort((ev_d, ev_t))          # at equal times the starts (-1) come first: never a phantom backlog
+    ev_t, backlog = ev_t[o], np.cumsum(ev_d[o])
+    dt = np.diff(ev_t).astype(np.float64)
+    if dt.sum() > 0:
+        out["mean_backlog_tiles"] = float((backlog[:-1] * dt).sum() / dt.sum())
+    # idle intervals of the workers, split by whether tiles were ready meanwhile (sampled at 4 points per gap)
+    wk = t["sm"].astype(np.int64) * 256 + t["worker"]
+    order = np.lexsort((t["t_start"], wk))
+    k2, s2, e2 = wk[order], ts[order], t["t_end"][order].astype(np.int64)
+    same = k2[1:] == k2[:-1]
+    g0, g1 = e2[:-1][same], s2[1:][same]
+    keep = g1 > g0
+    g0, g1 = g0[keep], g1[keep]
+    if len(g0):
+        length = (g1 - g0).astype(np.float64)
+        empty = np.zeros(len(g0)); few = np.zeros(len(g0))
+        for f in (0.125, 0.375, 0.625, 0.875):
+            at = g0 + (length * f).astype(np.int64)
+            b = backlog[np.clip(np.searchsorted(ev_t, at, side="right") - 1, 0, len(backlog) - 1)]
+            empty += (b <= 0) * 0.25
+            few += ((b > 0) & (b < n_workers // 8)) * 0.25
+        tot = length.sum()
+        out["idle_between_tiles"] = {"share_with_empty_backlog": float((empty * length).sum() / tot),
+                                     "share_with_short_backlog": float((few * length).sum() / tot),
+                                     "share_with_deep_backlog": float(((1.0 - empty - few) * length).sum() / tot),
+                                     "short_backlog_means_fewer_than": int(n_workers // 8)}
+    return out
+
+
 def summary(trace, program=None, n_sms: int | None = None, workers_per_sm: int = 3) -> dict:
     """Everything the benchmark line reports from one traced pass."""
     n_workers = (n_sms * workers_per_sm) if n_sms else None
@@ -224,4 +313,6 @@ def summary(trace, program=None, n_sms: int | None = None, workers_per_sm: int =
     if program is not None and n_workers:
         out["per_class"] = per_class_rates(trace, program, n_workers)
         out["smaller_side_of_concurrent_node_pairs"] = smaller_side_of_concurrent_pairs(trace, program)
+        if all("succ" in n for n in program):
+            out["backlog"] = backlog_stats(trace, program, n_workers)
     return out

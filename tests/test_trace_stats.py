@@ -80,3 +80,21 @@ def test_gap_stats():
     assert g["all"]["gaps"] == 3 and abs(g["all"]["mean_us"] - 10 / 3 * 1e-3) < 1e-12
     assert g["head_gemm"]["gaps"] == 2 and abs(g["head_gemm"]["mean_us"] - 5e-3) < 1e-12 and g["head_gemm"]["share_of_idle"] == 1.0
     assert g["vlm_gemm"]["gaps"] == 1 and g["vlm_gemm"]["mean_us"] == 0.0
+
+
+def test_backlog_stats_hand_case():
+    # node 0 (two tiles) -> node 1 (one tile); the frame is admitted at t = 0
+    program = [{"n_tiles": 2, "phase": 0, "succ": [1]}, {"n_tiles": 1, "phase": 1, "succ": []}]
+    tr = _trace([(0, 0, 0, TS.ADMIT_NODE, 0, 0, 0, 0),
+                 (0, 0, 0, 0, 10, 50, 0, 0), (0, 1, 0, 0, 10, 30, 0, 0),     # node 0: ready at 0, both tiles start at 10
+                 (0, 1, 4, 1, 60, 80, 0, 0)])                                # node 1: ready at 50 (last end of node 0), starts at 60
+    b = TS.backlog_stats(tr, program, n_workers=2)
+    assert b["wait_ready_to_start_us"]["vlm"]["mean"] == 10e-3 and b["wait_ready_to_start_us"]["head"]["mean"] == 10e-3
+    # backlog: 2 tiles over [0,10), none over [10,50), 1 over [50,60) -> (20 + 10) / 60
+    assert abs(b["mean_backlog_tiles"] - 30 / 60) < 1e-12
+    # the one idle interval, worker (0,1) from 30 to 60: nothing was ready until 50 (three of the four sample points)
+    idle = b["idle_between_tiles"]
+    assert abs(idle["share_with_empty_backlog"] - 0.75) < 1e-12 and abs(idle["share_with_deep_backlog"] - 0.25) < 1e-12
+    # and the summary carries it when the program lists successors
+    s = TS.summary(tr, [dict(p, flops=0.0, weight_bytes=0.0) for p in program], n_sms=1, workers_per_sm=2)
+    assert "backlog" in s
