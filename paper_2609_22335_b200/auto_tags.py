@@ -36,7 +36,7 @@ def quantise(u: float) -> int:
     return max(0, min(TAU_MAX, int(round(TAU_MAX * u))))
 
 
-def ncu_command(config: str, csv_path: str = "gpurun_out/auto_tags_launches.csv") -> str:
+def ncu_command(config: str, csv_path: str = "auto_tags_launches.csv") -> str:
     return ("ncu --metrics " + ",".join(METRICS) + " --clock-control none -k regex:" + KERNEL +
             f" --csv --log-file {csv_path} python -m paper_2609_22335_b200.auto_tags run --config {config}")
 
@@ -133,8 +133,8 @@ def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
     ap.add_argument("what", choices=["command", "run", "derive"])
     ap.add_argument("--config", default="cfg2")
-    ap.add_argument("--csv", default="gpurun_out/auto_tags_launches.csv")
-    ap.add_argument("--program", default="gpurun_out/auto_tags_program.json")
+    ap.add_argument("--csv", default="auto_tags_launches.csv")
+    ap.add_argument("--program", default="auto_tags_program.json")
     ap.add_argument("--relative", action="store_true", help="scale every pipeline so that its heaviest class gets 15")
     a = ap.parse_args(argv)
     if a.what == "command":
